@@ -1,0 +1,186 @@
+/*
+ * libmpipe_enc -- the data-parallel computation that the Mpipe "transpose" schedule relocates,
+ * written for NVIDIA B200 (sm_100a).
+ *
+ * Under the schedule <transpose, 1f1b> (Section 4.2, "Instantiation") the modality encoder is a
+ * Replicated region: every pipeline rank runs whole encoder microbatches, Fwd(enc, r, m) inside its
+ * warm-up bubble and -- only if the encoder is trainable -- Bwd(enc, r, m) in the cool-down; the
+ * encoder output then crosses the Replicated->Sharded seam of Table 2 ("Gather") into the first LLM
+ * stage.  This library provides the kernels of that region's attention and of the local half of the
+ * seam, over packed variable-length image-patch sequences (Section 2: resolutions, clip lengths and
+ * pure-text samples vary from microbatch to microbatch):
+ *
+ *   mpipe_seg_plan          patch counts -> cu_seqlens + longest-first tile work-lists   (host, integers)
+ *   mpipe_varlen_attn_fwd   per-image softmax attention, O and (if trained) row LSE      (device)
+ *   mpipe_varlen_attn_bwd   dQ, dK, dV; a no-op when the encoder is frozen               (device)
+ *   mpipe_merge_tokens      encoder tokens -> their placeholder rows of the LLM input    (device)
+ *   mpipe_merge_tokens_bwd  gradient rows at the placeholders -> encoder; no-op if frozen (device)
+ *
+ * Conventions
+ *   - Plain C ABI.  Every call returns an mpipe_status_t as int32_t; nothing throws or aborts.
+ *   - "host" / "device" is stated for every pointer.  The caller owns all memory, the workspace and
+ *     the CUDA stream; the library allocates no device memory.  Device calls enqueue work on `stream`
+ *     (a cudaStream_t passed as void*, NULL = default stream) and return without synchronising.
+ *   - Argument errors are detected on the host before anything is launched; outputs are untouched.
+ *   - bf16 = bfloat16.  Token tensors are [tokens, heads, head_dim] with explicit token and head
+ *     strides in ELEMENTS; head_dim is contiguous.  Base pointers must be 16-byte aligned and the
+ *     strides multiples of 8 elements (TMA needs 16-byte aligned global strides).
+ *   - `status_buf` (device int32[4], optional, zeroed by the caller) receives device-side findings:
+ *     [0] = first non-zero mpipe_status_t seen by a kernel, [1] = detail (e.g. offending index),
+ *     [2], [3] reserved.  Kernels never trap: a bounded wait that expires or an out-of-range index
+ *     sets this word, skips the offending work and returns.
+ *   - mode mirrors trainable(enc) of the paper's derive(): MPIPE_ENC_FROZEN deletes every optional
+ *     backward event (Lemma 1 and the "same schedule, two footprints" paragraph of Section 4.2);
+ *     the forward results are bit-identical in both modes (Corollary 1).
+ */
+#ifndef MPIPE_ENC_H_
+#define MPIPE_ENC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MPIPE_OK = 0,
+    MPIPE_ERR_INVALID_ARG = 1, /* NULL / negative / misaligned / inconsistent argument            */
+    MPIPE_ERR_UNSUPPORTED = 2, /* head_dim not in {64, 80}, tile_rows not a supported value       */
+    MPIPE_ERR_WORKSPACE = 3,   /* workspace NULL or smaller than mpipe_attn_workspace_bytes()     */
+    MPIPE_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (launch, tensor-map encode) */
+    MPIPE_ERR_TIMEOUT = 5,     /* device: a bounded wait expired (reported through status_buf)    */
+    MPIPE_ERR_INDEX = 6        /* device: merge position out of range (reported via status_buf)   */
+} mpipe_status_t;
+
+/* trainable(enc): the one model bit derive() reads for the encoder region (Section 4.2). */
+typedef enum { MPIPE_ENC_FROZEN = 0, MPIPE_ENC_TRAINED = 1 } mpipe_enc_mode_t;
+
+/* One tile of one segment.  Forward items tile the QUERY rows of a segment (rows = queries, kv_* =
+ * the segment's whole key range); backward items tile the KEY/VALUE rows (rows = keys, kv_* = the
+ * segment's whole query range, which is the same token range).  Heads are not listed: kernels
+ * iterate item x head. */
+typedef struct {
+    int32_t seg;       /* segment (image / clip) index                      */
+    int32_t tile;      /* tile index inside the segment                     */
+    int32_t row_start; /* first packed row of the tile                      */
+    int32_t row_len;   /* rows in the tile, 1..tile_rows                    */
+    int32_t kv_start;  /* first packed row of the segment (= cu_seqlens[seg]) */
+    int32_t kv_len;    /* tokens in the segment                             */
+} mpipe_work_item_t;
+
+/* Native tile heights of the kernels in this build (rows per work item). */
+int32_t mpipe_fwd_tile_rows(void);
+int32_t mpipe_bwd_tile_rows(void);
+
+/*
+ * (1) Segment planner -- host, integer only.  Not in the paper beyond the observation that the
+ * encoder's work is known before the LLM pipeline starts (Section 1) and that the static schedule
+ * has no run-time scheduling cost; it has to cost microseconds.
+ *
+ *   cu_seqlens[0] = 0, cu_seqlens[i+1] = cu_seqlens[i] + patch_counts[i];  *total_tokens = cu[n_seg];
+ *   *max_seqlen = max patch count (0 if none).
+ *   Items: segments ordered by patch count descending, ties by index ascending; empty segments
+ *   (pure-text samples) are skipped; per segment tiles t = 0.. in order:
+ *     { seg, t, cu[seg] + t*tile_rows, min(tile_rows, n - t*tile_rows), cu[seg], n }.
+ *   Forward items use fwd_tile_rows, backward items bwd_tile_rows.  FROZEN => *n_bwd_items = 0.
+ *
+ * Two-call pattern: with fwd_items == NULL (resp. bwd_items == NULL) only the counts are written.
+ * All pointers are HOST pointers.  cu_seqlens has room for n_seg + 1 entries.  patch_counts may be
+ * NULL iff n_seg == 0.  Errors: negative count or n_seg, total >= 2^31, tile_rows <= 0, NULL outputs
+ * -> MPIPE_ERR_INVALID_ARG.
+ */
+int32_t mpipe_seg_plan(const int32_t* patch_counts, int32_t n_seg, int32_t fwd_tile_rows, int32_t bwd_tile_rows,
+                       int32_t mode, int32_t* cu_seqlens, int32_t* total_tokens, int32_t* max_seqlen,
+                       mpipe_work_item_t* fwd_items, int32_t* n_fwd_items, mpipe_work_item_t* bwd_items,
+                       int32_t* n_bwd_items);
+
+/* Bytes of device workspace mpipe_varlen_attn_bwd needs (0 when FROZEN): an fp32 dQ accumulator
+ * [tokens, heads, head_dim] and the fp32 row terms Delta [heads, tokens], each rounded up to 256 B. */
+size_t mpipe_attn_workspace_bytes(int32_t total_tokens, int32_t n_heads, int32_t head_dim, int32_t mode);
+
+/*
+ * (2) Fwd(enc) attention (the relocated forward event of Section 4.2).  For every segment s with
+ * packed rows [a, b) = [cu[s], cu[s+1]) and every head h, with S = softmax_scale * Q K^T restricted
+ * to the segment (bidirectional, no mask inside it, nothing across segments):
+ *     O[i,h,:] = sum_j softmax_j(S_ij) V[j,h,:],     LSE[h,i] = ln sum_j exp(S_ij).
+ *
+ *   q, k, v   device, bf16 [total_tokens, n_heads, head_dim], strides tok_stride_qkv / head_stride_qkv
+ *   o         device, bf16, same shape, strides tok_stride_o / head_stride_o              (output)
+ *   lse       device, fp32 [n_heads, total_tokens] contiguous; written only when TRAINED (required
+ *             then); ignored when FROZEN                                                  (output)
+ *   cu_seqlens_dev   device int32[n_seg + 1]   (copy of the plan; validated on the host side only
+ *                    through the items, which carry the same ranges)
+ *   fwd_items_dev    device mpipe_work_item_t[n_fwd_items] from mpipe_seg_plan with
+ *                    fwd_tile_rows = mpipe_fwd_tile_rows()
+ *   total_tokens == 0 or n_fwd_items == 0: returns MPIPE_OK without launching.
+ * Rows past a segment's end inside a tile are computed but never stored.  fp32 accumulation,
+ * bf16 probabilities; results are deterministic run to run.
+ */
+int32_t mpipe_varlen_attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
+                              int64_t tok_stride_qkv, int64_t head_stride_qkv, int64_t tok_stride_o,
+                              int64_t head_stride_o, const int32_t* cu_seqlens_dev, int32_t n_seg,
+                              int32_t total_tokens, int32_t max_seqlen, const mpipe_work_item_t* fwd_items_dev,
+                              int32_t n_fwd_items, int32_t n_heads, int32_t head_dim, float softmax_scale,
+                              int32_t mode, int32_t* status_buf, void* stream);
+
+/*
+ * (3) Bwd(enc)? attention -- exists only when trainable(enc) (Lemma 1).  FROZEN: returns MPIPE_OK at
+ * once, launches nothing, touches nothing.  TRAINED, per segment and head, with P = exp(S - LSE):
+ *     Delta_i = sum_d dO[i,d] O[i,d];  dV = P^T dO;  dP = dO V^T;  dS = P o (dP - Delta);
+ *     dQ = softmax_scale * dS K;       dK = softmax_scale * dS^T Q.
+ *
+ *   dout, o   device bf16 (o strides);  q, k, v device bf16 (qkv strides);  lse device fp32 [H, T]
+ *   dq, dk, dv device bf16, strides tok_stride_grad / head_stride_grad                    (outputs)
+ *   bwd_items_dev  from mpipe_seg_plan with bwd_tile_rows = mpipe_bwd_tile_rows()
+ *   workspace      device, >= mpipe_attn_workspace_bytes(...), 256-byte aligned; contents are scratch
+ * dQ is accumulated with fp32 atomics across key tiles: its low bits may differ run to run.
+ */
+int32_t mpipe_varlen_attn_bwd(const void* dout, const void* q, const void* k, const void* v, const void* o,
+                              const float* lse, void* dq, void* dk, void* dv, int64_t tok_stride_qkv,
+                              int64_t head_stride_qkv, int64_t tok_stride_o, int64_t head_stride_o,
+                              int64_t tok_stride_grad, int64_t head_stride_grad, const int32_t* cu_seqlens_dev,
+                              int32_t n_seg, int32_t total_tokens, int32_t max_seqlen,
+                              const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items, int32_t n_heads,
+                              int32_t head_dim, float softmax_scale, int32_t mode, void* workspace,
+                              size_t workspace_bytes, int32_t* status_buf, void* stream);
+
+/*
+ * (4) Local half of Coll(Gather, (enc, llm), m), the Replicated->Sharded seam of Table 2: encoder
+ * token i is written over row positions[i] of the LLM input-embedding buffer, in place:
+ *     llm_embeds[positions[i], 0:hidden] = enc_tokens[i, 0:hidden].
+ * The forward seam is not gated by trainability, so `mode` is accepted and ignored.
+ *
+ *   enc_tokens  device bf16 [n_enc_tokens, hidden], row stride enc_row_stride elements
+ *   llm_embeds  device bf16 [n_llm_tokens, hidden], row stride emb_row_stride elements   (in/out)
+ *   positions_dev device int32[n_enc_tokens]; must be unique (precondition; see
+ *               mpipe_validate_positions).  An index outside [0, n_llm_tokens) is skipped and
+ *               reported as MPIPE_ERR_INDEX in status_buf.
+ *   hidden must be a multiple of 8 and both buffers 16-byte aligned with strides multiples of 8.
+ *   n_enc_tokens == 0: MPIPE_OK, nothing launched.
+ */
+int32_t mpipe_merge_tokens(const void* enc_tokens, int64_t enc_row_stride, void* llm_embeds, int64_t emb_row_stride,
+                           const int32_t* positions_dev, int32_t n_enc_tokens, int32_t n_llm_tokens, int32_t hidden,
+                           int32_t mode, int32_t* status_buf, void* stream);
+
+/*
+ * Local half of the reverse seam Coll(Scatter, (enc, llm), m)?, which fires only when some region
+ * before the LLM is trainable (Lemma 1, gate (i)):  d_enc[i, :] = d_llm_embeds[positions[i], :].
+ * FROZEN: returns MPIPE_OK at once and touches nothing.  Same layout rules as mpipe_merge_tokens;
+ * d_enc is the output.
+ */
+int32_t mpipe_merge_tokens_bwd(const void* d_llm_embeds, int64_t emb_row_stride, void* d_enc, int64_t enc_row_stride,
+                               const int32_t* positions_dev, int32_t n_enc_tokens, int32_t n_llm_tokens,
+                               int32_t hidden, int32_t mode, int32_t* status_buf, void* stream);
+
+/* Host helper: checks that HOST positions[0..n) are unique and inside [0, n_llm_tokens).
+ * Returns MPIPE_OK, MPIPE_ERR_INDEX (out of range) or MPIPE_ERR_INVALID_ARG (duplicate / NULL). */
+int32_t mpipe_validate_positions(const int32_t* positions, int32_t n, int32_t n_llm_tokens);
+
+const char* mpipe_status_str(int32_t status);
+int32_t mpipe_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MPIPE_ENC_H_ */

@@ -1,0 +1,230 @@
+"""ctypes binding of libmpipe_enc.so: argument marshalling only.
+
+Every function has the name of the C entry point without the ``mpipe_`` prefix and forwards
+to it; all arithmetic of the hot path runs in the CUDA kernels behind the C ABI
+(``include/mpipe_enc.h``).  torch is used for device memory and streams only.  There is no
+CPU fallback: if the shared library is missing the import of this module's functions fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmpipe_enc.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_INDEX = range(7)
+FROZEN, TRAINED = 0, 1
+
+_lib = None
+
+
+class WorkItem(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("seg", "tile", "row_start", "row_len", "kv_start", "kv_len")]
+
+
+ITEM_DTYPE = np.dtype([(n, np.int32) for n in ("seg", "tile", "row_start", "row_len", "kv_start", "kv_len")])
+
+_i32, _i64, _vp, _f32, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float, ctypes.c_size_t
+_SIGNATURES = {
+    "mpipe_fwd_tile_rows": (_i32, []),
+    "mpipe_bwd_tile_rows": (_i32, []),
+    "mpipe_seg_plan": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "mpipe_attn_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32]),
+    "mpipe_varlen_attn_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _vp, _i32, _i32, _i32, _vp,
+                                     _i32, _i32, _i32, _f32, _i32, _vp, _vp]),
+    "mpipe_varlen_attn_bwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _i64, _i64,
+                                     _vp, _i32, _i32, _i32, _vp, _i32, _i32, _i32, _f32, _i32, _vp, _sz, _vp, _vp]),
+    "mpipe_merge_tokens": (_i32, [_vp, _i64, _vp, _i64, _vp, _i32, _i32, _i32, _i32, _vp, _vp]),
+    "mpipe_merge_tokens_bwd": (_i32, [_vp, _i64, _vp, _i64, _vp, _i32, _i32, _i32, _i32, _vp, _vp]),
+    "mpipe_validate_positions": (_i32, [_vp, _i32, _i32]),
+    "mpipe_status_str": (ctypes.c_char_p, [_i32]),
+    "mpipe_version": (_i32, []),
+}
+EXPORTED_SYMBOLS = tuple(_SIGNATURES)
+
+
+def load() -> ctypes.CDLL:
+    """Load the shared library (built in-tree by ``build.py``); raises if it is not there."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2607_03229_b200.build` "
+                "(there is no fallback path)")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+class MpipeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {load().mpipe_status_str(status).decode()} (status {status})")
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise MpipeError(status, where)
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        return t.data_ptr() if t.numel() else None
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data if t.size else None
+    return int(t)
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream or None
+    return getattr(stream, "cuda_stream", stream) or None
+
+
+def fwd_tile_rows() -> int:
+    return load().mpipe_fwd_tile_rows()
+
+
+def bwd_tile_rows() -> int:
+    return load().mpipe_bwd_tile_rows()
+
+
+def version() -> int:
+    return load().mpipe_version()
+
+
+def status_str(status: int) -> str:
+    return load().mpipe_status_str(status).decode()
+
+
+@dataclass
+class SegPlan:
+    """Host result of ``seg_plan`` plus (after ``to_device``) the device copies the kernels read."""
+    mode: int
+    cu_seqlens: np.ndarray          # int32 [n_seg + 1]
+    total_tokens: int
+    max_seqlen: int
+    fwd_items: np.ndarray           # ITEM_DTYPE [n_fwd]
+    bwd_items: np.ndarray           # ITEM_DTYPE [n_bwd]
+    cu_seqlens_dev: Optional[torch.Tensor] = None
+    fwd_items_dev: Optional[torch.Tensor] = None
+    bwd_items_dev: Optional[torch.Tensor] = None
+
+    @property
+    def n_seg(self) -> int:
+        return self.cu_seqlens.size - 1
+
+    def to_device(self, device="cuda") -> "SegPlan":
+        def up(a, cols):
+            t = torch.from_numpy(np.ascontiguousarray(a).view(np.int32).reshape(-1, cols).copy())
+            return t.to(device, non_blocking=False)
+        self.cu_seqlens_dev = up(self.cu_seqlens, 1).reshape(-1)
+        self.fwd_items_dev = up(self.fwd_items, 6)
+        self.bwd_items_dev = up(self.bwd_items, 6)
+        return self
+
+
+def seg_plan(patch_counts, mode: int, fwd_rows: Optional[int] = None, bwd_rows: Optional[int] = None) -> SegPlan:
+    """mpipe_seg_plan with the two-call pattern (count, then fill).  Host only."""
+    lib = load()
+    counts = np.ascontiguousarray(np.asarray(patch_counts, dtype=np.int32).reshape(-1))
+    n_seg = counts.size
+    fwd_rows = fwd_tile_rows() if fwd_rows is None else fwd_rows
+    bwd_rows = bwd_tile_rows() if bwd_rows is None else bwd_rows
+    cu = np.zeros(n_seg + 1, dtype=np.int32)
+    total, mx, nf, nb = (ctypes.c_int32() for _ in range(4))
+    args = (_ptr(counts), n_seg, fwd_rows, bwd_rows, mode, _ptr(cu), ctypes.addressof(total), ctypes.addressof(mx))
+    _check(lib.mpipe_seg_plan(*args, None, ctypes.addressof(nf), None, ctypes.addressof(nb)), "mpipe_seg_plan")
+    fwd = np.zeros(nf.value, dtype=ITEM_DTYPE)
+    bwd = np.zeros(nb.value, dtype=ITEM_DTYPE)
+    _check(lib.mpipe_seg_plan(*args, _ptr(fwd), ctypes.addressof(nf), _ptr(bwd), ctypes.addressof(nb)),
+           "mpipe_seg_plan")
+    return SegPlan(mode, cu, total.value, mx.value, fwd, bwd)
+
+
+def attn_workspace_bytes(total_tokens: int, n_heads: int, head_dim: int, mode: int) -> int:
+    return load().mpipe_attn_workspace_bytes(total_tokens, n_heads, head_dim, mode)
+
+
+def _thd_strides(t: torch.Tensor):
+    assert t.dim() == 3 and t.stride(2) == 1, "expected [tokens, heads, head_dim] with contiguous head_dim"
+    return t.stride(0), t.stride(1)
+
+
+def varlen_attn_fwd(q, k, v, o, lse, plan: SegPlan, softmax_scale: float, status_buf=None, stream=None) -> None:
+    """mpipe_varlen_attn_fwd.  q,k,v,o: bf16 CUDA tensors [T,H,D]; lse: fp32 [H,T] or None (frozen)."""
+    T, H, D = q.shape
+    assert k.shape == q.shape and v.shape == q.shape and o.shape == q.shape
+    assert q.dtype == k.dtype == v.dtype == o.dtype == torch.bfloat16
+    ts, hs = _thd_strides(q)
+    assert _thd_strides(k) == (ts, hs) and _thd_strides(v) == (ts, hs), "q, k, v must share strides"
+    tso, hso = _thd_strides(o)
+    if lse is not None:
+        assert lse.dtype == torch.float32 and lse.is_contiguous() and tuple(lse.shape) == (H, T)
+    st = load().mpipe_varlen_attn_fwd(
+        _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), ts, hs, tso, hso, _ptr(plan.cu_seqlens_dev), plan.n_seg,
+        plan.total_tokens, plan.max_seqlen, _ptr(plan.fwd_items_dev), int(plan.fwd_items.size), H, D,
+        softmax_scale, plan.mode, _ptr(status_buf), _stream(stream))
+    _check(st, "mpipe_varlen_attn_fwd")
+
+
+def varlen_attn_bwd(dout, q, k, v, o, lse, dq, dk, dv, plan: SegPlan, softmax_scale: float, workspace,
+                    status_buf=None, stream=None) -> None:
+    """mpipe_varlen_attn_bwd.  A frozen plan returns at once (nothing is launched)."""
+    T, H, D = q.shape
+    ts, hs = _thd_strides(q)
+    tso, hso = _thd_strides(o)
+    if plan.mode == TRAINED:
+        assert _thd_strides(k) == (ts, hs) and _thd_strides(v) == (ts, hs)
+        assert _thd_strides(dout) == (tso, hso), "dout must share o's strides"
+        tsg, hsg = _thd_strides(dq)
+        assert _thd_strides(dk) == (tsg, hsg) and _thd_strides(dv) == (tsg, hsg)
+    else:
+        tsg, hsg = ts, hs
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    st = load().mpipe_varlen_attn_bwd(
+        _ptr(dout), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(dq), _ptr(dk), _ptr(dv), ts, hs, tso, hso,
+        tsg, hsg, _ptr(plan.cu_seqlens_dev), plan.n_seg, plan.total_tokens, plan.max_seqlen,
+        _ptr(plan.bwd_items_dev), int(plan.bwd_items.size), H, D, softmax_scale, plan.mode, _ptr(workspace),
+        ws_bytes, _ptr(status_buf), _stream(stream))
+    _check(st, "mpipe_varlen_attn_bwd")
+
+
+def merge_tokens(enc_tokens, llm_embeds, positions_dev, mode: int = TRAINED, status_buf=None, stream=None) -> None:
+    """mpipe_merge_tokens: llm_embeds[positions[i], :] = enc_tokens[i, :], in place."""
+    n_enc = int(positions_dev.numel())
+    n_llm, hidden = llm_embeds.shape
+    assert enc_tokens.dtype == llm_embeds.dtype == torch.bfloat16 and positions_dev.dtype == torch.int32
+    assert enc_tokens.shape[0] == n_enc and (n_enc == 0 or enc_tokens.shape[1] == hidden)
+    assert llm_embeds.stride(1) == 1 and (n_enc == 0 or enc_tokens.stride(1) == 1)
+    st = load().mpipe_merge_tokens(_ptr(enc_tokens), enc_tokens.stride(0) if n_enc else hidden, _ptr(llm_embeds),
+                                   llm_embeds.stride(0), _ptr(positions_dev), n_enc, n_llm, hidden, mode,
+                                   _ptr(status_buf), _stream(stream))
+    _check(st, "mpipe_merge_tokens")
+
+
+def merge_tokens_bwd(d_llm_embeds, d_enc, positions_dev, mode: int, status_buf=None, stream=None) -> None:
+    """mpipe_merge_tokens_bwd: d_enc[i, :] = d_llm_embeds[positions[i], :]; no-op when frozen."""
+    n_enc = int(positions_dev.numel())
+    n_llm, hidden = d_llm_embeds.shape
+    assert d_llm_embeds.dtype == torch.bfloat16 and positions_dev.dtype == torch.int32
+    st = load().mpipe_merge_tokens_bwd(_ptr(d_llm_embeds), d_llm_embeds.stride(0), _ptr(d_enc),
+                                       d_enc.stride(0) if n_enc else hidden, _ptr(positions_dev), n_enc, n_llm,
+                                       hidden, mode, _ptr(status_buf), _stream(stream))
+    _check(st, "mpipe_merge_tokens_bwd")
+
+
+def validate_positions(positions, n_llm_tokens: int) -> int:
+    pos = np.ascontiguousarray(np.asarray(positions, dtype=np.int32))
+    return load().mpipe_validate_positions(_ptr(pos), pos.size, n_llm_tokens)
