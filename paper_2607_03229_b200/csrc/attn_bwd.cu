@@ -1,23 +1,628 @@
-// mpipe_varlen_attn_bwd (placeholder until the tcgen05 backward lands).
+// mpipe_varlen_attn_bwd: gradient of the per-image softmax attention, the attention part of the
+// optional Bwd(enc, r, m) event (it exists only when trainable(enc), Lemma 1).
+//
+// Three launches on the caller's stream:
+//   1. prepass   Delta[h,t] = sum_d dO[t,h,d] O[t,h,d]  and the fp32 dQ accumulator is cleared
+//   2. main      one persistent CTA per SM walks (key tile x head) units; a unit keeps one 128-key
+//                K/V tile resident and loops over the 128-row query tiles of the same segment
+//   3. convert   dQ = softmax_scale * accumulator -> bf16
+//
+// Main kernel, per query tile i (everything transposed so that the key index is the TMEM lane):
+//   S^T  = K Q^T            tcgen05, operands in shared memory               -> TMEM
+//   dP^T = V dO^T           tcgen05                                           -> TMEM
+//   P^T  = exp2(S^T * scale*log2e - LSE*log2e)       softmax warps, written over S^T as bf16
+//   dS^T = P^T o (dP^T - Delta)                      softmax warps, over dP^T as bf16 + to shared memory
+//   dV  += P^T dO           tcgen05, A operand read from TMEM, dO as MN-major B
+//   dK  += dS^T Q           tcgen05, A operand read from TMEM, Q as MN-major B
+//   dQ_i = dS K             tcgen05, dS^T in shared memory read as an MN-major A, K as MN-major B
+// dQ_i is read back from TMEM by a reducer warpgroup and added to the global fp32 accumulator with
+// vector atomics; dK (x softmax_scale) and dV leave TMEM once per unit.
+//
+// Warp roles (512 threads): 0 TMA producer, 1 tcgen05 issuer, 2 TMEM allocation + LSE staging,
+// 3 Delta staging, 4-7 / 8-11 softmax on query columns 0-63 / 64-127, 12-15 dQ reducer and epilogue.
+// Every wait is bounded (see sm100_ptx.cuh); expiry sets status_buf and drains the CTA.
+#include <cuda.h>
+#include <math_constants.h>
 #include "common.h"
+#include "sm100_ptx.cuh"
+#include "tensormap.h"
+
+namespace mpipe {
+
+constexpr int kBwdThreads = 512;
+constexpr int kBT = 128;  // keys per unit = query rows per iteration = TMEM lanes
+
+template <int D>
+struct BwdCfg {
+    static constexpr int kTail = D - 64;
+    static constexpr int kTileMain = kBT * 128;                 // [128 rows][64 bf16], 128-byte swizzle
+    static constexpr int kTileTail = kTail ? kBT * 32 : 0;      // [128 rows][16 bf16], 32-byte swizzle
+    static constexpr int kTile = kTileMain + kTileTail;
+    static constexpr int kStages = 2;
+    static constexpr int kSmemK = 0;
+    static constexpr int kSmemV = kTile;
+    static constexpr int kSmemQ = 2 * kTile;                    // kStages tiles
+    static constexpr int kSmemDO = kSmemQ + kStages * kTile;    // kStages tiles
+    static constexpr int kSmemDS = kSmemDO + kStages * kTile;   // [key][q] as two 64-wide atoms: 32 KB
+    static constexpr int kSmemStat = kSmemDS + 2 * kBT * 128;   // kStages x (LSE[128], Delta[128]) fp32
+    static constexpr int kSmemTotal = kSmemStat + kStages * 2 * kBT * 4;
+    static constexpr int kSmemAlloc = kSmemTotal + 1024;
+    // TMEM columns
+    static constexpr int kColS = 0, kColDP = 128, kColDV = 256, kColDK = 256 + D, kColDQ = 256 + 2 * D;
+};
+
+struct BwdParams {
+    const mpipe_work_item_t* items;
+    int32_t n_items, n_heads, total_tokens;
+    const float* lse;    // [H, T]
+    const float* delta;  // [H, T]
+    float* dq_acc;       // [T, H, D] fp32
+    __nv_bfloat16 *dk, *dv;
+    int64_t tok_stride_g, head_stride_g;
+    float scale, scale_log2;
+    int32_t* status_buf;
+};
+
+struct BwdBarriers {
+    uint64_t kv_full, kv_empty, dkv_full, dkv_empty;
+    uint64_t qdo_full[2], qdo_empty[2], stat_full[2], stat_empty[2];
+    uint64_t s_full, p_full, dp_full, ds_full, dq_full, dq_empty;
+};
+
+__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+template <int D>
+__global__ void __launch_bounds__(kBwdThreads, 1)
+attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
+                const __grid_constant__ CUtensorMap map_q_tail, const __grid_constant__ CUtensorMap map_k_tail,
+                const __grid_constant__ CUtensorMap map_v_tail, const __grid_constant__ CUtensorMap map_do_tail,
+                const BwdParams p) {
+    using Cfg = BwdCfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ BwdBarriers bars;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(&bars.kv_full, 1);
+        mbar_init(&bars.kv_empty, 1);
+        mbar_init(&bars.dkv_full, 1);
+        mbar_init(&bars.dkv_empty, 4);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&bars.qdo_full[s], 1);
+            mbar_init(&bars.qdo_empty[s], 1);
+            mbar_init(&bars.stat_full[s], 2);
+            mbar_init(&bars.stat_empty[s], 8);
+        }
+        mbar_init(&bars.s_full, 1);
+        mbar_init(&bars.p_full, 8);
+        mbar_init(&bars.dp_full, 1);
+        mbar_init(&bars.ds_full, 8);
+        mbar_init(&bars.dq_full, 1);
+        mbar_init(&bars.dq_empty, 4);
+        fence_mbar_init();
+    }
+    if (warp == 2) {
+        tmem_alloc(&tmem_base_slot, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_slot;
+    const int n_units = p.n_items * p.n_heads;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        setmaxnreg_dec<72>();
+        if (lane == 0) {
+            uint32_t unit_it = 0, it_cnt = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
+                const mpipe_work_item_t it = p.items[u / p.n_heads];
+                const int head = u % p.n_heads;
+                const int nq = (it.kv_len + kBT - 1) / kBT;
+                ok = mbar_wait(&bars.kv_empty, (unit_it & 1) ^ 1, &abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(&bars.kv_full, 2 * Cfg::kTile);
+                tma_load_3d(smem + Cfg::kSmemK, &map_k, &bars.kv_full, 0, head, it.row_start);
+                tma_load_3d(smem + Cfg::kSmemV, &map_v, &bars.kv_full, 0, head, it.row_start);
+                if (Cfg::kTail) {
+                    tma_load_3d(smem + Cfg::kSmemK + Cfg::kTileMain, &map_k_tail, &bars.kv_full, 64, head, it.row_start);
+                    tma_load_3d(smem + Cfg::kSmemV + Cfg::kTileMain, &map_v_tail, &bars.kv_full, 64, head, it.row_start);
+                }
+                for (int i = 0; i < nq; ++i, ++it_cnt) {
+                    const int st = it_cnt & 1;
+                    const int row = it.kv_start + i * kBT;
+                    ok = mbar_wait(&bars.qdo_empty[st], ((it_cnt >> 1) & 1) ^ 1, &abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(&bars.qdo_full[st], 2 * Cfg::kTile);
+                    uint8_t* qd = smem + Cfg::kSmemQ + st * Cfg::kTile;
+                    uint8_t* dd = smem + Cfg::kSmemDO + st * Cfg::kTile;
+                    tma_load_3d(qd, &map_q, &bars.qdo_full[st], 0, head, row);
+                    tma_load_3d(dd, &map_do, &bars.qdo_full[st], 0, head, row);
+                    if (Cfg::kTail) {
+                        tma_load_3d(qd + Cfg::kTileMain, &map_q_tail, &bars.qdo_full[st], 64, head, row);
+                        tma_load_3d(dd + Cfg::kTileMain, &map_do_tail, &bars.qdo_full[st], 64, head, row);
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ tcgen05 issuer
+        setmaxnreg_dec<72>();
+        if (lane == 0) {
+            const uint32_t sbase = smem_u32(smem);
+            const uint32_t ka = sbase + Cfg::kSmemK, va = sbase + Cfg::kSmemV, dsa = sbase + Cfg::kSmemDS;
+            constexpr uint32_t idesc_s = umma_idesc_bf16(kBT, kBT, 0, 0);      // K-major x K-major, N = 128 queries
+            constexpr uint32_t idesc_ts = umma_idesc_bf16(kBT, 64, 0, 1);      // A in TMEM, MN-major B, N = 64
+            constexpr uint32_t idesc_ts_t = umma_idesc_bf16(kBT, 16, 0, 1);    // same, 16-wide head-dim tail
+            constexpr uint32_t idesc_dq = umma_idesc_bf16(kBT, 64, 1, 1);      // MN-major A and B
+            constexpr uint32_t idesc_dq_t = umma_idesc_bf16(kBT, 16, 1, 1);
+            // dst[128 x 128] = A[128 x D] * B[128 x D]^T, both K-major tiles (main 64 + optional 16 tail)
+            auto issue_kk = [&](uint32_t dcol, uint32_t a, uint32_t b) {
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_ss(tmem + dcol, umma_smem_desc(a + ks * 32, 0, 1024, kSwizzle128),
+                            umma_smem_desc(b + ks * 32, 0, 1024, kSwizzle128), idesc_s, ks > 0);
+                if (Cfg::kTail)
+                    umma_ss(tmem + dcol, umma_smem_desc(a + Cfg::kTileMain, 0, 256, kSwizzle32),
+                            umma_smem_desc(b + Cfg::kTileMain, 0, 256, kSwizzle32), idesc_s, 1);
+            };
+            // dst[128 keys x D] (+)= A^T-in-TMEM[128 keys x 128 q] * B[128 q x D] (B tile rows = q, MN-major)
+            auto issue_ts = [&](uint32_t dcol, uint32_t acol, uint32_t b, bool acc) {
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t a_t = tmem + acol + (ks < 4 ? ks * 8 : 64 + (ks - 4) * 8);
+                    umma_ts(tmem + dcol, a_t, umma_smem_desc(b + ks * 2048, 0, 1024, kSwizzle128), idesc_ts,
+                            (acc || ks > 0) ? 1u : 0u);
+                    if (Cfg::kTail)
+                        umma_ts(tmem + dcol + 64, a_t, umma_smem_desc(b + Cfg::kTileMain + ks * 512, 0, 256, kSwizzle32),
+                                idesc_ts_t, (acc || ks > 0) ? 1u : 0u);
+                }
+            };
+            uint32_t unit_it = 0, it_cnt = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
+                const mpipe_work_item_t it = p.items[u / p.n_heads];
+                const int nq = (it.kv_len + kBT - 1) / kBT;
+                ok = mbar_wait(&bars.kv_full, unit_it & 1, &abort_flag);
+                if (!ok) break;
+                ok = mbar_wait(&bars.qdo_full[it_cnt & 1], (it_cnt >> 1) & 1, &abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                {
+                    const uint32_t qa = sbase + Cfg::kSmemQ + (it_cnt & 1) * Cfg::kTile;
+                    const uint32_t da = sbase + Cfg::kSmemDO + (it_cnt & 1) * Cfg::kTile;
+                    issue_kk(Cfg::kColS, ka, qa);
+                    umma_commit(&bars.s_full);
+                    issue_kk(Cfg::kColDP, va, da);
+                    umma_commit(&bars.dp_full);
+                }
+                for (int i = 0; i < nq; ++i, ++it_cnt) {
+                    const int st = it_cnt & 1;
+                    const uint32_t qa = sbase + Cfg::kSmemQ + st * Cfg::kTile;
+                    const uint32_t da = sbase + Cfg::kSmemDO + st * Cfg::kTile;
+                    const uint32_t qa_n = sbase + Cfg::kSmemQ + (st ^ 1) * Cfg::kTile;
+                    const uint32_t da_n = sbase + Cfg::kSmemDO + (st ^ 1) * Cfg::kTile;
+                    const bool more = (i + 1 < nq);
+                    if (i == 0) {
+                        ok = mbar_wait(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag);
+                        if (!ok) break;
+                    }
+                    ok = mbar_wait(&bars.p_full, it_cnt & 1, &abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_ts(Cfg::kColDV, Cfg::kColS, da, i > 0);                 // dV += P^T dO
+                    if (more) {
+                        ok = mbar_wait(&bars.qdo_full[st ^ 1], ((it_cnt + 1) >> 1) & 1, &abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_kk(Cfg::kColS, ka, qa_n);                           // S^T(i+1)
+                        umma_commit(&bars.s_full);
+                    }
+                    ok = mbar_wait(&bars.ds_full, it_cnt & 1, &abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_ts(Cfg::kColDK, Cfg::kColDP, qa, i > 0);                // dK += dS^T Q
+                    ok = mbar_wait(&bars.dq_empty, (it_cnt & 1) ^ 1, &abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {                              // dQ_i = dS K
+                        const uint64_t adesc = umma_smem_desc(dsa + ks * 2048, kBT * 128, 1024, kSwizzle128);
+                        umma_ss(tmem + Cfg::kColDQ, adesc, umma_smem_desc(ka + ks * 2048, 0, 1024, kSwizzle128), idesc_dq,
+                                ks > 0);
+                        if (Cfg::kTail)
+                            umma_ss(tmem + Cfg::kColDQ + 64, adesc,
+                                    umma_smem_desc(ka + Cfg::kTileMain + ks * 512, 0, 256, kSwizzle32), idesc_dq_t, ks > 0);
+                    }
+                    umma_commit(&bars.dq_full);
+                    umma_commit(&bars.qdo_empty[st]);
+                    if (more) {
+                        issue_kk(Cfg::kColDP, va, da_n);                          // dP^T(i+1)
+                        umma_commit(&bars.dp_full);
+                    }
+                }
+                if (!ok) break;
+                umma_commit(&bars.dkv_full);
+                umma_commit(&bars.kv_empty);
+            }
+        }
+        __syncwarp();
+    } else if (warp < 4) {
+        // ------------------------------------------------------------------ LSE (warp 2) / Delta (warp 3) staging
+        setmaxnreg_dec<72>();
+        const bool is_lse = (warp == 2);
+        const float* src = is_lse ? p.lse : p.delta;
+        uint32_t it_cnt = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+            const mpipe_work_item_t it = p.items[u / p.n_heads];
+            const int head = u % p.n_heads;
+            const int nq = (it.kv_len + kBT - 1) / kBT;
+            const int q_end = it.kv_start + it.kv_len;
+            for (int i = 0; i < nq; ++i, ++it_cnt) {
+                const int st = it_cnt & 1;
+                ok = mbar_wait(&bars.stat_empty[st], ((it_cnt >> 1) & 1) ^ 1, &abort_flag);
+                if (!ok) break;
+                float* dst = reinterpret_cast<float*>(smem + Cfg::kSmemStat + st * (2 * kBT * 4)) + (is_lse ? 0 : kBT);
+                const int q0 = it.kv_start + i * kBT;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int c = lane + 32 * e;
+                    const int q = q0 + c;
+                    float val;
+                    if (q < q_end) {
+                        val = __ldg(src + int64_t(head) * p.total_tokens + q);
+                        if (is_lse) val *= 1.4426950408889634f;
+                    } else {
+                        val = is_lse ? CUDART_INF_F : 0.f;  // P = exp2(-inf) = 0 for query columns past the segment
+                    }
+                    dst[c] = val;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars.stat_full[st]);
+            }
+        }
+    } else if (warp < 12) {
+        // ------------------------------------------------------------------ softmax / dS warps
+        setmaxnreg_inc<168>();
+        const int g = (warp - 4) >> 2;                // query-column half handled by this warpgroup
+        const int r = ((warp & 3) << 5) | lane;       // key row inside the tile = TMEM lane
+        const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
+        const uint32_t t_s = tmem + lane_base + Cfg::kColS + g * 64;    // S^T columns of this half; P^T goes to the first 32 of them
+        const uint32_t t_dp = tmem + lane_base + Cfg::kColDP + g * 64;
+        uint8_t* ds_row = smem + Cfg::kSmemDS + g * (kBT * 128) + r * 128;
+        uint32_t it_cnt = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+            const mpipe_work_item_t it = p.items[u / p.n_heads];
+            const int nq = (it.kv_len + kBT - 1) / kBT;
+            const bool key_valid = r < it.row_len;
+            for (int i = 0; i < nq; ++i, ++it_cnt) {
+                const int st = it_cnt & 1;
+                const float* stat = reinterpret_cast<const float*>(smem + Cfg::kSmemStat + st * (2 * kBT * 4));
+                const float4* lse4 = reinterpret_cast<const float4*>(stat + g * 64);
+                const float4* dl4 = reinterpret_cast<const float4*>(stat + kBT + g * 64);
+                ok = mbar_wait(&bars.stat_full[st], (it_cnt >> 1) & 1, &abort_flag);
+                if (!ok) break;
+                ok = mbar_wait(&bars.s_full, it_cnt & 1, &abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                float pr[64];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t sr[32];
+                    tmem_ld32(t_s + h * 32, sr);
+                    tmem_wait_ld();
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int c4 = 0; c4 < 8; ++c4) {
+                        const float4 l4 = lse4[h * 8 + c4];
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(sr[4 * c4 + 0]), p.scale_log2, -l4.x));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(sr[4 * c4 + 1]), p.scale_log2, -l4.y));
+                        const float p2 = ex2_approx(fmaf(__uint_as_float(sr[4 * c4 + 2]), p.scale_log2, -l4.z));
+                        const float p3 = ex2_approx(fmaf(__uint_as_float(sr[4 * c4 + 3]), p.scale_log2, -l4.w));
+                        pr[h * 32 + 4 * c4 + 0] = p0;
+                        pr[h * 32 + 4 * c4 + 1] = p1;
+                        pr[h * 32 + 4 * c4 + 2] = p2;
+                        pr[h * 32 + 4 * c4 + 3] = p3;
+                        pk[2 * c4] = pack_bf16(p0, p1);
+                        pk[2 * c4 + 1] = pack_bf16(p2, p3);
+                    }
+                    tmem_st16(t_s + h * 16, pk);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars.p_full);
+
+                ok = mbar_wait(&bars.dp_full, it_cnt & 1, &abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t dr[32];
+                    tmem_ld32(t_dp + h * 32, dr);
+                    tmem_wait_ld();
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int c4 = 0; c4 < 8; ++c4) {
+                        const float4 d4 = dl4[h * 8 + c4];
+                        float s0 = pr[h * 32 + 4 * c4 + 0] * (__uint_as_float(dr[4 * c4 + 0]) - d4.x);
+                        float s1 = pr[h * 32 + 4 * c4 + 1] * (__uint_as_float(dr[4 * c4 + 1]) - d4.y);
+                        float s2 = pr[h * 32 + 4 * c4 + 2] * (__uint_as_float(dr[4 * c4 + 2]) - d4.z);
+                        float s3 = pr[h * 32 + 4 * c4 + 3] * (__uint_as_float(dr[4 * c4 + 3]) - d4.w);
+                        if (!key_valid) s0 = s1 = s2 = s3 = 0.f;  // rows past the segment must not reach dQ
+                        pk[2 * c4] = pack_bf16(s0, s1);
+                        pk[2 * c4 + 1] = pack_bf16(s2, s3);
+                    }
+                    tmem_st16(t_dp + h * 16, pk);
+                    // the same 32 values as 4 x 16 bytes of row r of the [key][q] tile (128-byte swizzle)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int chunk = h * 4 + c;
+                        *reinterpret_cast<uint4*>(ds_row + ((chunk ^ (r & 7)) << 4)) =
+                            make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                    }
+                }
+                tmem_wait_st();
+                fence_async_smem();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(&bars.ds_full);
+                    mbar_arrive(&bars.stat_empty[st]);
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ dQ reducer + dK/dV epilogue
+        setmaxnreg_dec<96>();
+        const int r = ((warp & 3) << 5) | lane;
+        const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
+        uint32_t it_cnt = 0, unit_it = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
+            const mpipe_work_item_t it = p.items[u / p.n_heads];
+            const int head = u % p.n_heads;
+            const int nq = (it.kv_len + kBT - 1) / kBT;
+            const int q_end = it.kv_start + it.kv_len;
+            for (int i = 0; i < nq; ++i, ++it_cnt) {
+                ok = mbar_wait(&bars.dq_full, it_cnt & 1, &abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const int q = it.kv_start + i * kBT + r;
+                float* dst = p.dq_acc + (int64_t(q) * p.n_heads + head) * D;
+#pragma unroll
+                for (int c0 = 0; c0 < D; c0 += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(tmem + lane_base + Cfg::kColDQ + c0, v);
+                    tmem_wait_ld();
+                    if (c0 + 16 >= D) {  // all reads of this row issued and complete: release dQ in TMEM
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars.dq_empty);
+                    }
+                    if (q < q_end) {
+#pragma unroll
+                        for (int c = 0; c < 16; c += 4)
+                            red_add_v4(dst + c0 + c, __uint_as_float(v[c]), __uint_as_float(v[c + 1]),
+                                       __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
+                    }
+                }
+            }
+            if (!ok) break;
+            ok = mbar_wait(&bars.dkv_full, unit_it & 1, &abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const bool store = r < it.row_len;
+            const int64_t tok = int64_t(it.row_start) + r;
+            __nv_bfloat16* dv_row = p.dv + tok * p.tok_stride_g + int64_t(head) * p.head_stride_g;
+            __nv_bfloat16* dk_row = p.dk + tok * p.tok_stride_g + int64_t(head) * p.head_stride_g;
+#pragma unroll
+            for (int which = 0; which < 2; ++which) {
+                const uint32_t col = which == 0 ? Cfg::kColDV : Cfg::kColDK;
+                const float mul = which == 0 ? 1.0f : p.scale;
+                __nv_bfloat16* row = which == 0 ? dv_row : dk_row;
+#pragma unroll
+                for (int c0 = 0; c0 < D; c0 += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(tmem + lane_base + col + c0, v);
+                    tmem_wait_ld();
+                    uint4 a, b;
+                    a.x = pack_bf16(__uint_as_float(v[0]) * mul, __uint_as_float(v[1]) * mul);
+                    a.y = pack_bf16(__uint_as_float(v[2]) * mul, __uint_as_float(v[3]) * mul);
+                    a.z = pack_bf16(__uint_as_float(v[4]) * mul, __uint_as_float(v[5]) * mul);
+                    a.w = pack_bf16(__uint_as_float(v[6]) * mul, __uint_as_float(v[7]) * mul);
+                    b.x = pack_bf16(__uint_as_float(v[8]) * mul, __uint_as_float(v[9]) * mul);
+                    b.y = pack_bf16(__uint_as_float(v[10]) * mul, __uint_as_float(v[11]) * mul);
+                    b.z = pack_bf16(__uint_as_float(v[12]) * mul, __uint_as_float(v[13]) * mul);
+                    b.w = pack_bf16(__uint_as_float(v[14]) * mul, __uint_as_float(v[15]) * mul);
+                    if (store) {
+                        *reinterpret_cast<uint4*>(row + c0) = a;
+                        *reinterpret_cast<uint4*>(row + c0 + 8) = b;
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars.dkv_empty);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) tmem_dealloc(tmem, 512);
+    if (tid == 0 && abort_flag) report_status(p.status_buf, MPIPE_ERR_TIMEOUT, int32_t(blockIdx.x));
+}
+
+// Delta[h,t] = sum_d dO[t,h,d] * O[t,h,d]; clears the fp32 dQ accumulator row of (t,h).  One thread per (t,h).
+template <int D>
+__global__ void __launch_bounds__(256)
+bwd_prepass_kernel(const __nv_bfloat16* __restrict__ dout, const __nv_bfloat16* __restrict__ o, int64_t tok_stride_o,
+                   int64_t head_stride_o, int32_t total_tokens, int32_t n_heads, float* __restrict__ delta,
+                   float* __restrict__ dq_acc) {
+    const int64_t idx = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= int64_t(total_tokens) * n_heads) return;
+    const int t = int(idx / n_heads), h = int(idx % n_heads);
+    const uint4* a = reinterpret_cast<const uint4*>(dout + t * tok_stride_o + h * head_stride_o);
+    const uint4* b = reinterpret_cast<const uint4*>(o + t * tok_stride_o + h * head_stride_o);
+    float acc = 0.f;
+#pragma unroll
+    for (int c = 0; c < D / 8; ++c) {
+        const uint4 x = __ldg(a + c), y = __ldg(b + c);
+        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            acc = fmaf(__uint_as_float(xs[e] << 16), __uint_as_float(ys[e] << 16), acc);
+            acc = fmaf(__uint_as_float(xs[e] & 0xFFFF0000u), __uint_as_float(ys[e] & 0xFFFF0000u), acc);
+        }
+    }
+    delta[int64_t(h) * total_tokens + t] = acc;
+    float4* z = reinterpret_cast<float4*>(dq_acc + idx * D);
+#pragma unroll
+    for (int c = 0; c < D / 4; ++c) z[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+// dQ[t,h,:] = scale * acc[t,h,:] as bf16.  One thread per 8 elements.
+__global__ void __launch_bounds__(256)
+bwd_dq_convert_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, int64_t tok_stride_g,
+                      int64_t head_stride_g, int32_t total_tokens, int32_t n_heads, int32_t head_dim, float scale) {
+    const int chunks = head_dim / 8;
+    const int64_t idx = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= int64_t(total_tokens) * n_heads * chunks) return;
+    const int c = int(idx % chunks);
+    const int64_t th = idx / chunks;
+    const int h = int(th % n_heads);
+    const int64_t t = th / n_heads;
+    const float4* src = reinterpret_cast<const float4*>(acc + th * head_dim + c * 8);
+    const float4 x = __ldg(src), y = __ldg(src + 1);
+    uint4 out;
+    out.x = pack_bf16(x.x * scale, x.y * scale);
+    out.y = pack_bf16(x.z * scale, x.w * scale);
+    out.z = pack_bf16(y.x * scale, y.y * scale);
+    out.w = pack_bf16(y.z * scale, y.w * scale);
+    *reinterpret_cast<uint4*>(dq + t * tok_stride_g + h * head_stride_g + c * 8) = out;
+}
+
+template <int D>
+static int32_t launch_bwd(const void* dout, const void* q, const void* k, const void* v, const void* o, void* dq,
+                          int64_t ts_qkv, int64_t hs_qkv, int64_t ts_o, int64_t hs_o, int32_t total_tokens,
+                          int32_t n_heads, BwdParams prm, float* delta, cudaStream_t stream) {
+    using Cfg = BwdCfg<D>;
+    CUtensorMap mq, mk, mv, mdo, mqt, mkt, mvt, mdot;
+    if (!make_tensor_map_thd(&mq, q, total_tokens, n_heads, D, ts_qkv, hs_qkv, 64, kBT, 128) ||
+        !make_tensor_map_thd(&mk, k, total_tokens, n_heads, D, ts_qkv, hs_qkv, 64, kBT, 128) ||
+        !make_tensor_map_thd(&mv, v, total_tokens, n_heads, D, ts_qkv, hs_qkv, 64, kBT, 128) ||
+        !make_tensor_map_thd(&mdo, dout, total_tokens, n_heads, D, ts_o, hs_o, 64, kBT, 128))
+        return MPIPE_ERR_CUDA;
+    mqt = mq, mkt = mk, mvt = mv, mdot = mdo;
+    if (Cfg::kTail) {
+        if (!make_tensor_map_thd(&mqt, q, total_tokens, n_heads, D, ts_qkv, hs_qkv, 16, kBT, 32) ||
+            !make_tensor_map_thd(&mkt, k, total_tokens, n_heads, D, ts_qkv, hs_qkv, 16, kBT, 32) ||
+            !make_tensor_map_thd(&mvt, v, total_tokens, n_heads, D, ts_qkv, hs_qkv, 16, kBT, 32) ||
+            !make_tensor_map_thd(&mdot, dout, total_tokens, n_heads, D, ts_o, hs_o, 16, kBT, 32))
+            return MPIPE_ERR_CUDA;
+    }
+    if (cudaFuncSetAttribute(attn_bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemAlloc) !=
+        cudaSuccess)
+        return MPIPE_ERR_CUDA;
+    const int64_t rows = int64_t(total_tokens) * n_heads;
+    bwd_prepass_kernel<D><<<unsigned((rows + 255) / 256), 256, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(dout), static_cast<const __nv_bfloat16*>(o), ts_o, hs_o, total_tokens, n_heads,
+        delta, prm.dq_acc);
+    const int n_units = prm.n_items * prm.n_heads;
+    const int grid = n_units < sm_count() ? n_units : sm_count();
+    attn_bwd_kernel<D><<<grid, kBwdThreads, Cfg::kSmemAlloc, stream>>>(mq, mk, mv, mdo, mqt, mkt, mvt, mdot, prm);
+    const int64_t chunks = rows * (D / 8);
+    bwd_dq_convert_kernel<<<unsigned((chunks + 255) / 256), 256, 0, stream>>>(
+        prm.dq_acc, static_cast<__nv_bfloat16*>(dq), prm.tok_stride_g, prm.head_stride_g, total_tokens, n_heads, D,
+        prm.scale);
+    return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
+}
+
+static size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
+
+}  // namespace mpipe
 
 extern "C" {
 
-int32_t mpipe_bwd_tile_rows(void) { return 128; }
+int32_t mpipe_bwd_tile_rows(void) { return mpipe::kBT; }
 
 size_t mpipe_attn_workspace_bytes(int32_t total_tokens, int32_t n_heads, int32_t head_dim, int32_t mode) {
     if (mode != MPIPE_ENC_TRAINED || total_tokens <= 0 || n_heads <= 0 || head_dim <= 0) return 0;
-    const size_t dq = (size_t(total_tokens) * n_heads * head_dim * 4 + 255) & ~size_t(255);
-    const size_t delta = (size_t(total_tokens) * n_heads * 4 + 255) & ~size_t(255);
-    return dq + delta;
+    return mpipe::round256(size_t(total_tokens) * n_heads * head_dim * 4) +
+           mpipe::round256(size_t(total_tokens) * n_heads * 4);
 }
 
-int32_t mpipe_varlen_attn_bwd(const void*, const void*, const void*, const void*, const void*, const float*, void*,
-                              void*, void*, int64_t, int64_t, int64_t, int64_t, int64_t, int64_t, const int32_t*,
-                              int32_t, int32_t, int32_t, const mpipe_work_item_t*, int32_t, int32_t, int32_t, float,
-                              int32_t mode, void*, size_t, int32_t*, void*) {
-    if (mode == MPIPE_ENC_FROZEN) return MPIPE_OK;
-    return MPIPE_ERR_UNSUPPORTED;
+int32_t mpipe_varlen_attn_bwd(const void* dout, const void* q, const void* k, const void* v, const void* o,
+                              const float* lse, void* dq, void* dk, void* dv, int64_t tok_stride_qkv,
+                              int64_t head_stride_qkv, int64_t tok_stride_o, int64_t head_stride_o,
+                              int64_t tok_stride_grad, int64_t head_stride_grad, const int32_t* cu_seqlens_dev,
+                              int32_t n_seg, int32_t total_tokens, int32_t max_seqlen,
+                              const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items, int32_t n_heads,
+                              int32_t head_dim, float softmax_scale, int32_t mode, void* workspace,
+                              size_t workspace_bytes, int32_t* status_buf, void* stream) {
+    using namespace mpipe;
+    if (mode != MPIPE_ENC_FROZEN && mode != MPIPE_ENC_TRAINED) return MPIPE_ERR_INVALID_ARG;
+    if (mode == MPIPE_ENC_FROZEN) return MPIPE_OK;  // Lemma 1: a frozen encoder has no backward event
+    if (n_seg < 0 || total_tokens < 0 || max_seqlen < 0 || n_bwd_items < 0 || n_heads <= 0) return MPIPE_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 80) return MPIPE_ERR_UNSUPPORTED;
+    if (total_tokens == 0 || n_bwd_items == 0) return MPIPE_OK;
+    if (dout == nullptr || q == nullptr || k == nullptr || v == nullptr || o == nullptr || lse == nullptr ||
+        dq == nullptr || dk == nullptr || dv == nullptr || bwd_items_dev == nullptr || cu_seqlens_dev == nullptr)
+        return MPIPE_ERR_INVALID_ARG;
+    if (!aligned16(dout) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv))
+        return MPIPE_ERR_INVALID_ARG;
+    if ((tok_stride_qkv & 7) || (head_stride_qkv & 7) || (tok_stride_o & 7) || (head_stride_o & 7) ||
+        (tok_stride_grad & 7) || (head_stride_grad & 7))
+        return MPIPE_ERR_INVALID_ARG;
+    if (head_stride_qkv < head_dim || head_stride_o < head_dim || head_stride_grad < head_dim ||
+        tok_stride_qkv < head_dim || tok_stride_o < head_dim || tok_stride_grad < head_dim)
+        return MPIPE_ERR_INVALID_ARG;
+    if (!(softmax_scale > 0.f) || !(softmax_scale < 1e30f)) return MPIPE_ERR_INVALID_ARG;
+    if (int64_t(n_bwd_items) * n_heads >= (int64_t(1) << 31)) return MPIPE_ERR_INVALID_ARG;
+    const size_t need = mpipe_attn_workspace_bytes(total_tokens, n_heads, head_dim, mode);
+    if (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+        return MPIPE_ERR_WORKSPACE;
+
+    float* dq_acc = static_cast<float*>(workspace);
+    float* delta = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) +
+                                            round256(size_t(total_tokens) * n_heads * head_dim * 4));
+    BwdParams prm;
+    prm.items = bwd_items_dev;
+    prm.n_items = n_bwd_items;
+    prm.n_heads = n_heads;
+    prm.total_tokens = total_tokens;
+    prm.lse = lse;
+    prm.delta = delta;
+    prm.dq_acc = dq_acc;
+    prm.dk = static_cast<__nv_bfloat16*>(dk);
+    prm.dv = static_cast<__nv_bfloat16*>(dv);
+    prm.tok_stride_g = tok_stride_grad;
+    prm.head_stride_g = head_stride_grad;
+    prm.scale = softmax_scale;
+    prm.scale_log2 = softmax_scale * 1.4426950408889634f;
+    prm.status_buf = status_buf;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (head_dim == 64)
+        return launch_bwd<64>(dout, q, k, v, o, dq, tok_stride_qkv, head_stride_qkv, tok_stride_o, head_stride_o,
+                              total_tokens, n_heads, prm, delta, st);
+    return launch_bwd<80>(dout, q, k, v, o, dq, tok_stride_qkv, head_stride_qkv, tok_stride_o, head_stride_o,
+                          total_tokens, n_heads, prm, delta, st);
 }
 
 }  // extern "C"

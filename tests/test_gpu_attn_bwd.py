@@ -1,0 +1,152 @@
+"""GPU parity of mpipe_varlen_attn_bwd against the fp64 oracle, and the trainability gate of
+Lemma 1: a frozen encoder launches no backward and touches no gradient buffer."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_03229_b200 import binding as B
+from paper_2607_03229_b200 import workloads as W
+from _util import GRAD_REL_L2, max_abs, rel_l2, status_buf, to_dev, to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+def gpu_fwd_bwd(q, k, v, do, counts, scale, mode=B.TRAINED):
+    """Forward then backward through the C ABI.  Returns (o, lse, dq, dk, dv) device tensors."""
+    T, H, D = q.shape
+    plan = B.seg_plan(counts, mode).to_device()
+    qd, kd, vd, dod = to_dev(q), to_dev(k), to_dev(v), to_dev(do)
+    o = torch.empty_like(qd)
+    lse = torch.empty((H, T), dtype=torch.float32, device="cuda") if mode == B.TRAINED else None
+    st = status_buf()
+    B.varlen_attn_fwd(qd, kd, vd, o, lse, plan, scale, st)
+    pad = 2
+    grads = [torch.full((T + 2 * pad, H, D), 333.0, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+    dq, dk, dv = (g[pad:pad + T] for g in grads)
+    ws_bytes = B.attn_workspace_bytes(T, H, D, mode)
+    ws = torch.empty(max(ws_bytes, 1), dtype=torch.uint8, device="cuda")
+    B.varlen_attn_bwd(dod, qd, kd, vd, o, lse, dq, dk, dv, plan, scale, ws, st)
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[0] == 0, f"device status {st.cpu().tolist()}"
+    for g in grads:
+        assert torch.all(g[:pad] == 333.0) and torch.all(g[pad + T:] == 333.0), "canary rows overwritten"
+    return o, lse, dq, dk, dv
+
+
+def check_bwd(counts, H, D, seed, scale=None):
+    T = int(sum(counts))
+    q, k, v, do = (W.normal_bf16(seed, s, (T, H, D)) for s in (1, 2, 3, 4))
+    scale = float(np.float32(1.0 / np.sqrt(D))) if scale is None else scale
+    _, _, dq, dk, dv = gpu_fwd_bwd(q, k, v, do, counts, scale)
+    cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    ref = oracle.attn_bwd(do, q, k, v, cu, scale)
+    errs = {}
+    for name, g, r in zip(("dq", "dk", "dv"), (dq, dk, dv), ref):
+        x = to_f64(g)
+        assert not np.isnan(x).any(), name
+        if np.linalg.norm(r) == 0:      # single-token segments only: dQ = dK = 0 exactly
+            assert np.abs(x).max() <= 1e-2, name
+            continue
+        errs[name] = rel_l2(x, r)
+        assert errs[name] <= GRAD_REL_L2, (counts, name, errs[name])
+    return errs
+
+
+def test_tiny_config():
+    w = W.tiny()
+    check_bwd(w.patch_counts, w.n_heads, w.head_dim, w.seed, w.softmax_scale)
+
+
+@pytest.mark.parametrize("D", [64, 80])
+@pytest.mark.parametrize("counts", [
+    [1], [16], [127], [128], [129], [255], [256], [257], [385], [700],
+    [1, 5, 0, 127, 128, 129, 0, 255, 256, 257, 300, 513],
+    [1040, 3, 260],
+])
+def test_ragged_segments(counts, D):
+    check_bwd(counts, 2, D, seed=200 + sum(counts) + D)
+
+
+@pytest.mark.parametrize("D", [64, 80])
+def test_many_units_per_cta(D):
+    counts = [int(x) for x in W.rand_int(19, 1, 24, 40, 900)]
+    check_bwd(counts, 8, D, seed=19)
+
+
+def test_frozen_backward_is_a_noop():
+    w = W.tiny()
+    q, k, v = w.qkv()
+    do = w.dout()
+    plan = B.seg_plan(w.patch_counts, B.FROZEN).to_device()
+    qd, kd, vd, dod = to_dev(q), to_dev(k), to_dev(v), to_dev(do)
+    o = torch.empty_like(qd)
+    B.varlen_attn_fwd(qd, kd, vd, o, None, plan, w.softmax_scale)
+    grads = [torch.full_like(qd, 5.0) for _ in range(3)]
+    B.varlen_attn_bwd(dod, qd, kd, vd, o, None, *grads, plan, w.softmax_scale, None)
+    torch.cuda.synchronize()
+    assert all(torch.all(g == 5.0) for g in grads)
+    assert plan.bwd_items.size == 0 and B.attn_workspace_bytes(229, 4, 64, B.FROZEN) == 0
+
+
+def test_gradient_identities_on_gpu_output():
+    """Properties that hold for the exact gradient at any size: sum_j dV_j = sum_i dO_i per (segment,
+    head), and <Q,dQ> = <K,dK>."""
+    counts = [513, 190]
+    T, H, D = sum(counts), 4, 64
+    q, k, v, do = (W.normal_bf16(29, s, (T, H, D)) for s in (1, 2, 3, 4))
+    _, _, dq, dk, dv = gpu_fwd_bwd(q, k, v, do, counts, 0.125)
+    qf, kf, dof = (W.bf16_bits_to_f64(x) for x in (q, k, do))
+    dqf, dkf, dvf = to_f64(dq), to_f64(dk), to_f64(dv)
+    cu = [0, 513, 703]
+    for s in range(2):
+        a, b = cu[s], cu[s + 1]
+        for h in range(H):
+            sv, sd = dvf[a:b, h].sum(0), dof[a:b, h].sum(0)
+            assert np.abs(sv - sd).max() <= 2e-2 * max(1.0, np.abs(sd).max())
+            lhs, rhs = (qf[a:b, h] * dqf[a:b, h]).sum(), (kf[a:b, h] * dkf[a:b, h]).sum()
+            assert abs(lhs - rhs) <= 2e-2 * max(1.0, abs(lhs))
+
+
+def _sampled_check(w, n_rows=96, n_kv=24, seed=7):
+    q, k, v = w.qkv()
+    do = w.dout()
+    _, _, dq, dk, dv = gpu_fwd_bwd(q, k, v, do, w.patch_counts, w.softmax_scale)
+    for g in (dq, dk, dv):
+        assert not torch.isnan(g.float()).any()
+    T, cu = w.total_tokens, w.cu_seqlens
+    rows = (W.rand_u64(seed, 1, n_rows) % np.uint64(T)).astype(np.int64)
+    heads = (W.rand_u64(seed, 2, n_rows) % np.uint64(w.n_heads)).astype(np.int32)
+    ref = oracle.attn_bwd_dq_rows(do, q, k, v, cu, w.softmax_scale, rows, heads)
+    got = to_f64(dq[torch.from_numpy(rows).cuda(), torch.from_numpy(heads.astype(np.int64)).cuda()])
+    assert rel_l2(got, ref) <= GRAD_REL_L2, ("dq", rel_l2(got, ref))
+    # dK / dV: a few key rows of three (segment, head) pairs: the longest segment, a middle one, the shortest
+    lens = np.diff(cu)
+    order = np.argsort(-lens, kind="stable")
+    nz = [int(s) for s in order if lens[s] > 0]
+    for pick, seg in enumerate((nz[0], nz[len(nz) // 2], nz[-1])):
+        head = int(W.rand_u64(seed, 10 + pick, 1)[0] % np.uint64(w.n_heads))
+        n = int(lens[seg])
+        kr = cu[seg] + (W.rand_u64(seed, 20 + pick, min(n_kv, n)) % np.uint64(n)).astype(np.int64)
+        kr = np.unique(np.concatenate([kr, [cu[seg], cu[seg + 1] - 1]]))
+        rk, rv = oracle.attn_bwd_dkv_rows(do, q, k, v, cu, w.softmax_scale, seg, head, kr)
+        idx = torch.from_numpy(kr).cuda()
+        assert rel_l2(to_f64(dk[idx, head]), rk) <= GRAD_REL_L2, ("dk", seg)
+        assert rel_l2(to_f64(dv[idx, head]), rv) <= GRAD_REL_L2, ("dv", seg)
+
+
+def test_vit_l_config_sampled():
+    _sampled_check(W.vit_l())
+
+
+def test_qwen2vl_config_sampled():
+    _sampled_check(W.qwen2vl(), n_rows=48, n_kv=12)
+
+
+def test_video_tail_config_sampled():
+    _sampled_check(W.video_tail(), n_rows=32, n_kv=8)
+
+
+@pytest.mark.parametrize("fraction", [0.10, 0.75])
+def test_modality_mix_sampled(fraction):
+    _sampled_check(W.modality_mix(fraction), n_rows=64, n_kv=16)
