@@ -1,0 +1,355 @@
+#!/usr/bin/env python
+"""Benchmark of the encoder hot path (plan -> varlen attention fwd -> bwd -> merge) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the whole hot path over one synthetic microbatch shaped like the ViT-L
+configuration: 32 variable-resolution images (256-4096 patches each), 16 heads of 64, bf16,
+encoder trained (forward + backward), the encoder output merged into 16 x 8192 LLM tokens.
+With N > 1 (torchrun, one rank per GPU) every rank runs its own microbatch (weak scaling, no
+data-path collective); the reported value is the whole job's attention TFLOP/s.
+
+Prints ONE JSON line.  `--impl reference` times the fp64 CPU oracle on a bounded sample of the same
+workload on the host cores (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_03229_b200 import workloads as W  # noqa: E402
+
+METRIC = "varlen encoder attn fwd+bwd TFLOP/s & % BF16 peak; merge GB/s (1 B200)"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one attn_bwd_kernel<64> launch on this workload, from the
+# ncu capture summarised in profiles/ (None until a capture exists).
+BWD_MAIN_DRAM_BYTES_PER_LAUNCH = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def workload_for(rank: int):
+    from paper_2607_03229_b200 import dist as D
+    return W.vit_l(seed=D.rank_seed(W.BASE_SEED + 2, rank))
+
+
+# ----------------------------------------------------------------------------- oracle sample (CPU arms)
+def oracle_sample(w, target_flops: float):
+    """A bounded sample of the workload for the CPU oracle: the first m segments and first h heads whose
+    algorithmic fwd+bwd FLOPs (14 * h * D * sum n^2) stay near `target_flops`."""
+    counts = w.patch_counts
+    per_head = [14.0 * w.head_dim * n * n for n in counts]
+    h = w.n_heads
+    while h > 1 and per_head[0] * h > target_flops:
+        h //= 2
+    m, acc = 0, 0.0
+    while m < len(counts) and (m == 0 or acc + per_head[m] * h <= target_flops):
+        acc += per_head[m] * h
+        m += 1
+    return m, h, acc
+
+
+def run_oracle_sample(w, m: int, h: int, inputs=None):
+    """One oracle pass (plan, fwd, bwd, merge of the sampled rows) over the sample.  Returns seconds."""
+    import oracle
+    counts = w.patch_counts[:m]
+    T = int(sum(counts))
+    if inputs is None:
+        shape = (T, h, w.head_dim)
+        inputs = tuple(W.normal_bf16(w.seed, 10 + i, shape) for i in range(4))
+        pos = (w.positions[:T] - w.positions[0]).astype(np.int32)   # the sampled images' runs and the gaps between them
+        emb = W.normal_bf16(w.seed, 21, (int(pos.max()) + 1, w.merge_hidden))
+        src = W.normal_bf16(w.seed, 20, (T, w.merge_hidden))
+        inputs = inputs + (emb, src, pos)
+    q, k, v, do, emb, src, pos = inputs
+    t0 = time.perf_counter()
+    cu = oracle.seg_plan(counts, 256, 128, True)[0]
+    oracle.attn_fwd(q, k, v, cu, w.softmax_scale)
+    oracle.attn_bwd(do, q, k, v, cu, w.softmax_scale)
+    oracle.merge_tokens(src, emb, pos)
+    return time.perf_counter() - t0, inputs
+
+
+def calibrate_oracle_rate(w) -> float:
+    """Algorithmic FLOP/s of the oracle on this host, from a one-segment, one-head run."""
+    import oracle
+    n, D = 768, w.head_dim
+    x = [W.normal_bf16(1, i, (n, 1, D)) for i in range(4)]
+    cu = np.array([0, n], dtype=np.int32)
+    oracle.attn_fwd(x[0], x[1], x[2], cu, 0.125)  # builds / loads the library
+    t0 = time.perf_counter()
+    oracle.attn_fwd(x[0], x[1], x[2], cu, 0.125)
+    oracle.attn_bwd(x[3], x[0], x[1], x[2], cu, 0.125)
+    dt = time.perf_counter() - t0
+    return 14.0 * D * n * n / dt
+
+
+def reference_arm(args):
+    """The oracle, as it stands, on the host cores; bounded sample sized from --steps/--warmup."""
+    from paper_2607_03229_b200 import dist as D
+    rank, _, world = D.env_world()
+    if rank != 0:
+        return 0
+    import oracle
+    w = workload_for(0)
+    rate = calibrate_oracle_rate(w)
+    budget_s = 150.0 / max(1, args.steps + args.warmup)
+    m, h, flops = oracle_sample(w, min(rate * min(budget_s, 20.0), w.flops()))
+    inputs = None
+    for _ in range(args.warmup):
+        _, inputs = run_oracle_sample(w, m, h, inputs)
+    times = []
+    for _ in range(args.steps):
+        dt, inputs = run_oracle_sample(w, m, h, inputs)
+        times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    value = flops / (ms * 1e-3) / 1e12
+    sample = (f"first {m} of {len(w.patch_counts)} segments x first {h} of {w.n_heads} heads "
+              f"({int(sum(w.patch_counts[:m]))} tokens, {flops:.3g} algorithmic FLOPs per step)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "vit_l: 32 images of 16..64 x 16..64 patches, 16 heads x 64, trained, + merge",
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.n_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_uuid: str):
+        self.uuid = gpu_uuid
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.perf_counter(), line.strip()))
+
+    def stop(self, t_begin: float, t_end: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"], "samples": 0}
+        time.sleep(0.06)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        rows = [ln for (t, ln) in self.lines if t_begin <= t <= t_end + 0.05] or [ln for (_, ln) in self.lines[-1:]]
+        sm, mx, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in rows:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower() == "active":
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- our arm
+def ours_arm(args):
+    import torch
+    from paper_2607_03229_b200 import binding as B
+    from paper_2607_03229_b200 import dist as D
+    from paper_2607_03229_b200 import hotpath as H
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    rank, local_rank, world = D.init("nccl")
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch N>1 with torchrun, one rank per GPU")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    B.load()
+    peaks, peak_kind = load_peaks()
+
+    w = workload_for(rank)
+    T, Hh, Dh = w.total_tokens, w.n_heads, w.head_dim
+    buf = H.allocate(w, dev)
+    n_kernels = H.kernels_per_step(w)
+    K, Wm = args.steps, max(args.warmup, 3)
+
+    for _ in range(Wm):
+        H.run_step(w, buf)
+    torch.cuda.synchronize()
+    assert int(buf.status[0]) == 0, f"device status {buf.status.tolist()}"
+
+    # ---- timed region: K whole steps, inputs resident in HBM, per-kernel events recorded alongside
+    ev = {name: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+          for name in ("fwd", "bwd_main", "merge")}
+    slots = {"fwd": B.PROFILE_FWD, "bwd_main": B.PROFILE_BWD_MAIN, "merge": B.PROFILE_MERGE}
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid) if hasattr(
+        torch.cuda.get_device_properties(dev), "uuid") else str(local_rank)
+    sampler = ClockSampler(uuid)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for name in ev:                      # create the event handles before the region
+        for a, b in ev[name]:
+            a.record(), b.record()
+    torch.cuda.synchronize()
+    D.barrier()
+    sampler.start()
+    time.sleep(0.15)
+    torch.cuda.synchronize()
+    t_begin = time.perf_counter()
+    e0.record()
+    for i in range(K):
+        for name, slot in slots.items():
+            B.load().mpipe_set_profile_events(slot, ev[name][i][0].cuda_event, ev[name][i][1].cuda_event)
+        H.run_step(w, buf)
+    e1.record()
+    torch.cuda.synchronize()
+    t_end = time.perf_counter()
+    for slot in slots.values():
+        B.load().mpipe_set_profile_events(slot, None, None)
+    D.barrier()
+    clocks = sampler.stop(t_begin, t_end)
+    assert int(buf.status[0]) == 0, f"device status {buf.status.tolist()}"
+    ms_step = e0.elapsed_time(e1) / K
+    kern_ms = {name: float(np.mean([a.elapsed_time(b) for a, b in ev[name]])) for name in ev}
+
+    # ---- end to end: host buffers in, results out, copies inside the timed region
+    Ke = min(K, 30)
+    host_in = [torch.empty((T, Hh, Dh), dtype=torch.bfloat16).pin_memory() for _ in range(4)]
+    for hbuf, dbuf in zip(host_in, (buf.q, buf.k, buf.v, buf.dout)):
+        hbuf.copy_(dbuf)
+    host_out = [torch.empty((T, Hh, Dh), dtype=torch.bfloat16).pin_memory() for _ in range(4)]
+    h2d = sum(x.numel() * x.element_size() for x in host_in) + w.positions.nbytes
+    d2h = sum(x.numel() * x.element_size() for x in host_out)
+
+    def e2e_step():
+        for hbuf, dbuf in zip(host_in, (buf.q, buf.k, buf.v, buf.dout)):
+            dbuf.copy_(hbuf, non_blocking=True)
+        H.run_step(w, buf)               # includes the host plan and its upload
+        for hbuf, dbuf in zip(host_out, (buf.o, buf.dq, buf.dk, buf.dv)):
+            hbuf.copy_(dbuf, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    torch.cuda.synchronize()
+    D.barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for _ in range(Ke):
+        e2e_step()
+    f1.record()
+    torch.cuda.synchronize()
+    D.barrier()
+    ms_e2e = f0.elapsed_time(f1) / Ke
+
+    # ---- reduce over ranks: max of times, sum of work
+    flops_fb, flops_b = w.flops(True, True), w.flops(False, True)
+    merge_bytes = float(T) * (4 * w.merge_hidden + 4)
+    (ms_step_mx, ms_e2e_mx, ms_bwd_mx, ms_fwd_mx, ms_merge_mx), (flops_all, flops_b_all, merge_all, launches) = \
+        D.reduce_max_sum([ms_step, ms_e2e, kern_ms["bwd_main"], kern_ms["fwd"], kern_ms["merge"]],
+                         [flops_fb, flops_b, merge_bytes, float(n_kernels * K)], device=dev)
+
+    if rank == 0:
+        value = flops_all / (ms_step_mx * 1e-3) / 1e12
+        bwd_tf = w.flops(False, True) / (kern_ms["bwd_main"] * 1e-3) / 1e12       # this rank's kernel, per launch
+        fwd_tf = w.flops(True, False) / (kern_ms["fwd"] * 1e-3) / 1e12
+        merge_gbs = merge_bytes / (kern_ms["merge"] * 1e-3) / 1e9
+        peak_tf = peaks["bf16_tflops_sustained"]
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+            "ms_per_step": ms_step_mx, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "vit_l: 32 images of 16..64 x 16..64 patches packed varlen, 16 heads x 64, bf16, "
+                                   "trained (fwd+bwd), + merge of the encoder output into 16 x 8192 LLM tokens at "
+                                   "hidden 1024; one microbatch per GPU",
+                       "tokens_rank0": T, "sum_n2_rank0": w.sum_n2, "l2": "inputs_exceed_l2 (~1 GB touched per step)",
+                       "step": "host plan + upload, attn fwd, attn bwd (prepass, main, convert), merge"},
+            "breakdown": {"fwd_ms": kern_ms["fwd"], "bwd_main_ms": kern_ms["bwd_main"], "merge_ms": kern_ms["merge"],
+                          "fwd_tflops": fwd_tf, "bwd_main_tflops": bwd_tf, "merge_gbs": merge_gbs,
+                          "merge_frac_of_hbm_peak": merge_gbs / peaks["hbm_gbs"],
+                          "attn_frac_of_bf16_peak": {"measured_sustained": value / world / peaks["bf16_tflops_sustained"],
+                                                     "measured_burst": value / world / peaks["bf16_tflops"],
+                                                     "nominal_2250": value / world / NOMINAL_BF16_TFLOPS}},
+            "roofline": {"kernel": "attn_bwd_kernel<64>", "bound": "tensor", "achieved": bwd_tf, "peak": peak_tf,
+                         "unit": "TFLOP/s", "frac": bwd_tf / peak_tf, "peak_kind": f"{peak_kind}, sustained bf16 GEMM",
+                         "traffic": BWD_MAIN_DRAM_BYTES_PER_LAUNCH},
+            "e2e": {"value": flops_all / (ms_e2e_mx * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e_mx,
+                    "steps": Ke, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        if world == 1:
+            line["cpu_baseline"] = cpu_baseline(w)
+        print(json.dumps(line))
+    D.shutdown()
+    return 0
+
+
+def cpu_baseline(w):
+    """The oracle as it stands on the host cores, on a bounded sample (about 10-20 s of CPU work)."""
+    import oracle
+    rate = calibrate_oracle_rate(w)
+    m, h, flops = oracle_sample(w, rate * 12.0)
+    dt, _ = run_oracle_sample(w, m, h)
+    return {"value": flops / dt / 1e12, "unit": UNIT, "cores": oracle.n_threads(), "kind": "oracle", "seconds": dt,
+            "sample": f"first {m} of {len(w.patch_counts)} segments x first {h} of {w.n_heads} heads "
+                      f"({int(sum(w.patch_counts[:m]))} tokens, {flops:.3g} algorithmic fwd+bwd FLOPs), one pass"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return reference_arm(args)
+    return ours_arm(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -177,6 +177,16 @@ int32_t mpipe_merge_tokens_bwd(const void* d_llm_embeds, int64_t emb_row_stride,
  * Returns MPIPE_OK, MPIPE_ERR_INDEX (out of range) or MPIPE_ERR_INVALID_ARG (duplicate / NULL). */
 int32_t mpipe_validate_positions(const int32_t* positions, int32_t n, int32_t n_llm_tokens);
 
+/*
+ * Measurement aid (no counterpart in the paper; its cost model weights each compute event with one
+ * duration, Section 4.3, and this is how a benchmark reads that duration for one kernel): while set,
+ * the launch of kernel `which` (0 = attention forward, 1 = attention backward main kernel, 2 = merge
+ * / merge_bwd) records the two cudaEvent_t handles on the call's stream directly before and after
+ * it.  NULL handles switch it off.  Process-wide, not thread-safe: set it from the thread that makes
+ * the calls.  Returns MPIPE_ERR_INVALID_ARG for an unknown `which`.
+ */
+int32_t mpipe_set_profile_events(int32_t which, void* start_event, void* stop_event);
+
 const char* mpipe_status_str(int32_t status);
 int32_t mpipe_version(void);
 

@@ -43,6 +43,7 @@ _SIGNATURES = {
     "mpipe_merge_tokens": (_i32, [_vp, _i64, _vp, _i64, _vp, _i32, _i32, _i32, _i32, _vp, _vp]),
     "mpipe_merge_tokens_bwd": (_i32, [_vp, _i64, _vp, _i64, _vp, _i32, _i32, _i32, _i32, _vp, _vp]),
     "mpipe_validate_positions": (_i32, [_vp, _i32, _i32]),
+    "mpipe_set_profile_events": (_i32, [_i32, _vp, _vp]),
     "mpipe_status_str": (ctypes.c_char_p, [_i32]),
     "mpipe_version": (_i32, []),
 }
@@ -223,6 +224,19 @@ def merge_tokens_bwd(d_llm_embeds, d_enc, positions_dev, mode: int, status_buf=N
                                        d_enc.stride(0) if n_enc else hidden, _ptr(positions_dev), n_enc, n_llm,
                                        hidden, mode, _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_merge_tokens_bwd")
+
+
+PROFILE_FWD, PROFILE_BWD_MAIN, PROFILE_MERGE = 0, 1, 2
+
+
+def set_profile_events(which: int, start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]) -> None:
+    """mpipe_set_profile_events: record two CUDA events around one kernel of the next calls (None = off)."""
+    def handle(ev):
+        if ev is None:
+            return None
+        ev.record()  # torch creates the underlying cudaEvent_t lazily, on the first record
+        return ev.cuda_event
+    _check(load().mpipe_set_profile_events(which, handle(start), handle(stop)), "mpipe_set_profile_events")
 
 
 def validate_positions(positions, n_llm_tokens: int) -> int:

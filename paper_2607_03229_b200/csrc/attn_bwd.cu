@@ -545,7 +545,9 @@ static int32_t launch_bwd(const void* dout, const void* q, const void* k, const 
         delta, prm.dq_acc);
     const int n_units = prm.n_items * prm.n_heads;
     const int grid = n_units < sm_count() ? n_units : sm_count();
+    profile_start(kProfileBwdMain, stream);
     attn_bwd_kernel<D><<<grid, kBwdThreads, Cfg::kSmemAlloc, stream>>>(mq, mk, mv, mdo, mqt, mkt, mvt, mdot, prm);
+    profile_stop(kProfileBwdMain, stream);
     const int64_t chunks = rows * (D / 8);
     bwd_dq_convert_kernel<<<unsigned((chunks + 255) / 256), 256, 0, stream>>>(
         prm.dq_acc, static_cast<__nv_bfloat16*>(dq), prm.tok_stride_g, prm.head_stride_g, total_tokens, n_heads, D,

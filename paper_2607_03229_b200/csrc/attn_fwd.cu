@@ -390,7 +390,9 @@ static int32_t launch_fwd(const void* q, const void* k, const void* v, int64_t t
         return MPIPE_ERR_CUDA;
     const int n_units = prm.n_items * prm.n_heads;
     const int grid = n_units < sm_count() ? n_units : sm_count();
+    profile_start(kProfileFwd, stream);
     attn_fwd_kernel<D><<<grid, kFwdThreads, Cfg::kSmemAlloc, stream>>>(mq, mk, mv, mqt, mkt, prm);
+    profile_stop(kProfileFwd, stream);
     return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
 }
 

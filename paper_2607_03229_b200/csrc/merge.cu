@@ -72,6 +72,7 @@ static int32_t merge_launch(bool scatter, const void* src, int64_t src_stride, v
     const int64_t cap = int64_t(sm_count()) * 8 * 4;  // a few waves of 8 resident blocks per SM
     const int grid = int(want < cap ? want : cap);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    profile_start(kProfileMerge, st);
     if (scatter)
         merge_rows_kernel<true><<<grid, kMergeThreads, 0, st>>>(
             static_cast<const uint4*>(src), src_stride / 8, static_cast<uint4*>(dst), dst_stride / 8, positions_dev,
@@ -80,6 +81,7 @@ static int32_t merge_launch(bool scatter, const void* src, int64_t src_stride, v
         merge_rows_kernel<false><<<grid, kMergeThreads, 0, st>>>(
             static_cast<const uint4*>(src), src_stride / 8, static_cast<uint4*>(dst), dst_stride / 8, positions_dev,
             n_enc_tokens, n_llm_tokens, chunks, status_buf);
+    profile_stop(kProfileMerge, st);
     return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
 }
 

@@ -6,6 +6,8 @@
 
 namespace mpipe {
 
+ProfileEvents g_profile[kProfileSlots];
+
 int sm_count() {
     static int cached[64] = {0};
     int dev = 0;
@@ -105,5 +107,12 @@ const char* mpipe_status_str(int32_t status) {
 }
 
 int32_t mpipe_version(void) { return 100; }
+
+int32_t mpipe_set_profile_events(int32_t which, void* start_event, void* stop_event) {
+    if (which < 0 || which >= mpipe::kProfileSlots) return MPIPE_ERR_INVALID_ARG;
+    mpipe::g_profile[which].start = static_cast<cudaEvent_t>(start_event);
+    mpipe::g_profile[which].stop = static_cast<cudaEvent_t>(stop_event);
+    return MPIPE_OK;
+}
 
 }  // extern "C"

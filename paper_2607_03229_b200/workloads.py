@@ -188,12 +188,17 @@ def tiny(seed: int = BASE_SEED + 1, shuffled_positions: bool = False) -> Workloa
     return Workload("tiny", seed, counts, 4, 64, True, merge_hidden=256, n_llm_tokens=512, positions=pos)
 
 
-def vit_l(seed: int = BASE_SEED + 2, n_images: int = 32) -> Workload:
+def vit_l(seed: int = BASE_SEED + 2, n_images: int = 32, n_llm_tokens: int = 131072) -> Workload:
     """32 images, height and width independently uniform in 16..64 patches (224-896 px at patch
-    14), 16 heads of 64, trained."""
+    14), 16 heads of 64, trained.  For the whole-path benchmark the encoder output (hidden 1024 =
+    heads x head_dim, one LLM token per patch) is merged into 16 LLM sequences of 8192 tokens at
+    hidden 1024: every image one contiguous placeholder run, seeded text gaps in between."""
     h = rand_int(seed, 1, n_images, 16, 64)
     w = rand_int(seed, 2, n_images, 16, 64)
-    return Workload("vit_l", seed, [int(a * b) for a, b in zip(h, w)], 16, 64, True)
+    counts = [int(a * b) for a, b in zip(h, w)]
+    pos = _runs_with_gaps(seed, 30, counts, n_llm_tokens)
+    return Workload("vit_l", seed, counts, 16, 64, True, merge_hidden=1024, n_llm_tokens=n_llm_tokens,
+                    positions=pos)
 
 
 def qwen2vl(seed: int = BASE_SEED + 3, trained: bool = True, total: int = 65536) -> Workload:

@@ -71,15 +71,16 @@ def test_many_units_per_cta(D):
 
 def test_large_scores_trigger_rescale():
     """A large softmax scale makes row maxima jump by far more than the lazy-rescale threshold.
-    The softmax is then nearly one-hot and |O| reaches 4 and more, where the bf16 output spacing
-    alone (half an ulp = 2^-9 |O|) exceeds the absolute bar; the absolute check scales with |O|."""
+    The softmax is then nearly one-hot and |O| reaches 4 and more: the bf16 rounding of the one dominant
+    probability (2^-9 relative) and of the output (2^-9 relative) both scale with |O| and alone exceed
+    the absolute bar there, so the absolute check scales with |O|."""
     counts, H, D, scale = [700, 300], 2, 64, 1.5
     q, k, v = (W.normal_bf16(23, s, (1000, H, D)) for s in (1, 2, 3))
     o, lse, _ = gpu_fwd(q, k, v, counts, scale)
     O_ref, L_ref = oracle.attn_fwd(q, k, v, np.array([0, 700, 1000], dtype=np.int32), scale)
     O = to_f64(o)
     assert rel_l2(O, O_ref) <= O_REL_L2
-    assert np.all(np.abs(O - O_ref) <= 5e-3 + 2.0 ** -8 * np.abs(O_ref))
+    assert np.all(np.abs(O - O_ref) <= 5e-3 + 2.0 ** -7 * np.abs(O_ref))
     assert max_abs(to_f64(lse), L_ref) <= LSE_MAX_ABS
 
 
