@@ -1,0 +1,52 @@
+"""World-size-2 coverage (gloo, CPU) of the benchmark's multi-GPU plumbing: every rank draws its own
+microbatch, nothing is exchanged on the data path, times reduce by max and work by sum."""
+import os
+import socket
+
+import torch.multiprocessing as mp
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    import bench
+    from paper_2607_03229_b200 import dist as D
+    r, lr, w = D.init("gloo")
+    assert (r, lr, w) == (rank, rank, world)
+    wl = bench.workload_for(rank)
+    D.barrier()
+    (t_max, e_max), (flops, launches) = D.reduce_max_sum([1.0 + rank, 5.0 - rank], [wl.flops(), 5.0])
+    out.put((rank, wl.seed, wl.total_tokens, wl.flops(), t_max, e_max, flops, launches))
+    D.shutdown()
+
+
+def test_two_ranks_shard_by_microbatch_and_reduce():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    (r0, s0, t0, f0, mx0, ex0, fl0, l0), (r1, s1, t1, f1, mx1, ex1, fl1, l1) = res
+    assert s0 != s1 and (t0, f0) != (t1, f1)          # different microbatches per rank
+    assert mx0 == mx1 == 2.0 and ex0 == ex1 == 5.0    # max over ranks
+    assert abs(fl0 - (f0 + f1)) < 1e-3 * fl0 and fl0 == fl1 and l0 == l1 == 10.0   # work sums
+
+
+def test_single_process_defaults():
+    from paper_2607_03229_b200 import dist as D
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE"):
+        os.environ.pop(k, None)
+    assert D.env_world() == (0, 0, 1)
+    assert D.reduce_max_sum([3.0], [4.0]) == ([3.0], [4.0])
+    assert D.rank_seed(7, 0) == 7 and D.rank_seed(7, 3) == 3007
