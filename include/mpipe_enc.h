@@ -146,6 +146,43 @@ int32_t mpipe_varlen_attn_bwd(const void* dout, const void* q, const void* k, co
                               size_t workspace_bytes, int32_t* status_buf, void* stream);
 
 /*
+ * The same backward for callers that are not allowed to allocate device memory.  (The paper has no
+ * counterpart: it never discusses where kernel scratch comes from.)
+ *
+ * Who needs it: a pipeline runtime that hands out all device memory from a plan fixed before the
+ * step and exposes no allocator to the code it runs in the bubbles; a host process whose device
+ * memory belongs to another component's pool; a latency-critical loop in which cudaMalloc is
+ * banned because it synchronises the whole device.  Such callers cannot produce the `workspace` of
+ * mpipe_varlen_attn_bwd, so this variant keeps the scratch (fp32 dQ accumulator + Delta) inside the
+ * library, in a fixed 32 MiB device array (mpipe_attn_bwd_static_scratch_bytes()).  Every GPU that
+ * loads the library holds those 32 MiB until the process exits, used or not.
+ *
+ *   - Arguments, layouts, results and error behaviour are those of mpipe_varlen_attn_bwd, minus
+ *     workspace / workspace_bytes.  Inputs and outputs are still the caller's buffers.
+ *   - Limit: mpipe_attn_workspace_bytes(total_tokens, n_heads, head_dim, TRAINED) must not exceed
+ *     the 32 MiB (e.g. 8000 tokens x 16 heads x 64).  Larger problems are refused with
+ *     MPIPE_ERR_WORKSPACE before anything is launched; use mpipe_varlen_attn_bwd for them.
+ *   - The call itself allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
+ *     The first call on each device looks up the array's device address once, with that device
+ *     current; make that first call before starting any stream capture.  A failed look-up returns
+ *     MPIPE_ERR_CUDA.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left in
+ *     it.  Nothing needs to be cleared by the caller: each call's first kernel zeroes the
+ *     accumulator and rewrites Delta for its own problem.  Because the array is shared, two calls
+ *     whose kernels may overlap on the GPU (different streams, no dependency between them) race on
+ *     it and produce garbage: serialise them.
+ */
+size_t mpipe_attn_bwd_static_scratch_bytes(void);
+int32_t mpipe_varlen_attn_bwd_static(const void* dout, const void* q, const void* k, const void* v, const void* o,
+                                     const float* lse, void* dq, void* dk, void* dv, int64_t tok_stride_qkv,
+                                     int64_t head_stride_qkv, int64_t tok_stride_o, int64_t head_stride_o,
+                                     int64_t tok_stride_grad, int64_t head_stride_grad,
+                                     const int32_t* cu_seqlens_dev, int32_t n_seg, int32_t total_tokens,
+                                     int32_t max_seqlen, const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items,
+                                     int32_t n_heads, int32_t head_dim, float softmax_scale, int32_t mode,
+                                     int32_t* status_buf, void* stream);
+
+/*
  * (4) Local half of Coll(Gather, (enc, llm), m), the Replicated->Sharded seam of Table 2: encoder
  * token i is written over row positions[i] of the LLM input-embedding buffer, in place:
  *     llm_embeds[positions[i], 0:hidden] = enc_tokens[i, 0:hidden].

@@ -40,6 +40,9 @@ _SIGNATURES = {
                                      _i32, _i32, _i32, _f32, _i32, _vp, _vp]),
     "mpipe_varlen_attn_bwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _i64, _i64,
                                      _vp, _i32, _i32, _i32, _vp, _i32, _i32, _i32, _f32, _i32, _vp, _sz, _vp, _vp]),
+    "mpipe_attn_bwd_static_scratch_bytes": (_sz, []),
+    "mpipe_varlen_attn_bwd_static": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _i64,
+                                            _i64, _vp, _i32, _i32, _i32, _vp, _i32, _i32, _i32, _f32, _i32, _vp, _vp]),
     "mpipe_merge_tokens": (_i32, [_vp, _i64, _vp, _i64, _vp, _i32, _i32, _i32, _i32, _vp, _vp]),
     "mpipe_merge_tokens_bwd": (_i32, [_vp, _i64, _vp, _i64, _vp, _i32, _i32, _i32, _i32, _vp, _vp]),
     "mpipe_validate_positions": (_i32, [_vp, _i32, _i32]),
@@ -200,6 +203,27 @@ def varlen_attn_bwd(dout, q, k, v, o, lse, dq, dk, dv, plan: SegPlan, softmax_sc
         _ptr(plan.bwd_items_dev), int(plan.bwd_items.size), H, D, softmax_scale, plan.mode, _ptr(workspace),
         ws_bytes, _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_varlen_attn_bwd")
+
+
+def attn_bwd_static_scratch_bytes() -> int:
+    return load().mpipe_attn_bwd_static_scratch_bytes()
+
+
+def varlen_attn_bwd_static(dout, q, k, v, o, lse, dq, dk, dv, plan: SegPlan, softmax_scale: float, status_buf=None,
+                           stream=None) -> None:
+    """mpipe_varlen_attn_bwd_static: the backward with the library's built-in 32 MiB scratch, for callers
+    that may not allocate device memory.  Same tensors as varlen_attn_bwd, no workspace argument; problems
+    whose scratch would not fit are refused with ERR_WORKSPACE.  Calls sharing a device must not overlap."""
+    T, H, D = q.shape
+    ts, hs = _thd_strides(q)
+    tso, hso = _thd_strides(o)
+    tsg, hsg = _thd_strides(dq) if plan.mode == TRAINED else (ts, hs)
+    st = load().mpipe_varlen_attn_bwd_static(
+        _ptr(dout), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(dq), _ptr(dk), _ptr(dv), ts, hs, tso, hso,
+        tsg, hsg, _ptr(plan.cu_seqlens_dev), plan.n_seg, plan.total_tokens, plan.max_seqlen,
+        _ptr(plan.bwd_items_dev), int(plan.bwd_items.size), H, D, softmax_scale, plan.mode, _ptr(status_buf),
+        _stream(stream))
+    _check(st, "mpipe_varlen_attn_bwd_static")
 
 
 def merge_tokens(enc_tokens, llm_embeds, positions_dev, mode: int = TRAINED, status_buf=None, stream=None) -> None:

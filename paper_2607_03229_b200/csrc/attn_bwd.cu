@@ -627,4 +627,61 @@ int32_t mpipe_varlen_attn_bwd(const void* dout, const void* q, const void* k, co
                           total_tokens, n_heads, prm, delta, st);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Backward for callers that cannot allocate: the scratch lives inside the library.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+// Scratch of mpipe_varlen_attn_bwd_static: fp32 dQ accumulator + Delta of one call.  Every GPU that
+// loads this library carries these 32 MiB from load until the process exits.
+constexpr size_t kStaticScratchBytes = size_t(32) << 20;
+static __device__ __align__(256) unsigned char g_bwd_static_scratch[kStaticScratchBytes];
+
+// Device address of the array, looked up once per device.  On the host the array's name is only a
+// stand-in symbol, not a device address, so kernels must be given the looked-up pointer.
+void* g_bwd_static_scratch_ptr[64] = {nullptr};
+
+int32_t static_scratch_for_current_device(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MPIPE_ERR_CUDA;
+    if (g_bwd_static_scratch_ptr[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_bwd_static_scratch) != cudaSuccess || ptr == nullptr) {
+            (void)cudaGetLastError();
+            return MPIPE_ERR_CUDA;
+        }
+        g_bwd_static_scratch_ptr[dev] = ptr;
+    }
+    *out = g_bwd_static_scratch_ptr[dev];
+    return MPIPE_OK;
+}
+
+}  // namespace
+
+size_t mpipe_attn_bwd_static_scratch_bytes(void) { return kStaticScratchBytes; }
+
+int32_t mpipe_varlen_attn_bwd_static(const void* dout, const void* q, const void* k, const void* v, const void* o,
+                                     const float* lse, void* dq, void* dk, void* dv, int64_t tok_stride_qkv,
+                                     int64_t head_stride_qkv, int64_t tok_stride_o, int64_t head_stride_o,
+                                     int64_t tok_stride_grad, int64_t head_stride_grad,
+                                     const int32_t* cu_seqlens_dev, int32_t n_seg, int32_t total_tokens,
+                                     int32_t max_seqlen, const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items,
+                                     int32_t n_heads, int32_t head_dim, float softmax_scale, int32_t mode,
+                                     int32_t* status_buf, void* stream) {
+    if (mode != MPIPE_ENC_FROZEN && mode != MPIPE_ENC_TRAINED) return MPIPE_ERR_INVALID_ARG;
+    if (mode == MPIPE_ENC_FROZEN) return MPIPE_OK;
+    if (total_tokens < 0 || n_heads <= 0 || head_dim <= 0) return MPIPE_ERR_INVALID_ARG;
+    // The problem must fit the built-in scratch; larger ones have to use mpipe_varlen_attn_bwd.
+    if (mpipe_attn_workspace_bytes(total_tokens, n_heads, head_dim, mode) > kStaticScratchBytes)
+        return MPIPE_ERR_WORKSPACE;
+    void* scratch = nullptr;
+    const int32_t rc = static_scratch_for_current_device(&scratch);
+    if (rc != MPIPE_OK) return rc;
+    return mpipe_varlen_attn_bwd(dout, q, k, v, o, lse, dq, dk, dv, tok_stride_qkv, head_stride_qkv, tok_stride_o,
+                                 head_stride_o, tok_stride_grad, head_stride_grad, cu_seqlens_dev, n_seg,
+                                 total_tokens, max_seqlen, bwd_items_dev, n_bwd_items, n_heads, head_dim,
+                                 softmax_scale, mode, scratch, kStaticScratchBytes, status_buf, stream);
+}
+
 }  // extern "C"
