@@ -29,6 +29,23 @@
 
 namespace mpipe {
 
+// Development aid, compiled in only with -DMPIPE_TRACE: CTA 0 records clock64() at a few pipeline
+// points per role into a global table that mpipe_dbg_read_trace() copies out.
+#ifdef MPIPE_TRACE
+__device__ long long g_trace[4][4096];
+__device__ int g_dbg_flags;   // knock-out switches for experiments: 1 no atomics, 2 no dS smem store, 4 no LSE/Delta smem loads, 8 no ex2
+#define MPIPE_DBG(bit) ((g_dbg_flags & (bit)) != 0)
+#define MPIPE_TR(role, idx)                                                                  \
+    do {                                                                                     \
+        if (blockIdx.x == 0 && (idx) < 4096) g_trace[role][(idx)] = clock64();               \
+    } while (0)
+#else
+#define MPIPE_DBG(bit) false
+#define MPIPE_TR(role, idx) \
+    do {                    \
+    } while (0)
+#endif
+
 constexpr int kBwdThreads = 512;
 constexpr int kBT = 128;  // keys per unit = query rows per iteration = TMEM lanes
 
@@ -160,35 +177,44 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ tcgen05 issuer
+        // The whole warp walks the loop (uniform control flow); one elected lane issues and commits.
+        // Descriptors are precomputed halves: a K-step only adds a constant to the low word.
         setmaxnreg_dec<72>();
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             const uint32_t sbase = smem_u32(smem);
-            const uint32_t ka = sbase + Cfg::kSmemK, va = sbase + Cfg::kSmemV, dsa = sbase + Cfg::kSmemDS;
+            constexpr uint32_t hi128 = umma_desc_hi(1024, kSwizzle128);
+            constexpr uint32_t hi32 = umma_desc_hi(256, kSwizzle32);
+            const uint32_t k_lo = umma_desc_lo(sbase + Cfg::kSmemK, 0), v_lo = umma_desc_lo(sbase + Cfg::kSmemV, 0);
+            const uint32_t kt_lo = umma_desc_lo(sbase + Cfg::kSmemK + Cfg::kTileMain, 0);
+            const uint32_t vt_lo = umma_desc_lo(sbase + Cfg::kSmemV + Cfg::kTileMain, 0);
+            const uint32_t ds_lo = umma_desc_lo(sbase + Cfg::kSmemDS, kBT * 128);   // two 64-query atoms 16 KB apart
             constexpr uint32_t idesc_s = umma_idesc_bf16(kBT, kBT, 0, 0);      // K-major x K-major, N = 128 queries
             constexpr uint32_t idesc_ts = umma_idesc_bf16(kBT, 64, 0, 1);      // A in TMEM, MN-major B, N = 64
             constexpr uint32_t idesc_ts_t = umma_idesc_bf16(kBT, 16, 0, 1);    // same, 16-wide head-dim tail
             constexpr uint32_t idesc_dq = umma_idesc_bf16(kBT, 64, 1, 1);      // MN-major A and B
             constexpr uint32_t idesc_dq_t = umma_idesc_bf16(kBT, 16, 1, 1);
-            // dst[128 x 128] = A[128 x D] * B[128 x D]^T, both K-major tiles (main 64 + optional 16 tail)
-            auto issue_kk = [&](uint32_t dcol, uint32_t a, uint32_t b) {
+            // dst[128 x 128] = A[128 x D] * B[128 x D]^T, both K-major tiles (main 64 + optional 16 tail);
+            // a / b are the low descriptor words of the main tiles, at / bt of the tails
+            auto issue_kk = [&](uint32_t dcol, uint32_t a, uint32_t at, uint32_t b, uint32_t bt) {
+                if (leader) {
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_ss(tmem + dcol, umma_smem_desc(a + ks * 32, 0, 1024, kSwizzle128),
-                            umma_smem_desc(b + ks * 32, 0, 1024, kSwizzle128), idesc_s, ks > 0);
-                if (Cfg::kTail)
-                    umma_ss(tmem + dcol, umma_smem_desc(a + Cfg::kTileMain, 0, 256, kSwizzle32),
-                            umma_smem_desc(b + Cfg::kTileMain, 0, 256, kSwizzle32), idesc_s, 1);
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_ss(tmem + dcol, umma_desc(a + ks * 2, hi128), umma_desc(b + ks * 2, hi128), idesc_s, ks > 0);
+                    if (Cfg::kTail) umma_ss(tmem + dcol, umma_desc(at, hi32), umma_desc(bt, hi32), idesc_s, 1);
+                }
             };
             // dst[128 keys x D] (+)= A^T-in-TMEM[128 keys x 128 q] * B[128 q x D] (B tile rows = q, MN-major)
-            auto issue_ts = [&](uint32_t dcol, uint32_t acol, uint32_t b, bool acc) {
+            auto issue_ts = [&](uint32_t dcol, uint32_t acol, uint32_t b, uint32_t bt, bool acc) {
+                if (leader) {
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t a_t = tmem + acol + (ks < 4 ? ks * 8 : 64 + (ks - 4) * 8);
-                    umma_ts(tmem + dcol, a_t, umma_smem_desc(b + ks * 2048, 0, 1024, kSwizzle128), idesc_ts,
-                            (acc || ks > 0) ? 1u : 0u);
-                    if (Cfg::kTail)
-                        umma_ts(tmem + dcol + 64, a_t, umma_smem_desc(b + Cfg::kTileMain + ks * 512, 0, 256, kSwizzle32),
-                                idesc_ts_t, (acc || ks > 0) ? 1u : 0u);
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint32_t a_t = tmem + acol + (ks < 4 ? ks * 8 : 64 + (ks - 4) * 8);
+                        umma_ts(tmem + dcol, a_t, umma_desc(b + ks * 128, hi128), idesc_ts, (acc || ks > 0) ? 1u : 0u);
+                        if (Cfg::kTail)
+                            umma_ts(tmem + dcol + 64, a_t, umma_desc(bt + ks * 32, hi32), idesc_ts_t,
+                                    (acc || ks > 0) ? 1u : 0u);
+                    }
                 }
             };
             uint32_t unit_it = 0, it_cnt = 0;
@@ -204,59 +230,66 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 {
                     const uint32_t qa = sbase + Cfg::kSmemQ + (it_cnt & 1) * Cfg::kTile;
                     const uint32_t da = sbase + Cfg::kSmemDO + (it_cnt & 1) * Cfg::kTile;
-                    issue_kk(Cfg::kColS, ka, qa);
-                    umma_commit(&bars.s_full);
-                    issue_kk(Cfg::kColDP, va, da);
-                    umma_commit(&bars.dp_full);
+                    issue_kk(Cfg::kColS, k_lo, kt_lo, umma_desc_lo(qa, 0), umma_desc_lo(qa + Cfg::kTileMain, 0));
+                    if (leader) umma_commit(&bars.s_full);
+                    issue_kk(Cfg::kColDP, v_lo, vt_lo, umma_desc_lo(da, 0), umma_desc_lo(da + Cfg::kTileMain, 0));
+                    if (leader) umma_commit(&bars.dp_full);
                 }
                 for (int i = 0; i < nq; ++i, ++it_cnt) {
                     const int st = it_cnt & 1;
-                    const uint32_t qa = sbase + Cfg::kSmemQ + st * Cfg::kTile;
-                    const uint32_t da = sbase + Cfg::kSmemDO + st * Cfg::kTile;
-                    const uint32_t qa_n = sbase + Cfg::kSmemQ + (st ^ 1) * Cfg::kTile;
-                    const uint32_t da_n = sbase + Cfg::kSmemDO + (st ^ 1) * Cfg::kTile;
+                    const uint32_t q_lo = umma_desc_lo(sbase + Cfg::kSmemQ + st * Cfg::kTile, 0);
+                    const uint32_t d_lo = umma_desc_lo(sbase + Cfg::kSmemDO + st * Cfg::kTile, 0);
+                    const uint32_t qn_lo = umma_desc_lo(sbase + Cfg::kSmemQ + (st ^ 1) * Cfg::kTile, 0);
+                    const uint32_t dn_lo = umma_desc_lo(sbase + Cfg::kSmemDO + (st ^ 1) * Cfg::kTile, 0);
+                    constexpr uint32_t kTailOff = Cfg::kTileMain >> 4;
                     const bool more = (i + 1 < nq);
                     if (i == 0) {
                         ok = mbar_wait(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag);
                         if (!ok) break;
                     }
+                    MPIPE_TR(0, it_cnt * 8 + 0);
                     ok = mbar_wait(&bars.p_full, it_cnt & 1, &abort_flag);
                     if (!ok) break;
+                    MPIPE_TR(0, it_cnt * 8 + 1);
                     tc_fence_after();
-                    issue_ts(Cfg::kColDV, Cfg::kColS, da, i > 0);                 // dV += P^T dO
+                    issue_ts(Cfg::kColDV, Cfg::kColS, d_lo, d_lo + kTailOff, i > 0);                 // dV += P^T dO
                     if (more) {
                         ok = mbar_wait(&bars.qdo_full[st ^ 1], ((it_cnt + 1) >> 1) & 1, &abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        issue_kk(Cfg::kColS, ka, qa_n);                           // S^T(i+1)
-                        umma_commit(&bars.s_full);
+                        issue_kk(Cfg::kColS, k_lo, kt_lo, qn_lo, qn_lo + kTailOff);                          // S^T(i+1)
+                        if (leader) umma_commit(&bars.s_full);
                     }
+                    MPIPE_TR(0, it_cnt * 8 + 2);
                     ok = mbar_wait(&bars.ds_full, it_cnt & 1, &abort_flag);
                     if (!ok) break;
+                    MPIPE_TR(0, it_cnt * 8 + 3);
                     tc_fence_after();
-                    issue_ts(Cfg::kColDK, Cfg::kColDP, qa, i > 0);                // dK += dS^T Q
+                    issue_ts(Cfg::kColDK, Cfg::kColDP, q_lo, q_lo + kTailOff, i > 0);                // dK += dS^T Q
                     ok = mbar_wait(&bars.dq_empty, (it_cnt & 1) ^ 1, &abort_flag);
                     if (!ok) break;
+                    MPIPE_TR(0, it_cnt * 8 + 4);
                     tc_fence_after();
+                    if (leader) {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {                              // dQ_i = dS K
-                        const uint64_t adesc = umma_smem_desc(dsa + ks * 2048, kBT * 128, 1024, kSwizzle128);
-                        umma_ss(tmem + Cfg::kColDQ, adesc, umma_smem_desc(ka + ks * 2048, 0, 1024, kSwizzle128), idesc_dq,
-                                ks > 0);
-                        if (Cfg::kTail)
-                            umma_ss(tmem + Cfg::kColDQ + 64, adesc,
-                                    umma_smem_desc(ka + Cfg::kTileMain + ks * 512, 0, 256, kSwizzle32), idesc_dq_t, ks > 0);
+                        for (int ks = 0; ks < 8; ++ks) {                          // dQ_i = dS K
+                            const uint64_t adesc = umma_desc(ds_lo + ks * 128, hi128);
+                            umma_ss(tmem + Cfg::kColDQ, adesc, umma_desc(k_lo + ks * 128, hi128), idesc_dq, ks > 0);
+                            if (Cfg::kTail)
+                                umma_ss(tmem + Cfg::kColDQ + 64, adesc, umma_desc(kt_lo + ks * 32, hi32), idesc_dq_t, ks > 0);
+                        }
                     }
-                    umma_commit(&bars.dq_full);
-                    umma_commit(&bars.qdo_empty[st]);
+                    if (leader) umma_commit(&bars.dq_full);
+                    if (leader) umma_commit(&bars.qdo_empty[st]);
                     if (more) {
-                        issue_kk(Cfg::kColDP, va, da_n);                          // dP^T(i+1)
-                        umma_commit(&bars.dp_full);
+                        issue_kk(Cfg::kColDP, v_lo, vt_lo, dn_lo, dn_lo + kTailOff);                         // dP^T(i+1)
+                        if (leader) umma_commit(&bars.dp_full);
                     }
+                    MPIPE_TR(0, it_cnt * 8 + 5);
                 }
                 if (!ok) break;
-                umma_commit(&bars.dkv_full);
-                umma_commit(&bars.kv_empty);
+                if (leader) umma_commit(&bars.dkv_full);
+                if (leader) umma_commit(&bars.kv_empty);
             }
         }
         __syncwarp();
@@ -317,8 +350,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const float4* dl4 = reinterpret_cast<const float4*>(stat + kBT + g * 64);
                 ok = mbar_wait(&bars.stat_full[st], (it_cnt >> 1) & 1, &abort_flag);
                 if (!ok) break;
+                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, it_cnt * 8 + 0);
                 ok = mbar_wait(&bars.s_full, it_cnt & 1, &abort_flag);
                 if (!ok) break;
+                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, it_cnt * 8 + 1);
                 tc_fence_after();
                 float pr[64];
 #pragma unroll
@@ -329,7 +364,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     uint32_t pk[16];
 #pragma unroll
                     for (int c4 = 0; c4 < 8; ++c4) {
-                        const float4 l4 = lse4[h * 8 + c4];
+                        const float4 l4 = MPIPE_DBG(4) ? make_float4(1.f, 1.f, 1.f, 1.f) : lse4[h * 8 + c4];
                         const float p0 = ex2_approx(fmaf(__uint_as_float(sr[4 * c4 + 0]), p.scale_log2, -l4.x));
                         const float p1 = ex2_approx(fmaf(__uint_as_float(sr[4 * c4 + 1]), p.scale_log2, -l4.y));
                         const float p2 = ex2_approx(fmaf(__uint_as_float(sr[4 * c4 + 2]), p.scale_log2, -l4.z));
@@ -347,9 +382,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars.p_full);
+                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, it_cnt * 8 + 2);
 
                 ok = mbar_wait(&bars.dp_full, it_cnt & 1, &abort_flag);
                 if (!ok) break;
+                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, it_cnt * 8 + 3);
                 tc_fence_after();
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
@@ -359,7 +396,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     uint32_t pk[16];
 #pragma unroll
                     for (int c4 = 0; c4 < 8; ++c4) {
-                        const float4 d4 = dl4[h * 8 + c4];
+                        const float4 d4 = MPIPE_DBG(4) ? make_float4(1.f, 1.f, 1.f, 1.f) : dl4[h * 8 + c4];
                         float s0 = pr[h * 32 + 4 * c4 + 0] * (__uint_as_float(dr[4 * c4 + 0]) - d4.x);
                         float s1 = pr[h * 32 + 4 * c4 + 1] * (__uint_as_float(dr[4 * c4 + 1]) - d4.y);
                         float s2 = pr[h * 32 + 4 * c4 + 2] * (__uint_as_float(dr[4 * c4 + 2]) - d4.z);
@@ -373,7 +410,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         const int chunk = h * 4 + c;
-                        *reinterpret_cast<uint4*>(ds_row + ((chunk ^ (r & 7)) << 4)) =
+                        if (!MPIPE_DBG(2)) *reinterpret_cast<uint4*>(ds_row + ((chunk ^ (r & 7)) << 4)) =
                             make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
                     }
                 }
@@ -385,6 +422,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     mbar_arrive(&bars.ds_full);
                     mbar_arrive(&bars.stat_empty[st]);
                 }
+                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, it_cnt * 8 + 4);
             }
         }
     } else {
@@ -400,8 +438,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const int nq = (it.kv_len + kBT - 1) / kBT;
             const int q_end = it.kv_start + it.kv_len;
             for (int i = 0; i < nq; ++i, ++it_cnt) {
+                if (lane == 0 && warp == 12) MPIPE_TR(3, it_cnt * 8 + 0);
                 ok = mbar_wait(&bars.dq_full, it_cnt & 1, &abort_flag);
                 if (!ok) break;
+                if (lane == 0 && warp == 12) MPIPE_TR(3, it_cnt * 8 + 1);
                 tc_fence_after();
                 const int q = it.kv_start + i * kBT + r;
                 float* dst = p.dq_acc + (int64_t(q) * p.n_heads + head) * D;
@@ -415,13 +455,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&bars.dq_empty);
                     }
-                    if (q < q_end) {
+                    if (q < q_end && !MPIPE_DBG(1)) {
 #pragma unroll
                         for (int c = 0; c < 16; c += 4)
                             red_add_v4(dst + c0 + c, __uint_as_float(v[c]), __uint_as_float(v[c + 1]),
                                        __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
                     }
                 }
+                if (lane == 0 && warp == 12) MPIPE_TR(3, it_cnt * 8 + 2);
             }
             if (!ok) break;
             ok = mbar_wait(&bars.dkv_full, unit_it & 1, &abort_flag);
@@ -560,6 +601,15 @@ static size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 }  // namespace mpipe
 
 extern "C" {
+
+#ifdef MPIPE_TRACE
+int32_t mpipe_dbg_set_flags(int32_t flags) {
+    return cudaMemcpyToSymbol(mpipe::g_dbg_flags, &flags, sizeof(int)) == cudaSuccess ? 0 : 1;
+}
+int32_t mpipe_dbg_read_trace(long long* host_out) {
+    return cudaMemcpyFromSymbol(host_out, mpipe::g_trace, sizeof(long long) * 4 * 4096) == cudaSuccess ? 0 : 1;
+}
+#endif
 
 int32_t mpipe_bwd_tile_rows(void) { return mpipe::kBT; }
 

@@ -152,34 +152,48 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ tcgen05 issuer
+        // The whole warp walks the loop (uniform control flow, uniform descriptors); one elected lane
+        // issues the MMAs and commits.  Descriptors are precomputed: a K-step only bumps the low word.
         setmaxnreg_dec<56>();
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             const uint32_t sbase = smem_u32(smem);
+            constexpr uint32_t hi128 = umma_desc_hi(1024, kSwizzle128);
+            constexpr uint32_t hi32 = umma_desc_hi(256, kSwizzle32);
             uint32_t kv_it = 0, unit_it = 0, cnt[2] = {0, 0};
             bool ok = true;
             // S_w = Q_w K^T for the KV tile in stage s; n_cols = keys to cover (multiple of 16)
             auto issue_s = [&](int w, int s, int n_cols) {
                 const uint32_t qa = sbase + Cfg::kSmemQ + w * Cfg::kQBytes;
                 const uint32_t ka = sbase + Cfg::kSmemK + s * Cfg::kQBytes;
+                const uint32_t qlo = umma_desc_lo(qa, 0), klo = umma_desc_lo(ka, 0);
                 const uint32_t idesc = umma_idesc_bf16(kTileM, n_cols, 0, 0);
                 const uint32_t d = tmem + w * 128;
+                if (leader) {
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_ss(d, umma_smem_desc(qa + ks * 32, 0, 1024, kSwizzle128),
-                            umma_smem_desc(ka + ks * 32, 0, 1024, kSwizzle128), idesc, ks > 0);
-                if (Cfg::kTail)
-                    umma_ss(d, umma_smem_desc(qa + Cfg::kQBytesMain, 0, 256, kSwizzle32),
-                            umma_smem_desc(ka + Cfg::kQBytesMain, 0, 256, kSwizzle32), idesc, 1);
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_ss(d, umma_desc(qlo + ks * 2, hi128), umma_desc(klo + ks * 2, hi128), idesc, ks > 0);
+                    if (Cfg::kTail)
+                        umma_ss(d, umma_desc(umma_desc_lo(qa + Cfg::kQBytesMain, 0), hi32),
+                                umma_desc(umma_desc_lo(ka + Cfg::kQBytesMain, 0), hi32), idesc, 1);
+                }
             };
             // O_w (+)= P_w V for the KV tile in stage s; n_keys = keys to cover (multiple of 16)
             auto issue_pv = [&](int w, int s, int n_keys, bool accumulate) {
-                const uint32_t va = sbase + Cfg::kSmemV + s * Cfg::kVBytes;
-                const uint32_t idesc = umma_idesc_bf16(kTileM, D, 0, 1);
+                const uint32_t vlo = umma_desc_lo(sbase + Cfg::kSmemV + s * Cfg::kVBytes, kTileN * 128);
+                constexpr uint32_t idesc = umma_idesc_bf16(kTileM, D, 0, 1);
                 const uint32_t d = tmem + 256 + w * 128;
                 const uint32_t pa = tmem + w * 128;
-                for (int ks = 0; ks < n_keys / 16; ++ks)
-                    umma_ts(d, pa + ks * 8, umma_smem_desc(va + ks * 2048, kTileN * 128, 1024, kSwizzle128), idesc,
-                            (accumulate || ks > 0) ? 1u : 0u);
+                if (leader) {
+                    if (n_keys == kTileN) {
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks)
+                            umma_ts(d, pa + ks * 8, umma_desc(vlo + ks * 128, hi128), idesc, (accumulate || ks > 0) ? 1u : 0u);
+                    } else {
+                        for (int ks = 0; ks < n_keys / 16; ++ks)
+                            umma_ts(d, pa + ks * 8, umma_desc(vlo + ks * 128, hi128), idesc, (accumulate || ks > 0) ? 1u : 0u);
+                    }
+                }
             };
             for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
                 const mpipe_work_item_t it = p.items[u / p.n_heads];
@@ -197,13 +211,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     if (!ok) break;
                     tc_fence_after();
                     issue_s(0, s, cols_of(0));
-                    umma_commit(&bars.s_full[0]);
+                    if (leader) umma_commit(&bars.s_full[0]);
                     if (two) {
                         issue_s(1, s, cols_of(0));
-                        umma_commit(&bars.s_full[1]);
+                        if (leader) umma_commit(&bars.s_full[1]);
                     }
-                    umma_commit(&bars.k_empty[s]);
-                    if (nkv == 1) umma_commit(&bars.q_empty);
+                    if (leader) umma_commit(&bars.k_empty[s]);
+                    if (nkv == 1) if (leader) umma_commit(&bars.q_empty);
                 }
                 for (int j = 0; j < nkv; ++j) {
                     const uint32_t itv = kv_it + j;
@@ -221,9 +235,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         if (!ok) break;
                         tc_fence_after();
                         issue_s(0, sk, cols_of(j + 1));
-                        umma_commit(&bars.s_full[0]);
+                        if (leader) umma_commit(&bars.s_full[0]);
                     } else {
-                        umma_commit(&bars.o_full[0]);
+                        if (leader) umma_commit(&bars.o_full[0]);
                     }
                     if (two) {
                         ok = mbar_wait(&bars.p_full[1], (cnt[1] + j) & 1, &abort_flag);
@@ -232,15 +246,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         issue_pv(1, sv, cols_of(j), j > 0);
                         if (more) {
                             issue_s(1, sk, cols_of(j + 1));
-                            umma_commit(&bars.s_full[1]);
+                            if (leader) umma_commit(&bars.s_full[1]);
                         } else {
-                            umma_commit(&bars.o_full[1]);
+                            if (leader) umma_commit(&bars.o_full[1]);
                         }
                     }
-                    umma_commit(&bars.v_empty[sv]);
+                    if (leader) umma_commit(&bars.v_empty[sv]);
                     if (more) {
-                        umma_commit(&bars.k_empty[sk]);
-                        if (j + 2 == nkv) umma_commit(&bars.q_empty);
+                        if (leader) umma_commit(&bars.k_empty[sk]);
+                        if (j + 2 == nkv) if (leader) umma_commit(&bars.q_empty);
                     }
                 }
                 kv_it += nkv;
@@ -285,9 +299,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     for (int c = 0; c < 128; ++c)
                         if (c >= n_valid) sr[c] = 0xFF800000u;  // -inf
                 }
-                float mx = __uint_as_float(sr[0]);
+                // eight independent running maxima (a single chain of 127 dependent max ops would cost
+                // ~4 cycles each with only two softmax warps per scheduler to hide it)
+                float mx8[8];
 #pragma unroll
-                for (int c = 1; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
+                for (int e = 0; e < 8; ++e) mx8[e] = __uint_as_float(sr[e]);
+#pragma unroll
+                for (int c = 8; c < 128; c += 8) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) mx8[e] = fmaxf(mx8[e], __uint_as_float(sr[c + e]));
+                }
+                const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                                       fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
                 const float m_tile = mx * p.scale_log2;
                 const bool grow = m_tile > m_ref + kRescaleThreshold;  // always true on the first tile
                 const float m_new = grow ? m_tile : m_ref;
@@ -306,21 +329,25 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         tmem_st16(t_o + c0, orr);
                     }
                 }
-                float sum = 0.f;
-                const float neg_m = -m_ref;
+                // p = exp2(s * scale*log2e - m_ref): packed fp32 pairs for the multiply-add and the row sum,
+                // four independent partial sums
+                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+                const float2 nm2 = make_float2(-m_ref, -m_ref);
+                float2 acc[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
                 for (int c0 = 0; c0 < 128; c0 += 32) {
                     uint32_t pk[16];
 #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(sr[c0 + c]), p.scale_log2, neg_m));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(sr[c0 + c + 1]), p.scale_log2, neg_m));
-                        sum += p0 + p1;
-                        pk[c >> 1] = pack_bf16(p0, p1);
+                        const float2 x = fma2(make_float2(__uint_as_float(sr[c0 + c]), __uint_as_float(sr[c0 + c + 1])), sc2, nm2);
+                        const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                        acc[(c >> 1) & 3] = add2(acc[(c >> 1) & 3], e);
+                        pk[c >> 1] = pack_bf16(e.x, e.y);
                     }
                     tmem_st16(t_s + (c0 >> 1), pk);
                 }
-                l = l * alpha + sum;
+                const float2 s01 = add2(add2(acc[0], acc[1]), add2(acc[2], acc[3]));
+                l = l * alpha + (s01.x + s01.y);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
