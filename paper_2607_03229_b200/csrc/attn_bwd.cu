@@ -47,25 +47,34 @@ __device__ int g_dbg_flags;   // knock-out switches for experiments: 1 no atomic
 #endif
 
 constexpr int kBwdThreads = 512;
-constexpr int kBT = 128;  // keys per unit = query rows per iteration = TMEM lanes
+constexpr int kBT = 128;  // keys per unit = TMEM lanes
+constexpr int kQS = 64;   // query rows per sub-tile (one pipeline stage of S^T / dP^T)
 
 template <int D>
 struct BwdCfg {
     static constexpr int kTail = D - 64;
-    static constexpr int kTileMain = kBT * 128;                 // [128 rows][64 bf16], 128-byte swizzle
-    static constexpr int kTileTail = kTail ? kBT * 32 : 0;      // [128 rows][16 bf16], 32-byte swizzle
+    static constexpr int kTileMain = kBT * 128;                 // K, V: [128 rows][64 bf16], 128-byte swizzle
+    static constexpr int kTileTail = kTail ? kBT * 32 : 0;      //       [128 rows][16 bf16], 32-byte swizzle
     static constexpr int kTile = kTileMain + kTileTail;
-    static constexpr int kStages = 2;
+    static constexpr int kSubMain = kQS * 128;                  // Q, dO sub-tiles: [64 rows][64 bf16]
+    static constexpr int kSubTail = kTail ? kQS * 32 : 0;
+    static constexpr int kSub = kSubMain + kSubTail;
+    static constexpr int kRing = 4;                             // Q/dO sub-tile stages
+    static constexpr int kStageBytes = kBT * (D * 4);           // dQ staging for the TMA reduction: [128 q][D fp32]
+    static constexpr int kStageBufs = (D == 64) ? 2 : 1;        // what fits next to the rest
     static constexpr int kSmemK = 0;
     static constexpr int kSmemV = kTile;
-    static constexpr int kSmemQ = 2 * kTile;                    // kStages tiles
-    static constexpr int kSmemDO = kSmemQ + kStages * kTile;    // kStages tiles
-    static constexpr int kSmemDS = kSmemDO + kStages * kTile;   // [key][q] as two 64-wide atoms: 32 KB
-    static constexpr int kSmemStat = kSmemDS + 2 * kBT * 128;   // kStages x (LSE[128], Delta[128]) fp32
-    static constexpr int kSmemTotal = kSmemStat + kStages * 2 * kBT * 4;
+    static constexpr int kSmemQ = 2 * kTile;
+    static constexpr int kSmemDO = kSmemQ + kRing * kSub;
+    static constexpr int kSmemDS = kSmemDO + kRing * kSub;      // dS^T as [key][q]: two 64-query atoms of 16 KB
+    static constexpr int kSmemStage = kSmemDS + 2 * kBT * 128;  // two staging buffers
+    static constexpr int kSmemStat = kSmemStage + kStageBufs * kStageBytes;   // kRing x (LSE[64], Delta[64]) fp32
+    static constexpr int kSmemTotal = kSmemStat + kRing * 2 * kQS * 4;
     static constexpr int kSmemAlloc = kSmemTotal + 1024;
-    // TMEM columns
+    // TMEM columns: S^T stage b at 64*b, dP^T stage b at 128 + 64*b (P^T / dS^T overlay their first 32 columns)
     static constexpr int kColS = 0, kColDP = 128, kColDV = 256, kColDK = 256 + D, kColDQ = 256 + 2 * D;
+    static_assert(kSmemAlloc <= 227 * 1024, "shared memory budget");
+    static_assert(kColDQ + D <= 512, "TMEM budget");
 };
 
 struct BwdParams {
@@ -73,7 +82,6 @@ struct BwdParams {
     int32_t n_items, n_heads, total_tokens;
     const float* lse;    // [H, T]
     const float* delta;  // [H, T]
-    float* dq_acc;       // [T, H, D] fp32
     __nv_bfloat16 *dk, *dv;
     int64_t tok_stride_g, head_stride_g;
     float scale, scale_log2;
@@ -82,22 +90,19 @@ struct BwdParams {
 
 struct BwdBarriers {
     uint64_t kv_full, kv_empty, dkv_full, dkv_empty;
-    uint64_t qdo_full[2], qdo_empty[2], stat_full[2], stat_empty[2];
-    uint64_t s_full, p_full, dp_full, ds_full, dq_full, dq_empty;
+    uint64_t qdo_full[4], qdo_empty[4], stat_full[4], stat_empty[4];
+    uint64_t s_full[2], p_full[2], dp_full[2], ds_full[2], dq_full, dq_empty;
 };
 
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
+struct BwdMaps {
+    CUtensorMap q, k, v, dout, q_tail, k_tail, v_tail, dout_tail, dq_acc, dq_acc_tail;
+};
 
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
-attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
-                const __grid_constant__ CUtensorMap map_q_tail, const __grid_constant__ CUtensorMap map_k_tail,
-                const __grid_constant__ CUtensorMap map_v_tail, const __grid_constant__ CUtensorMap map_do_tail,
-                const BwdParams p) {
+attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
     using Cfg = BwdCfg<D>;
+    constexpr int NR = Cfg::kRing;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ BwdBarriers bars;
@@ -114,16 +119,18 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         mbar_init(&bars.kv_empty, 1);
         mbar_init(&bars.dkv_full, 1);
         mbar_init(&bars.dkv_empty, 4);
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < 4; ++s) {
             mbar_init(&bars.qdo_full[s], 1);
             mbar_init(&bars.qdo_empty[s], 1);
             mbar_init(&bars.stat_full[s], 2);
-            mbar_init(&bars.stat_empty[s], 8);
+            mbar_init(&bars.stat_empty[s], 4);
         }
-        mbar_init(&bars.s_full, 1);
-        mbar_init(&bars.p_full, 8);
-        mbar_init(&bars.dp_full, 1);
-        mbar_init(&bars.ds_full, 8);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&bars.s_full[b], 1);
+            mbar_init(&bars.p_full[b], 4);
+            mbar_init(&bars.dp_full[b], 1);
+            mbar_init(&bars.ds_full[b], 4);
+        }
         mbar_init(&bars.dq_full, 1);
         mbar_init(&bars.dq_empty, 4);
         fence_mbar_init();
@@ -137,39 +144,42 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
     const int n_units = p.n_items * p.n_heads;
+    // Every unit runs an even number of 64-query sub-tiles (a 128-query tile is two of them); a padding
+    // sub-tile past the segment end contributes nothing because its probabilities are forced to zero.
+    auto subtiles_of = [](const mpipe_work_item_t& it) { return 2 * ((it.kv_len + kBT - 1) / kBT); };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         setmaxnreg_dec<72>();
         if (lane == 0) {
-            uint32_t unit_it = 0, it_cnt = 0;
+            uint32_t unit_it = 0, sc = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
                 const mpipe_work_item_t it = p.items[u / p.n_heads];
                 const int head = u % p.n_heads;
-                const int nq = (it.kv_len + kBT - 1) / kBT;
+                const int n2 = subtiles_of(it);
                 ok = mbar_wait(&bars.kv_empty, (unit_it & 1) ^ 1, &abort_flag);
                 if (!ok) break;
                 mbar_expect_tx(&bars.kv_full, 2 * Cfg::kTile);
-                tma_load_3d(smem + Cfg::kSmemK, &map_k, &bars.kv_full, 0, head, it.row_start);
-                tma_load_3d(smem + Cfg::kSmemV, &map_v, &bars.kv_full, 0, head, it.row_start);
+                tma_load_3d(smem + Cfg::kSmemK, &maps.k, &bars.kv_full, 0, head, it.row_start);
+                tma_load_3d(smem + Cfg::kSmemV, &maps.v, &bars.kv_full, 0, head, it.row_start);
                 if (Cfg::kTail) {
-                    tma_load_3d(smem + Cfg::kSmemK + Cfg::kTileMain, &map_k_tail, &bars.kv_full, 64, head, it.row_start);
-                    tma_load_3d(smem + Cfg::kSmemV + Cfg::kTileMain, &map_v_tail, &bars.kv_full, 64, head, it.row_start);
+                    tma_load_3d(smem + Cfg::kSmemK + Cfg::kTileMain, &maps.k_tail, &bars.kv_full, 64, head, it.row_start);
+                    tma_load_3d(smem + Cfg::kSmemV + Cfg::kTileMain, &maps.v_tail, &bars.kv_full, 64, head, it.row_start);
                 }
-                for (int i = 0; i < nq; ++i, ++it_cnt) {
-                    const int st = it_cnt & 1;
-                    const int row = it.kv_start + i * kBT;
-                    ok = mbar_wait(&bars.qdo_empty[st], ((it_cnt >> 1) & 1) ^ 1, &abort_flag);
+                for (int s = 0; s < n2; ++s, ++sc) {
+                    const int rs = sc % NR;
+                    const int row = it.kv_start + s * kQS;
+                    ok = mbar_wait(&bars.qdo_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
                     if (!ok) break;
-                    mbar_expect_tx(&bars.qdo_full[st], 2 * Cfg::kTile);
-                    uint8_t* qd = smem + Cfg::kSmemQ + st * Cfg::kTile;
-                    uint8_t* dd = smem + Cfg::kSmemDO + st * Cfg::kTile;
-                    tma_load_3d(qd, &map_q, &bars.qdo_full[st], 0, head, row);
-                    tma_load_3d(dd, &map_do, &bars.qdo_full[st], 0, head, row);
+                    mbar_expect_tx(&bars.qdo_full[rs], 2 * Cfg::kSub);
+                    uint8_t* qd = smem + Cfg::kSmemQ + rs * Cfg::kSub;
+                    uint8_t* dd = smem + Cfg::kSmemDO + rs * Cfg::kSub;
+                    tma_load_3d(qd, &maps.q, &bars.qdo_full[rs], 0, head, row);
+                    tma_load_3d(dd, &maps.dout, &bars.qdo_full[rs], 0, head, row);
                     if (Cfg::kTail) {
-                        tma_load_3d(qd + Cfg::kTileMain, &map_q_tail, &bars.qdo_full[st], 64, head, row);
-                        tma_load_3d(dd + Cfg::kTileMain, &map_do_tail, &bars.qdo_full[st], 64, head, row);
+                        tma_load_3d(qd + Cfg::kSubMain, &maps.q_tail, &bars.qdo_full[rs], 64, head, row);
+                        tma_load_3d(dd + Cfg::kSubMain, &maps.dout_tail, &bars.qdo_full[rs], 64, head, row);
                     }
                 }
             }
@@ -189,103 +199,102 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const uint32_t kt_lo = umma_desc_lo(sbase + Cfg::kSmemK + Cfg::kTileMain, 0);
             const uint32_t vt_lo = umma_desc_lo(sbase + Cfg::kSmemV + Cfg::kTileMain, 0);
             const uint32_t ds_lo = umma_desc_lo(sbase + Cfg::kSmemDS, kBT * 128);   // two 64-query atoms 16 KB apart
-            constexpr uint32_t idesc_s = umma_idesc_bf16(kBT, kBT, 0, 0);      // K-major x K-major, N = 128 queries
+            constexpr uint32_t idesc_s = umma_idesc_bf16(kBT, kQS, 0, 0);      // K-major x K-major, N = 64 queries
             constexpr uint32_t idesc_ts = umma_idesc_bf16(kBT, 64, 0, 1);      // A in TMEM, MN-major B, N = 64
             constexpr uint32_t idesc_ts_t = umma_idesc_bf16(kBT, 16, 0, 1);    // same, 16-wide head-dim tail
             constexpr uint32_t idesc_dq = umma_idesc_bf16(kBT, 64, 1, 1);      // MN-major A and B
             constexpr uint32_t idesc_dq_t = umma_idesc_bf16(kBT, 16, 1, 1);
-            // dst[128 x 128] = A[128 x D] * B[128 x D]^T, both K-major tiles (main 64 + optional 16 tail);
-            // a / b are the low descriptor words of the main tiles, at / bt of the tails
-            auto issue_kk = [&](uint32_t dcol, uint32_t a, uint32_t at, uint32_t b, uint32_t bt) {
+            constexpr uint32_t kSubTailOff = Cfg::kSubMain >> 4;
+            auto q_lo_of = [&](uint32_t c) { return umma_desc_lo(sbase + Cfg::kSmemQ + (c % NR) * Cfg::kSub, 0); };
+            auto do_lo_of = [&](uint32_t c) { return umma_desc_lo(sbase + Cfg::kSmemDO + (c % NR) * Cfg::kSub, 0); };
+            // dst[128 keys x 64 q] = A[128 x D] * B[64 x D]^T, both K-major (main 64 columns + optional 16 tail)
+            auto issue_kk = [&](uint32_t dcol, uint32_t a, uint32_t at, uint32_t b) {
                 if (leader) {
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
                         umma_ss(tmem + dcol, umma_desc(a + ks * 2, hi128), umma_desc(b + ks * 2, hi128), idesc_s, ks > 0);
-                    if (Cfg::kTail) umma_ss(tmem + dcol, umma_desc(at, hi32), umma_desc(bt, hi32), idesc_s, 1);
+                    if (Cfg::kTail) umma_ss(tmem + dcol, umma_desc(at, hi32), umma_desc(b + kSubTailOff, hi32), idesc_s, 1);
                 }
             };
-            // dst[128 keys x D] (+)= A^T-in-TMEM[128 keys x 128 q] * B[128 q x D] (B tile rows = q, MN-major)
-            auto issue_ts = [&](uint32_t dcol, uint32_t acol, uint32_t b, uint32_t bt, bool acc) {
+            // dst[128 keys x D] (+)= A^T-in-TMEM[128 keys x 64 q] * B[64 q x D] (B rows = q, MN-major)
+            auto issue_ts = [&](uint32_t dcol, uint32_t acol, uint32_t b, bool acc) {
                 if (leader) {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t a_t = tmem + acol + (ks < 4 ? ks * 8 : 64 + (ks - 4) * 8);
-                        umma_ts(tmem + dcol, a_t, umma_desc(b + ks * 128, hi128), idesc_ts, (acc || ks > 0) ? 1u : 0u);
+                    for (int ks = 0; ks < 4; ++ks) {
+                        umma_ts(tmem + dcol, tmem + acol + ks * 8, umma_desc(b + ks * 128, hi128), idesc_ts,
+                                (acc || ks > 0) ? 1u : 0u);
                         if (Cfg::kTail)
-                            umma_ts(tmem + dcol + 64, a_t, umma_desc(bt + ks * 32, hi32), idesc_ts_t,
-                                    (acc || ks > 0) ? 1u : 0u);
+                            umma_ts(tmem + dcol + 64, tmem + acol + ks * 8, umma_desc(b + kSubTailOff + ks * 32, hi32),
+                                    idesc_ts_t, (acc || ks > 0) ? 1u : 0u);
                     }
                 }
             };
-            uint32_t unit_it = 0, it_cnt = 0;
+            uint32_t unit_it = 0, sc = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
                 const mpipe_work_item_t it = p.items[u / p.n_heads];
-                const int nq = (it.kv_len + kBT - 1) / kBT;
+                const int n2 = subtiles_of(it);
                 ok = mbar_wait(&bars.kv_full, unit_it & 1, &abort_flag);
                 if (!ok) break;
-                ok = mbar_wait(&bars.qdo_full[it_cnt & 1], (it_cnt >> 1) & 1, &abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                {
-                    const uint32_t qa = sbase + Cfg::kSmemQ + (it_cnt & 1) * Cfg::kTile;
-                    const uint32_t da = sbase + Cfg::kSmemDO + (it_cnt & 1) * Cfg::kTile;
-                    issue_kk(Cfg::kColS, k_lo, kt_lo, umma_desc_lo(qa, 0), umma_desc_lo(qa + Cfg::kTileMain, 0));
-                    if (leader) umma_commit(&bars.s_full);
-                    issue_kk(Cfg::kColDP, v_lo, vt_lo, umma_desc_lo(da, 0), umma_desc_lo(da + Cfg::kTileMain, 0));
-                    if (leader) umma_commit(&bars.dp_full);
+                for (int s = 0; s < 2; ++s) {   // prologue: S^T and dP^T of the first two sub-tiles
+                    ok = mbar_wait(&bars.qdo_full[(sc + s) % NR], ((sc + s) / NR) & 1, &abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_kk(Cfg::kColS + 64 * s, k_lo, kt_lo, q_lo_of(sc + s));
+                    if (leader) umma_commit(&bars.s_full[s]);
+                    issue_kk(Cfg::kColDP + 64 * s, v_lo, vt_lo, do_lo_of(sc + s));
+                    if (leader) umma_commit(&bars.dp_full[s]);
                 }
-                for (int i = 0; i < nq; ++i, ++it_cnt) {
-                    const int st = it_cnt & 1;
-                    const uint32_t q_lo = umma_desc_lo(sbase + Cfg::kSmemQ + st * Cfg::kTile, 0);
-                    const uint32_t d_lo = umma_desc_lo(sbase + Cfg::kSmemDO + st * Cfg::kTile, 0);
-                    const uint32_t qn_lo = umma_desc_lo(sbase + Cfg::kSmemQ + (st ^ 1) * Cfg::kTile, 0);
-                    const uint32_t dn_lo = umma_desc_lo(sbase + Cfg::kSmemDO + (st ^ 1) * Cfg::kTile, 0);
-                    constexpr uint32_t kTailOff = Cfg::kTileMain >> 4;
-                    const bool more = (i + 1 < nq);
-                    if (i == 0) {
+                if (!ok) break;
+                for (int s = 0; s < n2; ++s, ++sc) {
+                    const int b = s & 1;
+                    const uint32_t ph = (sc >> 1) & 1;   // phase of the per-stage barriers
+                    const bool more = (s + 2 < n2);
+                    if (s == 0) {
                         ok = mbar_wait(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag);
                         if (!ok) break;
                     }
-                    MPIPE_TR(0, it_cnt * 8 + 0);
-                    ok = mbar_wait(&bars.p_full, it_cnt & 1, &abort_flag);
+                    MPIPE_TR(0, sc * 8 + 0);
+                    ok = mbar_wait(&bars.p_full[b], ph, &abort_flag);
                     if (!ok) break;
-                    MPIPE_TR(0, it_cnt * 8 + 1);
+                    MPIPE_TR(0, sc * 8 + 1);
                     tc_fence_after();
-                    issue_ts(Cfg::kColDV, Cfg::kColS, d_lo, d_lo + kTailOff, i > 0);                 // dV += P^T dO
+                    issue_ts(Cfg::kColDV, Cfg::kColS + 64 * b, do_lo_of(sc), s > 0);          // dV += P^T dO
                     if (more) {
-                        ok = mbar_wait(&bars.qdo_full[st ^ 1], ((it_cnt + 1) >> 1) & 1, &abort_flag);
+                        ok = mbar_wait(&bars.qdo_full[(sc + 2) % NR], ((sc + 2) / NR) & 1, &abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        issue_kk(Cfg::kColS, k_lo, kt_lo, qn_lo, qn_lo + kTailOff);                          // S^T(i+1)
-                        if (leader) umma_commit(&bars.s_full);
+                        issue_kk(Cfg::kColS + 64 * b, k_lo, kt_lo, q_lo_of(sc + 2));          // S^T(s+2)
+                        if (leader) umma_commit(&bars.s_full[b]);
                     }
-                    MPIPE_TR(0, it_cnt * 8 + 2);
-                    ok = mbar_wait(&bars.ds_full, it_cnt & 1, &abort_flag);
+                    MPIPE_TR(0, sc * 8 + 2);
+                    ok = mbar_wait(&bars.ds_full[b], ph, &abort_flag);
                     if (!ok) break;
-                    MPIPE_TR(0, it_cnt * 8 + 3);
+                    MPIPE_TR(0, sc * 8 + 3);
                     tc_fence_after();
-                    issue_ts(Cfg::kColDK, Cfg::kColDP, q_lo, q_lo + kTailOff, i > 0);                // dK += dS^T Q
-                    ok = mbar_wait(&bars.dq_empty, (it_cnt & 1) ^ 1, &abort_flag);
-                    if (!ok) break;
-                    MPIPE_TR(0, it_cnt * 8 + 4);
-                    tc_fence_after();
-                    if (leader) {
+                    issue_ts(Cfg::kColDK, Cfg::kColDP + 64 * b, q_lo_of(sc), s > 0);          // dK += dS^T Q
+                    if (leader) umma_commit(&bars.qdo_empty[sc % NR]);
+                    if (more) {
+                        issue_kk(Cfg::kColDP + 64 * b, v_lo, vt_lo, do_lo_of(sc + 2));        // dP^T(s+2)
+                        if (leader) umma_commit(&bars.dp_full[b]);
+                    }
+                    if (b == 1) {                                                             // dQ of the 128-query pair
+                        ok = mbar_wait(&bars.dq_empty, ((sc >> 1) & 1) ^ 1, &abort_flag);
+                        if (!ok) break;
+                        MPIPE_TR(0, sc * 8 + 4);
+                        tc_fence_after();
+                        if (leader) {
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks) {                          // dQ_i = dS K
-                            const uint64_t adesc = umma_desc(ds_lo + ks * 128, hi128);
-                            umma_ss(tmem + Cfg::kColDQ, adesc, umma_desc(k_lo + ks * 128, hi128), idesc_dq, ks > 0);
-                            if (Cfg::kTail)
-                                umma_ss(tmem + Cfg::kColDQ + 64, adesc, umma_desc(kt_lo + ks * 32, hi32), idesc_dq_t, ks > 0);
+                            for (int ks = 0; ks < 8; ++ks) {
+                                const uint64_t adesc = umma_desc(ds_lo + ks * 128, hi128);
+                                umma_ss(tmem + Cfg::kColDQ, adesc, umma_desc(k_lo + ks * 128, hi128), idesc_dq, ks > 0);
+                                if (Cfg::kTail)
+                                    umma_ss(tmem + Cfg::kColDQ + 64, adesc, umma_desc(kt_lo + ks * 32, hi32), idesc_dq_t, ks > 0);
+                            }
+                            umma_commit(&bars.dq_full);
                         }
                     }
-                    if (leader) umma_commit(&bars.dq_full);
-                    if (leader) umma_commit(&bars.qdo_empty[st]);
-                    if (more) {
-                        issue_kk(Cfg::kColDP, v_lo, vt_lo, dn_lo, dn_lo + kTailOff);                         // dP^T(i+1)
-                        if (leader) umma_commit(&bars.dp_full);
-                    }
-                    MPIPE_TR(0, it_cnt * 8 + 5);
+                    MPIPE_TR(0, sc * 8 + 5);
                 }
                 if (!ok) break;
                 if (leader) umma_commit(&bars.dkv_full);
@@ -298,21 +307,21 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         setmaxnreg_dec<72>();
         const bool is_lse = (warp == 2);
         const float* src = is_lse ? p.lse : p.delta;
-        uint32_t it_cnt = 0;
+        uint32_t sc = 0;
         bool ok = true;
         for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
             const mpipe_work_item_t it = p.items[u / p.n_heads];
             const int head = u % p.n_heads;
-            const int nq = (it.kv_len + kBT - 1) / kBT;
+            const int n2 = subtiles_of(it);
             const int q_end = it.kv_start + it.kv_len;
-            for (int i = 0; i < nq; ++i, ++it_cnt) {
-                const int st = it_cnt & 1;
-                ok = mbar_wait(&bars.stat_empty[st], ((it_cnt >> 1) & 1) ^ 1, &abort_flag);
+            for (int s = 0; s < n2; ++s, ++sc) {
+                const int rs = sc % NR;
+                ok = mbar_wait(&bars.stat_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
                 if (!ok) break;
-                float* dst = reinterpret_cast<float*>(smem + Cfg::kSmemStat + st * (2 * kBT * 4)) + (is_lse ? 0 : kBT);
-                const int q0 = it.kv_start + i * kBT;
+                float* dst = reinterpret_cast<float*>(smem + Cfg::kSmemStat + rs * (2 * kQS * 4)) + (is_lse ? 0 : kQS);
+                const int q0 = it.kv_start + s * kQS;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
+                for (int e = 0; e < 2; ++e) {
                     const int c = lane + 32 * e;
                     const int q = q0 + c;
                     float val;
@@ -325,35 +334,38 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     dst[c] = val;
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bars.stat_full[st]);
+                if (lane == 0) mbar_arrive(&bars.stat_full[rs]);
             }
         }
     } else if (warp < 12) {
         // ------------------------------------------------------------------ softmax / dS warps
+        // Warpgroup g owns TMEM stage g, i.e. every other 64-query sub-tile; thread = key row.
         setmaxnreg_inc<168>();
-        const int g = (warp - 4) >> 2;                // query-column half handled by this warpgroup
-        const int r = ((warp & 3) << 5) | lane;       // key row inside the tile = TMEM lane
+        const int g = (warp - 4) >> 2;
+        const int r = ((warp & 3) << 5) | lane;
         const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
-        const uint32_t t_s = tmem + lane_base + Cfg::kColS + g * 64;    // S^T columns of this half; P^T goes to the first 32 of them
+        const uint32_t t_s = tmem + lane_base + Cfg::kColS + g * 64;
         const uint32_t t_dp = tmem + lane_base + Cfg::kColDP + g * 64;
         uint8_t* ds_row = smem + Cfg::kSmemDS + g * (kBT * 128) + r * 128;
-        uint32_t it_cnt = 0;
+        uint32_t sc = 0;   // global sub-tile counter at the start of the unit (always even)
         bool ok = true;
         for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
             const mpipe_work_item_t it = p.items[u / p.n_heads];
-            const int nq = (it.kv_len + kBT - 1) / kBT;
+            const int n2 = subtiles_of(it);
             const bool key_valid = r < it.row_len;
-            for (int i = 0; i < nq; ++i, ++it_cnt) {
-                const int st = it_cnt & 1;
-                const float* stat = reinterpret_cast<const float*>(smem + Cfg::kSmemStat + st * (2 * kBT * 4));
-                const float4* lse4 = reinterpret_cast<const float4*>(stat + g * 64);
-                const float4* dl4 = reinterpret_cast<const float4*>(stat + kBT + g * 64);
-                ok = mbar_wait(&bars.stat_full[st], (it_cnt >> 1) & 1, &abort_flag);
+            for (int s = g; s < n2; s += 2) {
+                const uint32_t c = sc + s;
+                const int rs = c % NR;
+                const uint32_t ph = (c >> 1) & 1;
+                const float* stat = reinterpret_cast<const float*>(smem + Cfg::kSmemStat + rs * (2 * kQS * 4));
+                const float4* lse4 = reinterpret_cast<const float4*>(stat);
+                const float4* dl4 = reinterpret_cast<const float4*>(stat + kQS);
+                ok = mbar_wait(&bars.stat_full[rs], (c / NR) & 1, &abort_flag);
                 if (!ok) break;
-                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, it_cnt * 8 + 0);
-                ok = mbar_wait(&bars.s_full, it_cnt & 1, &abort_flag);
+                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 0);
+                ok = mbar_wait(&bars.s_full[g], ph, &abort_flag);
                 if (!ok) break;
-                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, it_cnt * 8 + 1);
+                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 1);
                 tc_fence_after();
                 float pr[64];
 #pragma unroll
@@ -381,12 +393,17 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bars.p_full);
-                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, it_cnt * 8 + 2);
+                if (lane == 0) mbar_arrive(&bars.p_full[g]);
+                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 2);
 
-                ok = mbar_wait(&bars.dp_full, it_cnt & 1, &abort_flag);
+                ok = mbar_wait(&bars.dp_full[g], ph, &abort_flag);
                 if (!ok) break;
-                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, it_cnt * 8 + 3);
+                // the dS^T tile in shared memory is free once the previous pair's dQ MMA has completed
+                if ((c >> 1) > 0) {
+                    ok = mbar_wait(&bars.dq_full, ((c >> 1) - 1) & 1, &abort_flag);
+                    if (!ok) break;
+                }
+                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 3);
                 tc_fence_after();
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
@@ -408,10 +425,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     tmem_st16(t_dp + h * 16, pk);
                     // the same 32 values as 4 x 16 bytes of row r of the [key][q] tile (128-byte swizzle)
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const int chunk = h * 4 + c;
+                    for (int cc = 0; cc < 4; ++cc) {
+                        const int chunk = h * 4 + cc;
                         if (!MPIPE_DBG(2)) *reinterpret_cast<uint4*>(ds_row + ((chunk ^ (r & 7)) << 4)) =
-                            make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                            make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
                     }
                 }
                 tmem_wait_st();
@@ -419,54 +436,75 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(&bars.ds_full);
-                    mbar_arrive(&bars.stat_empty[st]);
+                    mbar_arrive(&bars.ds_full[g]);
+                    mbar_arrive(&bars.stat_empty[rs]);
                 }
-                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, it_cnt * 8 + 4);
+                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 4);
             }
+            sc += n2;
         }
     } else {
         // ------------------------------------------------------------------ dQ reducer + dK/dV epilogue
+        // dQ of a 128-query pair: TMEM -> registers -> swizzled staging in shared memory -> one TMA
+        // reduce-add per 32 fp32 columns into the global accumulator (the copy engine does the atomics).
         setmaxnreg_dec<96>();
         const int r = ((warp & 3) << 5) | lane;
+        const int rt = tid - 12 * 32;   // 0..127 inside the warpgroup
         const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
-        uint32_t it_cnt = 0, unit_it = 0;
+        uint32_t pc = 0, unit_it = 0;   // pair counter
         bool ok = true;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
+        for (int u = blockIdx.x; u < n_units; u += gridDim.x, ++unit_it) {
             const mpipe_work_item_t it = p.items[u / p.n_heads];
             const int head = u % p.n_heads;
-            const int nq = (it.kv_len + kBT - 1) / kBT;
-            const int q_end = it.kv_start + it.kv_len;
-            for (int i = 0; i < nq; ++i, ++it_cnt) {
-                if (lane == 0 && warp == 12) MPIPE_TR(3, it_cnt * 8 + 0);
-                ok = mbar_wait(&bars.dq_full, it_cnt & 1, &abort_flag);
-                if (!ok) break;
-                if (lane == 0 && warp == 12) MPIPE_TR(3, it_cnt * 8 + 1);
+            const int npairs = (it.kv_len + kBT - 1) / kBT;
+            // No early exit inside this loop: the four warps meet at named barriers, so after a time-out
+            // they keep walking the (now empty) iterations together instead of leaving one another behind.
+            for (int i = 0; i < npairs; ++i, ++pc) {
+                if (lane == 0 && warp == 12) MPIPE_TR(3, pc * 8 + 0);
+                if (ok) ok = mbar_wait(&bars.dq_full, pc & 1, &abort_flag);
+                if (lane == 0 && warp == 12) MPIPE_TR(3, pc * 8 + 1);
                 tc_fence_after();
-                const int q = it.kv_start + i * kBT + r;
-                float* dst = p.dq_acc + (int64_t(q) * p.n_heads + head) * D;
+                uint8_t* stage = smem + Cfg::kSmemStage + (pc % Cfg::kStageBufs) * Cfg::kStageBytes;
+                // the staging buffer must have been read by the copy engine before it is overwritten
+                if (rt == 0) bulk_wait_group_read<Cfg::kStageBufs - 1>();
+                named_barrier_sync(1, 128);
+                if (ok) {
 #pragma unroll
-                for (int c0 = 0; c0 < D; c0 += 16) {
-                    uint32_t v[16];
-                    tmem_ld16(tmem + lane_base + Cfg::kColDQ + c0, v);
-                    tmem_wait_ld();
-                    if (c0 + 16 >= D) {  // all reads of this row issued and complete: release dQ in TMEM
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&bars.dq_empty);
-                    }
-                    if (q < q_end && !MPIPE_DBG(1)) {
+                    for (int c0 = 0; c0 < D; c0 += 16) {
+                        uint32_t v[16];
+                        tmem_ld16(tmem + lane_base + Cfg::kColDQ + c0, v);
+                        tmem_wait_ld();
+                        if (c0 + 16 >= D) {  // last read of this row issued and complete: release dQ in TMEM
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&bars.dq_empty);
+                        }
+                        // box j = columns [32j, 32j+32): [128 rows][128 B], 128-byte swizzle; the D=80 tail box
+                        // (columns 64..79) is [128 rows][64 B] with 64-byte swizzle
+                        const int box = c0 >> 5;
+                        uint8_t* brow = stage + box * (kBT * 128);
 #pragma unroll
-                        for (int c = 0; c < 16; c += 4)
-                            red_add_v4(dst + c0 + c, __uint_as_float(v[c]), __uint_as_float(v[c + 1]),
-                                       __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
+                        for (int cc = 0; cc < 4; ++cc) {
+                            const int chunk = ((c0 & 31) >> 2) + cc;   // 16-byte chunk inside the box row
+                            uint8_t* dst = (box < 2) ? brow + r * 128 + ((chunk ^ (r & 7)) << 4)
+                                                     : brow + r * 64 + ((chunk ^ ((r >> 1) & 3)) << 4);
+                            *reinterpret_cast<uint4*>(dst) = make_uint4(v[4 * cc], v[4 * cc + 1], v[4 * cc + 2], v[4 * cc + 3]);
+                        }
                     }
                 }
-                if (lane == 0 && warp == 12) MPIPE_TR(3, it_cnt * 8 + 2);
+                fence_async_smem();
+                named_barrier_sync(1, 128);
+                if (ok && rt == 0 && !MPIPE_DBG(1)) {
+                    const int q0 = it.kv_start + i * kBT;
+                    tma_reduce_add_3d(&maps.dq_acc, stage, 0, head, q0);
+                    tma_reduce_add_3d(&maps.dq_acc, stage + kBT * 128, 32, head, q0);
+                    if (Cfg::kTail) tma_reduce_add_3d(&maps.dq_acc_tail, stage + 2 * kBT * 128, 64, head, q0);
+                    bulk_commit_group();
+                }
+                if (lane == 0 && warp == 12) MPIPE_TR(3, pc * 8 + 2);
             }
-            if (!ok) break;
-            ok = mbar_wait(&bars.dkv_full, unit_it & 1, &abort_flag);
-            if (!ok) break;
+            if (ok) ok = mbar_wait(&bars.dkv_full, unit_it & 1, &abort_flag);
+            if (!ok) continue;   // keep walking the units so that the named barriers above stay matched
             tc_fence_after();
             const bool store = r < it.row_len;
             const int64_t tok = int64_t(it.row_start) + r;
@@ -501,6 +539,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars.dkv_empty);
         }
+        if (rt == 0) bulk_wait_group<0>();   // all reductions have landed before the CTA exits
     }
 
     tc_fence_before();
@@ -561,20 +600,22 @@ bwd_dq_convert_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__
 template <int D>
 static int32_t launch_bwd(const void* dout, const void* q, const void* k, const void* v, const void* o, void* dq,
                           int64_t ts_qkv, int64_t hs_qkv, int64_t ts_o, int64_t hs_o, int32_t total_tokens,
-                          int32_t n_heads, BwdParams prm, float* delta, cudaStream_t stream) {
+                          int32_t n_heads, BwdParams prm, float* delta, float* dq_acc, cudaStream_t stream) {
     using Cfg = BwdCfg<D>;
-    CUtensorMap mq, mk, mv, mdo, mqt, mkt, mvt, mdot;
-    if (!make_tensor_map_thd(&mq, q, total_tokens, n_heads, D, ts_qkv, hs_qkv, 64, kBT, 128) ||
-        !make_tensor_map_thd(&mk, k, total_tokens, n_heads, D, ts_qkv, hs_qkv, 64, kBT, 128) ||
-        !make_tensor_map_thd(&mv, v, total_tokens, n_heads, D, ts_qkv, hs_qkv, 64, kBT, 128) ||
-        !make_tensor_map_thd(&mdo, dout, total_tokens, n_heads, D, ts_o, hs_o, 64, kBT, 128))
+    BwdMaps m;
+    if (!make_tensor_map_thd(&m.q, q, total_tokens, n_heads, D, ts_qkv, hs_qkv, 64, kQS, 128) ||
+        !make_tensor_map_thd(&m.k, k, total_tokens, n_heads, D, ts_qkv, hs_qkv, 64, kBT, 128) ||
+        !make_tensor_map_thd(&m.v, v, total_tokens, n_heads, D, ts_qkv, hs_qkv, 64, kBT, 128) ||
+        !make_tensor_map_thd(&m.dout, dout, total_tokens, n_heads, D, ts_o, hs_o, 64, kQS, 128) ||
+        !make_tensor_map_thd(&m.dq_acc, dq_acc, total_tokens, n_heads, D, int64_t(n_heads) * D, D, 32, kBT, 128, 4))
         return MPIPE_ERR_CUDA;
-    mqt = mq, mkt = mk, mvt = mv, mdot = mdo;
+    m.q_tail = m.q, m.k_tail = m.k, m.v_tail = m.v, m.dout_tail = m.dout, m.dq_acc_tail = m.dq_acc;
     if (Cfg::kTail) {
-        if (!make_tensor_map_thd(&mqt, q, total_tokens, n_heads, D, ts_qkv, hs_qkv, 16, kBT, 32) ||
-            !make_tensor_map_thd(&mkt, k, total_tokens, n_heads, D, ts_qkv, hs_qkv, 16, kBT, 32) ||
-            !make_tensor_map_thd(&mvt, v, total_tokens, n_heads, D, ts_qkv, hs_qkv, 16, kBT, 32) ||
-            !make_tensor_map_thd(&mdot, dout, total_tokens, n_heads, D, ts_o, hs_o, 16, kBT, 32))
+        if (!make_tensor_map_thd(&m.q_tail, q, total_tokens, n_heads, D, ts_qkv, hs_qkv, 16, kQS, 32) ||
+            !make_tensor_map_thd(&m.k_tail, k, total_tokens, n_heads, D, ts_qkv, hs_qkv, 16, kBT, 32) ||
+            !make_tensor_map_thd(&m.v_tail, v, total_tokens, n_heads, D, ts_qkv, hs_qkv, 16, kBT, 32) ||
+            !make_tensor_map_thd(&m.dout_tail, dout, total_tokens, n_heads, D, ts_o, hs_o, 16, kQS, 32) ||
+            !make_tensor_map_thd(&m.dq_acc_tail, dq_acc, total_tokens, n_heads, D, int64_t(n_heads) * D, D, 16, kBT, 64, 4))
             return MPIPE_ERR_CUDA;
     }
     if (cudaFuncSetAttribute(attn_bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemAlloc) !=
@@ -583,15 +624,15 @@ static int32_t launch_bwd(const void* dout, const void* q, const void* k, const 
     const int64_t rows = int64_t(total_tokens) * n_heads;
     bwd_prepass_kernel<D><<<unsigned((rows + 255) / 256), 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(dout), static_cast<const __nv_bfloat16*>(o), ts_o, hs_o, total_tokens, n_heads,
-        delta, prm.dq_acc);
+        delta, dq_acc);
     const int n_units = prm.n_items * prm.n_heads;
     const int grid = n_units < sm_count() ? n_units : sm_count();
     profile_start(kProfileBwdMain, stream);
-    attn_bwd_kernel<D><<<grid, kBwdThreads, Cfg::kSmemAlloc, stream>>>(mq, mk, mv, mdo, mqt, mkt, mvt, mdot, prm);
+    attn_bwd_kernel<D><<<grid, kBwdThreads, Cfg::kSmemAlloc, stream>>>(m, prm);
     profile_stop(kProfileBwdMain, stream);
     const int64_t chunks = rows * (D / 8);
     bwd_dq_convert_kernel<<<unsigned((chunks + 255) / 256), 256, 0, stream>>>(
-        prm.dq_acc, static_cast<__nv_bfloat16*>(dq), prm.tok_stride_g, prm.head_stride_g, total_tokens, n_heads, D,
+        dq_acc, static_cast<__nv_bfloat16*>(dq), prm.tok_stride_g, prm.head_stride_g, total_tokens, n_heads, D,
         prm.scale);
     return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
 }
@@ -661,7 +702,6 @@ int32_t mpipe_varlen_attn_bwd(const void* dout, const void* q, const void* k, co
     prm.total_tokens = total_tokens;
     prm.lse = lse;
     prm.delta = delta;
-    prm.dq_acc = dq_acc;
     prm.dk = static_cast<__nv_bfloat16*>(dk);
     prm.dv = static_cast<__nv_bfloat16*>(dv);
     prm.tok_stride_g = tok_stride_grad;
@@ -672,9 +712,9 @@ int32_t mpipe_varlen_attn_bwd(const void* dout, const void* q, const void* k, co
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (head_dim == 64)
         return launch_bwd<64>(dout, q, k, v, o, dq, tok_stride_qkv, head_stride_qkv, tok_stride_o, head_stride_o,
-                              total_tokens, n_heads, prm, delta, st);
+                              total_tokens, n_heads, prm, delta, dq_acc, st);
     return launch_bwd<80>(dout, q, k, v, o, dq, tok_stride_qkv, head_stride_qkv, tok_stride_o, head_stride_o,
-                          total_tokens, n_heads, prm, delta, st);
+                          total_tokens, n_heads, prm, delta, dq_acc, st);
 }
 
 

@@ -20,18 +20,19 @@ static EncodeTiledFn encode_fn() {
 }
 
 bool make_tensor_map_thd(CUtensorMap* out, const void* base, int64_t T, int64_t H, int64_t D, int64_t tok_stride,
-                         int64_t head_stride, uint32_t box_d, uint32_t box_rows, int swizzle_bytes) {
+                         int64_t head_stride, uint32_t box_d, uint32_t box_rows, int swizzle_bytes, int elem_bytes) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return false;
     const cuuint64_t dims[3] = {cuuint64_t(D), cuuint64_t(H), cuuint64_t(T)};
-    const cuuint64_t strides[2] = {cuuint64_t(head_stride) * 2, cuuint64_t(tok_stride) * 2};
+    const cuuint64_t strides[2] = {cuuint64_t(head_stride) * elem_bytes, cuuint64_t(tok_stride) * elem_bytes};
     const cuuint32_t box[3] = {box_d, 1, box_rows};
     const cuuint32_t elem_strides[3] = {1, 1, 1};
     const CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                   : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
                                   : swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
                                                         : CU_TENSOR_MAP_SWIZZLE_NONE;
-    const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+    const CUtensorMapDataType dt = elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const CUresult r = fn(out, dt, 3, const_cast<void*>(base), dims, strides, box,
                           elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
