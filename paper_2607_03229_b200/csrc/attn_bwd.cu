@@ -46,6 +46,12 @@ __device__ int g_dbg_flags;   // knock-out switches for experiments: 1 no atomic
     } while (0)
 #endif
 
+#ifndef MPIPE_SLEEP_AUX
+#define MPIPE_SLEEP_AUX 100
+#endif
+#ifndef MPIPE_SLEEP_MMA
+#define MPIPE_SLEEP_MMA 0
+#endif
 constexpr int kBwdThreads = 512;
 constexpr int kBT = 128;  // keys per unit = TMEM lanes
 constexpr int kQS = 64;   // query rows per sub-tile (one pipeline stage of S^T / dP^T)
@@ -158,7 +164,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 const mpipe_work_item_t it = p.items[u / p.n_heads];
                 const int head = u % p.n_heads;
                 const int n2 = subtiles_of(it);
-                ok = mbar_wait(&bars.kv_empty, (unit_it & 1) ^ 1, &abort_flag);
+                ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.kv_empty, (unit_it & 1) ^ 1, &abort_flag);
                 if (!ok) break;
                 mbar_expect_tx(&bars.kv_full, 2 * Cfg::kTile);
                 tma_load_3d(smem + Cfg::kSmemK, &maps.k, &bars.kv_full, 0, head, it.row_start);
@@ -170,7 +176,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 for (int s = 0; s < n2; ++s, ++sc) {
                     const int rs = sc % NR;
                     const int row = it.kv_start + s * kQS;
-                    ok = mbar_wait(&bars.qdo_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
+                    ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.qdo_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
                     if (!ok) break;
                     mbar_expect_tx(&bars.qdo_full[rs], 2 * Cfg::kSub);
                     uint8_t* qd = smem + Cfg::kSmemQ + rs * Cfg::kSub;
@@ -234,10 +240,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
                 const mpipe_work_item_t it = p.items[u / p.n_heads];
                 const int n2 = subtiles_of(it);
-                ok = mbar_wait(&bars.kv_full, unit_it & 1, &abort_flag);
+                ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.kv_full, unit_it & 1, &abort_flag);
                 if (!ok) break;
                 for (int s = 0; s < 2; ++s) {   // prologue: S^T and dP^T of the first two sub-tiles
-                    ok = mbar_wait(&bars.qdo_full[(sc + s) % NR], ((sc + s) / NR) & 1, &abort_flag);
+                    ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[(sc + s) % NR], ((sc + s) / NR) & 1, &abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     issue_kk(Cfg::kColS + 64 * s, k_lo, kt_lo, q_lo_of(sc + s));
@@ -251,24 +257,24 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     const uint32_t ph = (sc >> 1) & 1;   // phase of the per-stage barriers
                     const bool more = (s + 2 < n2);
                     if (s == 0) {
-                        ok = mbar_wait(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag);
+                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag);
                         if (!ok) break;
                     }
                     MPIPE_TR(0, sc * 8 + 0);
-                    ok = mbar_wait(&bars.p_full[b], ph, &abort_flag);
+                    ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.p_full[b], ph, &abort_flag);
                     if (!ok) break;
                     MPIPE_TR(0, sc * 8 + 1);
                     tc_fence_after();
                     issue_ts(Cfg::kColDV, Cfg::kColS + 64 * b, do_lo_of(sc), s > 0);          // dV += P^T dO
                     if (more) {
-                        ok = mbar_wait(&bars.qdo_full[(sc + 2) % NR], ((sc + 2) / NR) & 1, &abort_flag);
+                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[(sc + 2) % NR], ((sc + 2) / NR) & 1, &abort_flag);
                         if (!ok) break;
                         tc_fence_after();
                         issue_kk(Cfg::kColS + 64 * b, k_lo, kt_lo, q_lo_of(sc + 2));          // S^T(s+2)
                         if (leader) umma_commit(&bars.s_full[b]);
                     }
                     MPIPE_TR(0, sc * 8 + 2);
-                    ok = mbar_wait(&bars.ds_full[b], ph, &abort_flag);
+                    ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.ds_full[b], ph, &abort_flag);
                     if (!ok) break;
                     MPIPE_TR(0, sc * 8 + 3);
                     tc_fence_after();
@@ -279,7 +285,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                         if (leader) umma_commit(&bars.dp_full[b]);
                     }
                     if (b == 1) {                                                             // dQ of the 128-query pair
-                        ok = mbar_wait(&bars.dq_empty, ((sc >> 1) & 1) ^ 1, &abort_flag);
+                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.dq_empty, ((sc >> 1) & 1) ^ 1, &abort_flag);
                         if (!ok) break;
                         MPIPE_TR(0, sc * 8 + 4);
                         tc_fence_after();
@@ -316,7 +322,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             const int q_end = it.kv_start + it.kv_len;
             for (int s = 0; s < n2; ++s, ++sc) {
                 const int rs = sc % NR;
-                ok = mbar_wait(&bars.stat_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
+                ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.stat_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
                 if (!ok) break;
                 float* dst = reinterpret_cast<float*>(smem + Cfg::kSmemStat + rs * (2 * kQS * 4)) + (is_lse ? 0 : kQS);
                 const int q0 = it.kv_start + s * kQS;
@@ -367,29 +373,37 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 if (!ok) break;
                 if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 1);
                 tc_fence_after();
+                // P^T = exp2(S^T * scale*log2e - LSE*log2e): both 32-column halves are requested before the
+                // one wait; multiply-add on packed fp32 pairs
                 float pr[64];
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t sr[32];
-                    tmem_ld32(t_s + h * 32, sr);
+                {
+                    uint32_t sr[64];
+                    tmem_ld32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
+                    tmem_ld32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
                     tmem_wait_ld();
-                    uint32_t pk[16];
+                    const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
 #pragma unroll
-                    for (int c4 = 0; c4 < 8; ++c4) {
-                        const float4 l4 = MPIPE_DBG(4) ? make_float4(1.f, 1.f, 1.f, 1.f) : lse4[h * 8 + c4];
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(sr[4 * c4 + 0]), p.scale_log2, -l4.x));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(sr[4 * c4 + 1]), p.scale_log2, -l4.y));
-                        const float p2 = ex2_approx(fmaf(__uint_as_float(sr[4 * c4 + 2]), p.scale_log2, -l4.z));
-                        const float p3 = ex2_approx(fmaf(__uint_as_float(sr[4 * c4 + 3]), p.scale_log2, -l4.w));
-                        pr[h * 32 + 4 * c4 + 0] = p0;
-                        pr[h * 32 + 4 * c4 + 1] = p1;
-                        pr[h * 32 + 4 * c4 + 2] = p2;
-                        pr[h * 32 + 4 * c4 + 3] = p3;
-                        pk[2 * c4] = pack_bf16(p0, p1);
-                        pk[2 * c4 + 1] = pack_bf16(p2, p3);
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int c4 = 0; c4 < 8; ++c4) {
+                            const float4 l4 = MPIPE_DBG(4) ? make_float4(1.f, 1.f, 1.f, 1.f) : lse4[h * 8 + c4];
+                            const int e = h * 32 + 4 * c4;
+                            const float2 x01 = fma2(make_float2(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), sc2,
+                                                    make_float2(-l4.x, -l4.y));
+                            const float2 x23 = fma2(make_float2(__uint_as_float(sr[e + 2]), __uint_as_float(sr[e + 3])), sc2,
+                                                    make_float2(-l4.z, -l4.w));
+                            pr[e] = ex2_approx(x01.x);
+                            pr[e + 1] = ex2_approx(x01.y);
+                            pr[e + 2] = ex2_approx(x23.x);
+                            pr[e + 3] = ex2_approx(x23.y);
+                            pk[2 * c4] = pack_bf16(pr[e], pr[e + 1]);
+                            pk[2 * c4 + 1] = pack_bf16(pr[e + 2], pr[e + 3]);
+                        }
+                        tmem_st16(t_s + h * 16, pk);
                     }
-                    tmem_st16(t_s + h * 16, pk);
                 }
+                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 6);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
@@ -405,30 +419,43 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 }
                 if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 3);
                 tc_fence_after();
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t dr[32];
-                    tmem_ld32(t_dp + h * 32, dr);
+                // dS^T = P^T o (dP^T - Delta); key rows past the segment are zeroed on the packed words
+                {
+                    uint32_t dr[64];
+                    tmem_ld32(t_dp, *reinterpret_cast<uint32_t(*)[32]>(&dr[0]));
+                    tmem_ld32(t_dp + 32, *reinterpret_cast<uint32_t(*)[32]>(&dr[32]));
                     tmem_wait_ld();
-                    uint32_t pk[16];
+                    if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 7);
+                    uint32_t pk[32];
 #pragma unroll
-                    for (int c4 = 0; c4 < 8; ++c4) {
-                        const float4 d4 = MPIPE_DBG(4) ? make_float4(1.f, 1.f, 1.f, 1.f) : dl4[h * 8 + c4];
-                        float s0 = pr[h * 32 + 4 * c4 + 0] * (__uint_as_float(dr[4 * c4 + 0]) - d4.x);
-                        float s1 = pr[h * 32 + 4 * c4 + 1] * (__uint_as_float(dr[4 * c4 + 1]) - d4.y);
-                        float s2 = pr[h * 32 + 4 * c4 + 2] * (__uint_as_float(dr[4 * c4 + 2]) - d4.z);
-                        float s3 = pr[h * 32 + 4 * c4 + 3] * (__uint_as_float(dr[4 * c4 + 3]) - d4.w);
-                        if (!key_valid) s0 = s1 = s2 = s3 = 0.f;  // rows past the segment must not reach dQ
-                        pk[2 * c4] = pack_bf16(s0, s1);
-                        pk[2 * c4 + 1] = pack_bf16(s2, s3);
+                    for (int c4 = 0; c4 < 16; ++c4) {
+                        const float4 d4 = MPIPE_DBG(4) ? make_float4(1.f, 1.f, 1.f, 1.f) : dl4[c4];
+                        const int e = 4 * c4;
+                        const float2 t01 = add2(make_float2(__uint_as_float(dr[e]), __uint_as_float(dr[e + 1])),
+                                                make_float2(-d4.x, -d4.y));
+                        const float2 t23 = add2(make_float2(__uint_as_float(dr[e + 2]), __uint_as_float(dr[e + 3])),
+                                                make_float2(-d4.z, -d4.w));
+                        const float2 s01 = mul2(make_float2(pr[e], pr[e + 1]), t01);
+                        const float2 s23 = mul2(make_float2(pr[e + 2], pr[e + 3]), t23);
+                        pk[2 * c4] = key_valid ? pack_bf16(s01.x, s01.y) : 0u;
+                        pk[2 * c4 + 1] = key_valid ? pack_bf16(s23.x, s23.y) : 0u;
                     }
-                    tmem_st16(t_dp + h * 16, pk);
-                    // the same 32 values as 4 x 16 bytes of row r of the [key][q] tile (128-byte swizzle)
+#ifdef MPIPE_TRACE
+                    {   // keep the math above from sinking below the trace point
+                        uint32_t x = 0;
 #pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        const int chunk = h * 4 + cc;
+                        for (int i = 0; i < 32; ++i) x ^= pk[i];
+                        if (x == 0x12345678u) MPIPE_TR(3, 4095);
+                    }
+                    if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 5);   // reuses slot 5 (after P phase)
+#endif
+                    tmem_st16(t_dp, *reinterpret_cast<uint32_t(*)[16]>(&pk[0]));
+                    tmem_st16(t_dp + 16, *reinterpret_cast<uint32_t(*)[16]>(&pk[16]));
+                    // the same 64 values as 8 x 16 bytes of row r of the [key][q] tile (128-byte swizzle)
+#pragma unroll
+                    for (int chunk = 0; chunk < 8; ++chunk) {
                         if (!MPIPE_DBG(2)) *reinterpret_cast<uint4*>(ds_row + ((chunk ^ (r & 7)) << 4)) =
-                            make_uint4(pk[4 * cc], pk[4 * cc + 1], pk[4 * cc + 2], pk[4 * cc + 3]);
+                            make_uint4(pk[4 * chunk], pk[4 * chunk + 1], pk[4 * chunk + 2], pk[4 * chunk + 3]);
                     }
                 }
                 tmem_wait_st();
@@ -461,7 +488,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             // they keep walking the (now empty) iterations together instead of leaving one another behind.
             for (int i = 0; i < npairs; ++i, ++pc) {
                 if (lane == 0 && warp == 12) MPIPE_TR(3, pc * 8 + 0);
-                if (ok) ok = mbar_wait(&bars.dq_full, pc & 1, &abort_flag);
+                if (ok) ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.dq_full, pc & 1, &abort_flag);
                 if (lane == 0 && warp == 12) MPIPE_TR(3, pc * 8 + 1);
                 tc_fence_after();
                 uint8_t* stage = smem + Cfg::kSmemStage + (pc % Cfg::kStageBufs) * Cfg::kStageBytes;
@@ -503,7 +530,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 }
                 if (lane == 0 && warp == 12) MPIPE_TR(3, pc * 8 + 2);
             }
-            if (ok) ok = mbar_wait(&bars.dkv_full, unit_it & 1, &abort_flag);
+            if (ok) ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.dkv_full, unit_it & 1, &abort_flag);
             if (!ok) continue;   // keep walking the units so that the named barriers above stay matched
             tc_fence_after();
             const bool store = r < it.row_len;

@@ -55,12 +55,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 #ifndef MPIPE_WAIT_BUDGET_CYCLES
 #define MPIPE_WAIT_BUDGET_CYCLES (2000000000ll)
 #endif
+// kSleepNs > 0 backs off between polls: roles with slack (producer, staging, reducer) must not compete
+// with the softmax warps of their scheduler for issue slots and shared-memory queue entries.
+template <int kSleepNs = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0xFF) == 0) {
+        if (kSleepNs > 0) __nanosleep(kSleepNs);
+        if ((++spins & (kSleepNs > 0 ? 0xF : 0xFF)) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > MPIPE_WAIT_BUDGET_CYCLES) {
                 *abort_flag = 1;
@@ -254,6 +258,11 @@ __device__ __forceinline__ float ex2_approx(float x) {
 }
 
 // Packed pairs of fp32 (sm_100): one instruction for two lanes of a row's arithmetic.
+#ifdef MPIPE_NO_F32X2
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return make_float2(fmaf(a.x, b.x, c.x), fmaf(a.y, b.y, c.y)); }
+__device__ __forceinline__ float2 add2(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return make_float2(a.x * b.x, a.y * b.y); }
+#else
 __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
     float2 d;
     asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
@@ -284,6 +293,8 @@ __device__ __forceinline__ float2 mul2(float2 a, float2 b) {
         : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
     return d;
 }
+
+#endif
 
 template <int kRegs>
 __device__ __forceinline__ void setmaxnreg_inc() {
