@@ -124,18 +124,32 @@ class SegPlan:
     cu_seqlens_dev: Optional[torch.Tensor] = None
     fwd_items_dev: Optional[torch.Tensor] = None
     bwd_items_dev: Optional[torch.Tensor] = None
+    _host_staging: Optional[torch.Tensor] = None
 
     @property
     def n_seg(self) -> int:
         return self.cu_seqlens.size - 1
 
     def to_device(self, device="cuda") -> "SegPlan":
-        def up(a, cols):
-            t = torch.from_numpy(np.ascontiguousarray(a).view(np.int32).reshape(-1, cols).copy())
-            return t.to(device, non_blocking=False)
-        self.cu_seqlens_dev = up(self.cu_seqlens, 1).reshape(-1)
-        self.fwd_items_dev = up(self.fwd_items, 6)
-        self.bwd_items_dev = up(self.bwd_items, 6)
+        """Upload cu_seqlens and both item lists with ONE asynchronous copy from a pinned staging buffer
+        (stream-ordered on the current stream; the host does not wait for the device)."""
+        parts = [np.ascontiguousarray(self.cu_seqlens).view(np.int32).reshape(-1),
+                 np.ascontiguousarray(self.fwd_items).view(np.int32).reshape(-1),
+                 np.ascontiguousarray(self.bwd_items).view(np.int32).reshape(-1)]
+        sizes = [x.size for x in parts]
+        offs = np.concatenate([[0], np.cumsum([(n + 3) // 4 * 4 for n in sizes])])   # 16-byte aligned sections
+        total = int(offs[-1])
+        host = torch.empty(max(total, 4), dtype=torch.int32)
+        if torch.device(device).type == "cuda":
+            host = host.pin_memory()
+        hv = host.numpy()
+        for x, o, n in zip(parts, offs[:-1], sizes):
+            hv[o:o + n] = x
+        dev = host.to(device, non_blocking=True)
+        self._host_staging = host     # keep the pinned buffer alive until the copy has run
+        self.cu_seqlens_dev = dev[offs[0]:offs[0] + sizes[0]]
+        self.fwd_items_dev = dev[offs[1]:offs[1] + sizes[1]].view(-1, 6)
+        self.bwd_items_dev = dev[offs[2]:offs[2] + sizes[2]].view(-1, 6)
         return self
 
 

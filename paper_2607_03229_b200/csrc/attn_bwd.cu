@@ -34,7 +34,7 @@ namespace mpipe {
 #ifdef MPIPE_TRACE
 __device__ long long g_trace[4][4096];
 __device__ int g_dbg_flags;   // knock-out switches for experiments: 1 no atomics, 2 no dS smem store, 4 no LSE/Delta smem loads, 8 no ex2
-#define MPIPE_DBG(bit) ((g_dbg_flags & (bit)) != 0)
+#define MPIPE_DBG(bit) ((dbg_flags & (bit)) != 0)
 #define MPIPE_TR(role, idx)                                                                  \
     do {                                                                                     \
         if (blockIdx.x == 0 && (idx) < 4096) g_trace[role][(idx)] = clock64();               \
@@ -53,6 +53,12 @@ __device__ int g_dbg_flags;   // knock-out switches for experiments: 1 no atomic
 #define MPIPE_SLEEP_MMA 0
 #endif
 constexpr int kBwdThreads = 512;
+// Register re-balancing (setmaxnreg): an increase can only draw on registers that other warps of the
+// same CTA have released, so what the 4 service and 4 reducer warps give back must cover what the 8
+// softmax warps take -- otherwise the increase blocks forever.
+constexpr int kRegsLaunch = 128, kRegsService = 72, kRegsReducer = 96, kRegsSoftmax = 168;
+static_assert(4 * (kRegsLaunch - kRegsService) + 4 * (kRegsLaunch - kRegsReducer) >= 8 * (kRegsSoftmax - kRegsLaunch),
+              "setmaxnreg pool arithmetic");
 constexpr int kBT = 128;  // keys per unit = TMEM lanes
 constexpr int kQS = 64;   // query rows per sub-tile (one pipeline stage of S^T / dP^T)
 
@@ -105,7 +111,7 @@ struct BwdMaps {
 };
 
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads, 1)
+__global__ void __maxnreg__(kRegsLaunch)
 attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
     using Cfg = BwdCfg<D>;
     constexpr int NR = Cfg::kRing;
@@ -118,6 +124,9 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
+#ifdef MPIPE_TRACE
+    const int dbg_flags = g_dbg_flags;
+#endif
 
     if (tid == 0) {
         abort_flag = 0;
@@ -156,7 +165,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        setmaxnreg_dec<72>();
+        setmaxnreg_dec<kRegsService>();
         if (lane == 0) {
             uint32_t unit_it = 0, sc = 0;
             bool ok = true;
@@ -195,7 +204,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         // ------------------------------------------------------------------ tcgen05 issuer
         // The whole warp walks the loop (uniform control flow); one elected lane issues and commits.
         // Descriptors are precomputed halves: a K-step only adds a constant to the low word.
-        setmaxnreg_dec<72>();
+        setmaxnreg_dec<kRegsService>();
         {
             const bool leader = elect_one();
             const uint32_t sbase = smem_u32(smem);
@@ -310,7 +319,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         __syncwarp();
     } else if (warp < 4) {
         // ------------------------------------------------------------------ LSE (warp 2) / Delta (warp 3) staging
-        setmaxnreg_dec<72>();
+        setmaxnreg_dec<kRegsService>();
         const bool is_lse = (warp == 2);
         const float* src = is_lse ? p.lse : p.delta;
         uint32_t sc = 0;
@@ -330,12 +339,12 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 for (int e = 0; e < 2; ++e) {
                     const int c = lane + 32 * e;
                     const int q = q0 + c;
-                    float val;
+                    float val;   // stored negated: -LSE*log2e and -Delta are what the softmax warps add
                     if (q < q_end) {
-                        val = __ldg(src + int64_t(head) * p.total_tokens + q);
+                        val = -__ldg(src + int64_t(head) * p.total_tokens + q);
                         if (is_lse) val *= 1.4426950408889634f;
                     } else {
-                        val = is_lse ? CUDART_INF_F : 0.f;  // P = exp2(-inf) = 0 for query columns past the segment
+                        val = is_lse ? -CUDART_INF_F : 0.f;  // P = exp2(-inf) = 0 for query columns past the segment
                     }
                     dst[c] = val;
                 }
@@ -346,7 +355,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
     } else if (warp < 12) {
         // ------------------------------------------------------------------ softmax / dS warps
         // Warpgroup g owns TMEM stage g, i.e. every other 64-query sub-tile; thread = key row.
-        setmaxnreg_inc<168>();
+        setmaxnreg_inc<kRegsSoftmax>();
         const int g = (warp - 4) >> 2;
         const int r = ((warp & 3) << 5) | lane;
         const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
@@ -359,6 +368,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             const mpipe_work_item_t it = p.items[u / p.n_heads];
             const int n2 = subtiles_of(it);
             const bool key_valid = r < it.row_len;
+            const bool ragged_keys = it.row_len < kBT;
             for (int s = g; s < n2; s += 2) {
                 const uint32_t c = sc + s;
                 const int rs = c % NR;
@@ -390,9 +400,9 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                             const float4 l4 = MPIPE_DBG(4) ? make_float4(1.f, 1.f, 1.f, 1.f) : lse4[h * 8 + c4];
                             const int e = h * 32 + 4 * c4;
                             const float2 x01 = fma2(make_float2(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), sc2,
-                                                    make_float2(-l4.x, -l4.y));
+                                                    make_float2(l4.x, l4.y));
                             const float2 x23 = fma2(make_float2(__uint_as_float(sr[e + 2]), __uint_as_float(sr[e + 3])), sc2,
-                                                    make_float2(-l4.z, -l4.w));
+                                                    make_float2(l4.z, l4.w));
                             pr[e] = ex2_approx(x01.x);
                             pr[e + 1] = ex2_approx(x01.y);
                             pr[e + 2] = ex2_approx(x23.x);
@@ -432,23 +442,19 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                         const float4 d4 = MPIPE_DBG(4) ? make_float4(1.f, 1.f, 1.f, 1.f) : dl4[c4];
                         const int e = 4 * c4;
                         const float2 t01 = add2(make_float2(__uint_as_float(dr[e]), __uint_as_float(dr[e + 1])),
-                                                make_float2(-d4.x, -d4.y));
+                                                make_float2(d4.x, d4.y));
                         const float2 t23 = add2(make_float2(__uint_as_float(dr[e + 2]), __uint_as_float(dr[e + 3])),
-                                                make_float2(-d4.z, -d4.w));
+                                                make_float2(d4.z, d4.w));
                         const float2 s01 = mul2(make_float2(pr[e], pr[e + 1]), t01);
                         const float2 s23 = mul2(make_float2(pr[e + 2], pr[e + 3]), t23);
-                        pk[2 * c4] = key_valid ? pack_bf16(s01.x, s01.y) : 0u;
-                        pk[2 * c4 + 1] = key_valid ? pack_bf16(s23.x, s23.y) : 0u;
+                        pk[2 * c4] = pack_bf16(s01.x, s01.y);
+                        pk[2 * c4 + 1] = pack_bf16(s23.x, s23.y);
                     }
-#ifdef MPIPE_TRACE
-                    {   // keep the math above from sinking below the trace point
-                        uint32_t x = 0;
+                    if (ragged_keys) {   // uniform per unit: only a segment's last key tile has rows to zero
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) x ^= pk[i];
-                        if (x == 0x12345678u) MPIPE_TR(3, 4095);
+                        for (int i = 0; i < 32; ++i) pk[i] = key_valid ? pk[i] : 0u;
                     }
-                    if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 5);   // reuses slot 5 (after P phase)
-#endif
+                    if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 5);
                     tmem_st16(t_dp, *reinterpret_cast<uint32_t(*)[16]>(&pk[0]));
                     tmem_st16(t_dp + 16, *reinterpret_cast<uint32_t(*)[16]>(&pk[16]));
                     // the same 64 values as 8 x 16 bytes of row r of the [key][q] tile (128-byte swizzle)
@@ -474,7 +480,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         // ------------------------------------------------------------------ dQ reducer + dK/dV epilogue
         // dQ of a 128-query pair: TMEM -> registers -> swizzled staging in shared memory -> one TMA
         // reduce-add per 32 fp32 columns into the global accumulator (the copy engine does the atomics).
-        setmaxnreg_dec<96>();
+        setmaxnreg_dec<kRegsReducer>();
         const int r = ((warp & 3) << 5) | lane;
         const int rt = tid - 12 * 32;   // 0..127 inside the warpgroup
         const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;

@@ -28,6 +28,10 @@ constexpr int kFwdThreads = 384;
 constexpr int kTileM = 128;        // query rows per tile (= TMEM lanes)
 constexpr int kTileN = 128;        // keys per K/V tile
 constexpr float kRescaleThreshold = 8.0f;  // in log2 units
+// setmaxnreg: the 4 light warps release what the 8 softmax warps take (an increase blocks until the CTA's
+// own pool has the registers).
+constexpr int kFwdRegsLaunch = 168, kFwdRegsLight = 56, kFwdRegsSoftmax = 224;
+static_assert(4 * (kFwdRegsLaunch - kFwdRegsLight) >= 8 * (kFwdRegsSoftmax - kFwdRegsLaunch), "setmaxnreg pool arithmetic");
 
 template <int D>
 struct FwdCfg {
@@ -62,7 +66,7 @@ struct FwdBarriers {
 };
 
 template <int D>
-__global__ void __launch_bounds__(kFwdThreads, 1)
+__global__ void __maxnreg__(kFwdRegsLaunch)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_q_tail,
                 const __grid_constant__ CUtensorMap map_k_tail, const FwdParams p) {
@@ -112,7 +116,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const int n_units = p.n_items * p.n_heads;
 
     if (warp == 0) {
-        setmaxnreg_dec<56>();
+        setmaxnreg_dec<kFwdRegsLight>();
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t kv_it = 0, unit_it = 0;
@@ -154,7 +158,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // ------------------------------------------------------------------ tcgen05 issuer
         // The whole warp walks the loop (uniform control flow, uniform descriptors); one elected lane
         // issues the MMAs and commits.  Descriptors are precomputed: a K-step only bumps the low word.
-        setmaxnreg_dec<56>();
+        setmaxnreg_dec<kFwdRegsLight>();
         {
             const bool leader = elect_one();
             const uint32_t sbase = smem_u32(smem);
@@ -264,10 +268,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         __syncwarp();
     } else if (warp < 4) {
-        setmaxnreg_dec<56>();
+        setmaxnreg_dec<kFwdRegsLight>();
     } else {
         // ------------------------------------------------------------------ softmax + epilogue
-        setmaxnreg_inc<224>();
+        setmaxnreg_inc<kFwdRegsSoftmax>();
         const int w = (warp - 4) >> 2;              // query tile handled by this warpgroup
         const int r = ((warp & 3) << 5) | lane;     // row inside the tile = TMEM lane
         const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
