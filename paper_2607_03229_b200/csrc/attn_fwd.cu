@@ -28,6 +28,10 @@ constexpr int kFwdThreads = 384;
 constexpr int kTileM = 128;        // query rows per tile (= TMEM lanes)
 constexpr int kTileN = 128;        // keys per K/V tile
 constexpr float kRescaleThreshold = 8.0f;  // in log2 units
+#ifndef MPIPE_FWD_POLY_MASK
+#define MPIPE_FWD_POLY_MASK 0x52
+#endif
+constexpr unsigned kPolyMask = MPIPE_FWD_POLY_MASK;   // bit i: column pair i (mod 8) uses the polynomial exp2
 // setmaxnreg: the 4 light warps release what the 8 softmax warps take (an increase blocks until the CTA's
 // own pool has the registers).
 constexpr int kFwdRegsLaunch = 168, kFwdRegsLight = 56, kFwdRegsSoftmax = 224;
@@ -303,18 +307,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     for (int c = 0; c < 128; ++c)
                         if (c >= n_valid) sr[c] = 0xFF800000u;  // -inf
                 }
-                // eight independent running maxima (a single chain of 127 dependent max ops would cost
-                // ~4 cycles each with only two softmax warps per scheduler to hide it)
+                // eight independent running maxima, three inputs per instruction (a single chain of 127
+                // dependent max ops would cost ~4 cycles each with only two softmax warps per scheduler)
                 float mx8[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) mx8[e] = __uint_as_float(sr[e]);
+                for (int e = 0; e < 8; ++e) mx8[e] = fmaxf(__uint_as_float(sr[e]), __uint_as_float(sr[8 + e]));
 #pragma unroll
-                for (int c = 8; c < 128; c += 8) {
+                for (int c = 16; c < 128; c += 16) {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) mx8[e] = fmaxf(mx8[e], __uint_as_float(sr[c + e]));
+                    for (int e = 0; e < 8; ++e)
+                        mx8[e] = fmax3(mx8[e], __uint_as_float(sr[c + e]), __uint_as_float(sr[c + 8 + e]));
                 }
-                const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
-                                       fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+                const float mx = fmax3(fmax3(mx8[0], mx8[1], mx8[2]), fmax3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7]));
                 const float m_tile = mx * p.scale_log2;
                 const bool grow = m_tile > m_ref + kRescaleThreshold;  // always true on the first tile
                 const float m_new = grow ? m_tile : m_ref;
@@ -344,7 +348,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
                         const float2 x = fma2(make_float2(__uint_as_float(sr[c0 + c]), __uint_as_float(sr[c0 + c + 1])), sc2, nm2);
-                        const float2 e = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+                        // kPolyMask picks, out of every 8 column pairs, those whose exponential runs on the FMA
+                        // pipes; the rest use the special-function unit.  The split balances the two.
+                        const float2 e = ((kPolyMask >> ((c >> 1) & 7)) & 1) ? exp2_poly2(x)
+                                                                           : make_float2(ex2_approx(x.x), ex2_approx(x.y));
                         acc[(c >> 1) & 3] = add2(acc[(c >> 1) & 3], e);
                         pk[c >> 1] = pack_bf16(e.x, e.y);
                     }

@@ -251,6 +251,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+// Three-input maximum (one instruction on sm_100).
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -295,6 +301,26 @@ __device__ __forceinline__ float2 mul2(float2 a, float2 b) {
 }
 
 #endif
+
+// 2^x for a pair of values on the FMA/ALU pipes instead of the special-function unit (which delivers
+// only 16 results per clock per SM and is the forward softmax's bottleneck at head_dim 64):
+// x = n + f with n = round(x) taken from the mantissa of x + 1.5*2^23, f in [-0.5, 0.5];
+// 2^f by a degree-3 minimax polynomial (relative error 7.5e-5, far below the bf16 rounding of P);
+// 2^n by adding n to the exponent field.  Inputs are clamped at -126 (covers -inf of masked columns).
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
+    const float2 t = add2(x, make_float2(12582912.f, 12582912.f));
+    const float2 n = add2(t, make_float2(-12582912.f, -12582912.f));
+    const float2 f = fma2(n, make_float2(-1.f, -1.f), x);
+    float2 p = fma2(f, make_float2(0.05517167f, 0.05517167f), make_float2(0.24261113f, 0.24261113f));
+    p = fma2(p, f, make_float2(0.69326097f, 0.69326097f));
+    p = fma2(p, f, make_float2(0.99992806f, 0.99992806f));
+    float2 r;
+    r.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+    r.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+    return r;
+}
 
 template <int kRegs>
 __device__ __forceinline__ void setmaxnreg_inc() {
