@@ -581,32 +581,45 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
     if (tid == 0 && abort_flag) report_status(p.status_buf, MPIPE_ERR_TIMEOUT, int32_t(blockIdx.x));
 }
 
-// Delta[h,t] = sum_d dO[t,h,d] * O[t,h,d]; clears the fp32 dQ accumulator row of (t,h).  One thread per (t,h).
+// Delta[h,t] = sum_d dO[t,h,d] * O[t,h,d], and the fp32 dQ accumulator is cleared.  HBM-bound helper:
+// kLanes lanes share one (t,h) row (16 bytes of dO and of O each, coalesced across the row), partial
+// dot products are combined with shuffles; the accumulator is cleared with flat 16-byte stores.
 template <int D>
 __global__ void __launch_bounds__(256)
 bwd_prepass_kernel(const __nv_bfloat16* __restrict__ dout, const __nv_bfloat16* __restrict__ o, int64_t tok_stride_o,
                    int64_t head_stride_o, int32_t total_tokens, int32_t n_heads, float* __restrict__ delta,
                    float* __restrict__ dq_acc) {
-    const int64_t idx = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (idx >= int64_t(total_tokens) * n_heads) return;
-    const int t = int(idx / n_heads), h = int(idx % n_heads);
-    const uint4* a = reinterpret_cast<const uint4*>(dout + t * tok_stride_o + h * head_stride_o);
-    const uint4* b = reinterpret_cast<const uint4*>(o + t * tok_stride_o + h * head_stride_o);
-    float acc = 0.f;
+    constexpr int kLanes = (D == 64) ? 8 : 16;   // lanes per row (D = 80 uses 10 of 16)
+    constexpr int kRowsPerBlock = 256 / kLanes;
+    const int64_t n_rows = int64_t(total_tokens) * n_heads;
+    const int sub = threadIdx.x % kLanes;
+    for (int64_t row0 = int64_t(blockIdx.x) * kRowsPerBlock; row0 < n_rows; row0 += int64_t(gridDim.x) * kRowsPerBlock) {
+        const int64_t idx = row0 + threadIdx.x / kLanes;
+        float acc = 0.f;
+        int t = 0, h = 0;
+        if (idx < n_rows) {
+            t = int(idx / n_heads);
+            h = int(idx % n_heads);
+            if (sub * 8 < D) {
+                const uint4 x = __ldg(reinterpret_cast<const uint4*>(dout + t * tok_stride_o + h * head_stride_o) + sub);
+                const uint4 y = __ldg(reinterpret_cast<const uint4*>(o + t * tok_stride_o + h * head_stride_o) + sub);
+                const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
-    for (int c = 0; c < D / 8; ++c) {
-        const uint4 x = __ldg(a + c), y = __ldg(b + c);
-        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            acc = fmaf(__uint_as_float(xs[e] << 16), __uint_as_float(ys[e] << 16), acc);
-            acc = fmaf(__uint_as_float(xs[e] & 0xFFFF0000u), __uint_as_float(ys[e] & 0xFFFF0000u), acc);
+                for (int e = 0; e < 4; ++e) {
+                    acc = fmaf(__uint_as_float(xs[e] << 16), __uint_as_float(ys[e] << 16), acc);
+                    acc = fmaf(__uint_as_float(xs[e] & 0xFFFF0000u), __uint_as_float(ys[e] & 0xFFFF0000u), acc);
+                }
+            }
         }
-    }
-    delta[int64_t(h) * total_tokens + t] = acc;
-    float4* z = reinterpret_cast<float4*>(dq_acc + idx * D);
 #pragma unroll
-    for (int c = 0; c < D / 4; ++c) z[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int m = kLanes / 2; m > 0; m >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
+        if (idx < n_rows && sub == 0) delta[int64_t(h) * total_tokens + t] = acc;
+        // clear the accumulator rows of this block: kRowsPerBlock * D floats, contiguous
+        const int64_t z0 = row0 * D;
+        const int64_t z1 = (row0 + kRowsPerBlock < n_rows ? row0 + kRowsPerBlock : n_rows) * D;
+        float4* z = reinterpret_cast<float4*>(dq_acc);
+        for (int64_t i = z0 / 4 + threadIdx.x; i < z1 / 4; i += 256) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
 }
 
 // dQ[t,h,:] = scale * acc[t,h,:] as bf16.  One thread per 8 elements.
@@ -655,7 +668,9 @@ static int32_t launch_bwd(const void* dout, const void* q, const void* k, const 
         cudaSuccess)
         return MPIPE_ERR_CUDA;
     const int64_t rows = int64_t(total_tokens) * n_heads;
-    bwd_prepass_kernel<D><<<unsigned((rows + 255) / 256), 256, 0, stream>>>(
+    const int64_t prepass_blocks = (rows + (D == 64 ? 32 : 16) - 1) / (D == 64 ? 32 : 16);
+    const int64_t prepass_cap = int64_t(sm_count()) * 64;
+    bwd_prepass_kernel<D><<<unsigned(prepass_blocks < prepass_cap ? prepass_blocks : prepass_cap), 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(dout), static_cast<const __nv_bfloat16*>(o), ts_o, hs_o, total_tokens, n_heads,
         delta, dq_acc);
     const int n_units = prm.n_items * prm.n_heads;
