@@ -72,11 +72,12 @@ struct BwdCfg {
     static constexpr int kSubTail = kTail ? kQS * 32 : 0;
     static constexpr int kSub = kSubMain + kSubTail;
     static constexpr int kRing = 4;                             // Q/dO sub-tile stages
+    static constexpr int kKVBufs = (D == 64) ? 2 : 1;           // D = 64: the next unit's K/V tiles load during the current unit
     static constexpr int kStageBytes = kBT * (D * 4);           // dQ staging for the TMA reduction: [128 q][D fp32]
-    static constexpr int kStageBufs = (D == 64) ? 2 : 1;        // what fits next to the rest
-    static constexpr int kSmemK = 0;
+    static constexpr int kStageBufs = 1;
+    static constexpr int kSmemK = 0;                            // buffer i at kSmemK + i * 2 * kTile (K then V)
     static constexpr int kSmemV = kTile;
-    static constexpr int kSmemQ = 2 * kTile;
+    static constexpr int kSmemQ = kKVBufs * 2 * kTile;
     static constexpr int kSmemDO = kSmemQ + kRing * kSub;
     static constexpr int kSmemDS = kSmemDO + kRing * kSub;      // dS^T as [key][q]: two 64-query atoms of 16 KB
     static constexpr int kSmemStage = kSmemDS + 2 * kBT * 128;  // two staging buffers
@@ -101,7 +102,7 @@ struct BwdParams {
 };
 
 struct BwdBarriers {
-    uint64_t kv_full, kv_empty, dkv_full, dkv_empty;
+    uint64_t kv_full[2], kv_empty[2], dkv_full, dkv_empty;
     uint64_t qdo_full[4], qdo_empty[4], stat_full[4], stat_empty[4];
     uint64_t s_full[2], p_full[2], dp_full[2], ds_full[2], dq_full, dq_empty;
 };
@@ -130,8 +131,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
 
     if (tid == 0) {
         abort_flag = 0;
-        mbar_init(&bars.kv_full, 1);
-        mbar_init(&bars.kv_empty, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bars.kv_full[i], 1);
+            mbar_init(&bars.kv_empty[i], 1);
+        }
         mbar_init(&bars.dkv_full, 1);
         mbar_init(&bars.dkv_empty, 4);
         for (int s = 0; s < 4; ++s) {
@@ -173,14 +176,16 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 const mpipe_work_item_t it = p.items[u / p.n_heads];
                 const int head = u % p.n_heads;
                 const int n2 = subtiles_of(it);
-                ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.kv_empty, (unit_it & 1) ^ 1, &abort_flag);
+                const int kb = unit_it % Cfg::kKVBufs;            // K/V buffer of this unit
+                uint8_t* kv = smem + kb * (2 * Cfg::kTile);
+                ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.kv_empty[kb], ((unit_it / Cfg::kKVBufs) & 1) ^ 1, &abort_flag);
                 if (!ok) break;
-                mbar_expect_tx(&bars.kv_full, 2 * Cfg::kTile);
-                tma_load_3d(smem + Cfg::kSmemK, &maps.k, &bars.kv_full, 0, head, it.row_start);
-                tma_load_3d(smem + Cfg::kSmemV, &maps.v, &bars.kv_full, 0, head, it.row_start);
+                mbar_expect_tx(&bars.kv_full[kb], 2 * Cfg::kTile);
+                tma_load_3d(kv + Cfg::kSmemK, &maps.k, &bars.kv_full[kb], 0, head, it.row_start);
+                tma_load_3d(kv + Cfg::kSmemV, &maps.v, &bars.kv_full[kb], 0, head, it.row_start);
                 if (Cfg::kTail) {
-                    tma_load_3d(smem + Cfg::kSmemK + Cfg::kTileMain, &maps.k_tail, &bars.kv_full, 64, head, it.row_start);
-                    tma_load_3d(smem + Cfg::kSmemV + Cfg::kTileMain, &maps.v_tail, &bars.kv_full, 64, head, it.row_start);
+                    tma_load_3d(kv + Cfg::kSmemK + Cfg::kTileMain, &maps.k_tail, &bars.kv_full[kb], 64, head, it.row_start);
+                    tma_load_3d(kv + Cfg::kSmemV + Cfg::kTileMain, &maps.v_tail, &bars.kv_full[kb], 64, head, it.row_start);
                 }
                 for (int s = 0; s < n2; ++s, ++sc) {
                     const int rs = sc % NR;
@@ -210,9 +215,6 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             const uint32_t sbase = smem_u32(smem);
             constexpr uint32_t hi128 = umma_desc_hi(1024, kSwizzle128);
             constexpr uint32_t hi32 = umma_desc_hi(256, kSwizzle32);
-            const uint32_t k_lo = umma_desc_lo(sbase + Cfg::kSmemK, 0), v_lo = umma_desc_lo(sbase + Cfg::kSmemV, 0);
-            const uint32_t kt_lo = umma_desc_lo(sbase + Cfg::kSmemK + Cfg::kTileMain, 0);
-            const uint32_t vt_lo = umma_desc_lo(sbase + Cfg::kSmemV + Cfg::kTileMain, 0);
             const uint32_t ds_lo = umma_desc_lo(sbase + Cfg::kSmemDS, kBT * 128);   // two 64-query atoms 16 KB apart
             constexpr uint32_t idesc_s = umma_idesc_bf16(kBT, kQS, 0, 0);      // K-major x K-major, N = 64 queries
             constexpr uint32_t idesc_ts = umma_idesc_bf16(kBT, 64, 0, 1);      // A in TMEM, MN-major B, N = 64
@@ -249,7 +251,12 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
                 const mpipe_work_item_t it = p.items[u / p.n_heads];
                 const int n2 = subtiles_of(it);
-                ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.kv_full, unit_it & 1, &abort_flag);
+                const int kb = unit_it % Cfg::kKVBufs;
+                const uint32_t kvb = sbase + kb * (2 * Cfg::kTile);
+                const uint32_t k_lo = umma_desc_lo(kvb + Cfg::kSmemK, 0), v_lo = umma_desc_lo(kvb + Cfg::kSmemV, 0);
+                const uint32_t kt_lo = umma_desc_lo(kvb + Cfg::kSmemK + Cfg::kTileMain, 0);
+                const uint32_t vt_lo = umma_desc_lo(kvb + Cfg::kSmemV + Cfg::kTileMain, 0);
+                ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.kv_full[kb], (unit_it / Cfg::kKVBufs) & 1, &abort_flag);
                 if (!ok) break;
                 for (int s = 0; s < 2; ++s) {   // prologue: S^T and dP^T of the first two sub-tiles
                     ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[(sc + s) % NR], ((sc + s) / NR) & 1, &abort_flag);
@@ -313,7 +320,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 }
                 if (!ok) break;
                 if (leader) umma_commit(&bars.dkv_full);
-                if (leader) umma_commit(&bars.kv_empty);
+                if (leader) umma_commit(&bars.kv_empty[kb]);
             }
         }
         __syncwarp();
