@@ -36,7 +36,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one attn_bwd_kernel<64> launch on this workload, from the
 # ncu capture summarised in profiles/attn_bwd_kernel_vit_l.md.
-BWD_MAIN_DRAM_BYTES_PER_LAUNCH = 1.0497e9
+BWD_MAIN_DRAM_BYTES_PER_LAUNCH = 1.0757e9
 
 
 def load_peaks():
@@ -48,9 +48,38 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
+WORKLOADS = {
+    "vit_l": lambda seed: W.vit_l(seed=seed),
+    "qwen2vl": lambda seed: W.qwen2vl(seed=seed + 1),
+    "qwen2vl_frozen": lambda seed: W.qwen2vl(seed=seed + 1, trained=False),
+    "video_tail": lambda seed: W.video_tail(seed=seed + 2),
+    "mix10": lambda seed: W.modality_mix(0.10, seed=seed + 3),
+    "mix25": lambda seed: W.modality_mix(0.25, seed=seed + 3),
+    "mix50": lambda seed: W.modality_mix(0.50, seed=seed + 3),
+    "mix75": lambda seed: W.modality_mix(0.75, seed=seed + 3),
+    "mix75_frozen": lambda seed: W.modality_mix(0.75, seed=seed + 3, trained=False),
+    "tiny": lambda seed: W.tiny(seed=seed - 1),
+}
+WORKLOAD_TEXT = {
+    "vit_l": "vit_l: 32 images of 16..64 x 16..64 patches packed varlen, 16 heads x 64, bf16, trained (fwd+bwd), + merge "
+             "of the encoder output into 16 x 8192 LLM tokens at hidden 1024",
+    "qwen2vl": "qwen2vl: patch counts log-uniform in [64,16384] packed to 65536 tokens, 16 heads x 80, bf16, trained",
+    "qwen2vl_frozen": "qwen2vl: patch counts log-uniform in [64,16384] packed to 65536 tokens, 16 heads x 80, bf16, frozen",
+    "video_tail": "video_tail: 200 images of 64..256 patches + 4 clips of 16384 tokens, 16 heads x 80, bf16, trained",
+    "mix10": "modality mix 10%: 8 x 8192 LLM tokens at hidden 4096, images of 256..4096 patches, 16 heads x 64, trained, + merge",
+    "mix25": "modality mix 25%: 8 x 8192 LLM tokens at hidden 4096, images of 256..4096 patches, 16 heads x 64, trained, + merge",
+    "mix50": "modality mix 50%: 8 x 8192 LLM tokens at hidden 4096, images of 256..4096 patches, 16 heads x 64, trained, + merge",
+    "mix75": "modality mix 75%: 8 x 8192 LLM tokens at hidden 4096, images of 256..4096 patches, 16 heads x 64, trained, + merge",
+    "mix75_frozen": "modality mix 75%: 8 x 8192 LLM tokens at hidden 4096, images of 256..4096 patches, 16 heads x 64, frozen, + merge",
+    "tiny": "tiny: 4 images of 16/49/64/100 patches, 4 heads x 64, trained, + merge into 512 tokens at hidden 256",
+}
+_WORKLOAD_NAME = "vit_l"
+
+
 def workload_for(rank: int):
+    """The benchmark's microbatch for one rank (default: the ViT-L configuration the metric is quoted on)."""
     from paper_2607_03229_b200 import dist as D
-    return W.vit_l(seed=D.rank_seed(W.BASE_SEED + 2, rank))
+    return WORKLOADS[_WORKLOAD_NAME](D.rank_seed(W.BASE_SEED + 2, rank))
 
 
 # ----------------------------------------------------------------------------- oracle sample (CPU arms)
@@ -224,8 +253,9 @@ def ours_arm(args):
     assert int(buf.status[0]) == 0, f"device status {buf.status.tolist()}"
 
     # ---- timed region: K whole steps, inputs resident in HBM, per-kernel events recorded alongside
+    kernels = ["fwd"] + (["bwd_main"] if w.trained else []) + (["merge"] if w.merge_hidden is not None else [])
     ev = {name: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-          for name in ("fwd", "bwd_main", "merge")}
+          for name in kernels}
     slots = {"fwd": B.PROFILE_FWD, "bwd_main": B.PROFILE_BWD_MAIN, "merge": B.PROFILE_MERGE}
     uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid) if hasattr(
         torch.cuda.get_device_properties(dev), "uuid") else str(local_rank)
@@ -242,8 +272,8 @@ def ours_arm(args):
     t_begin = time.perf_counter()
     e0.record()
     for i in range(K):
-        for name, slot in slots.items():
-            B.load().mpipe_set_profile_events(slot, ev[name][i][0].cuda_event, ev[name][i][1].cuda_event)
+        for name in kernels:
+            B.load().mpipe_set_profile_events(slots[name], ev[name][i][0].cuda_event, ev[name][i][1].cuda_event)
         H.run_step(w, buf)
     e1.record()
     torch.cuda.synchronize()
@@ -258,18 +288,20 @@ def ours_arm(args):
 
     # ---- end to end: host buffers in, results out, copies inside the timed region
     Ke = 1 if args.profile_mode else min(K, 30)
-    host_in = [torch.empty((T, Hh, Dh), dtype=torch.bfloat16).pin_memory() for _ in range(4)]
-    for hbuf, dbuf in zip(host_in, (buf.q, buf.k, buf.v, buf.dout)):
+    dev_in = [buf.q, buf.k, buf.v] + ([buf.dout] if w.trained else [])
+    dev_out = [buf.o] + ([buf.dq, buf.dk, buf.dv] if w.trained else [])
+    host_in = [torch.empty(tuple(x.shape), dtype=torch.bfloat16).pin_memory() for x in dev_in]
+    for hbuf, dbuf in zip(host_in, dev_in):
         hbuf.copy_(dbuf)
-    host_out = [torch.empty((T, Hh, Dh), dtype=torch.bfloat16).pin_memory() for _ in range(4)]
-    h2d = sum(x.numel() * x.element_size() for x in host_in) + w.positions.nbytes
+    host_out = [torch.empty(tuple(x.shape), dtype=torch.bfloat16).pin_memory() for x in dev_out]
+    h2d = sum(x.numel() * x.element_size() for x in host_in) + (w.positions.nbytes if w.positions is not None else 0)
     d2h = sum(x.numel() * x.element_size() for x in host_out)
 
     def e2e_step():
-        for hbuf, dbuf in zip(host_in, (buf.q, buf.k, buf.v, buf.dout)):
+        for hbuf, dbuf in zip(host_in, dev_in):
             dbuf.copy_(hbuf, non_blocking=True)
         H.run_step(w, buf)               # includes the host plan and its upload
-        for hbuf, dbuf in zip(host_out, (buf.o, buf.dq, buf.dk, buf.dv)):
+        for hbuf, dbuf in zip(host_out, dev_out):
             hbuf.copy_(dbuf, non_blocking=True)
 
     for _ in range(2):
@@ -286,42 +318,47 @@ def ours_arm(args):
     ms_e2e = f0.elapsed_time(f1) / Ke
 
     # ---- reduce over ranks: max of times, sum of work
-    flops_fb, flops_b = w.flops(True, True), w.flops(False, True)
-    merge_bytes = float(T) * (4 * w.merge_hidden + 4)
-    (ms_step_mx, ms_e2e_mx, ms_bwd_mx, ms_fwd_mx, ms_merge_mx), (flops_all, flops_b_all, merge_all, launches) = \
-        D.reduce_max_sum([ms_step, ms_e2e, kern_ms["bwd_main"], kern_ms["fwd"], kern_ms["merge"]],
-                         [flops_fb, flops_b, merge_bytes, float(n_kernels * K)], device=dev)
+    flops_step = w.flops(True, w.trained)
+    merge_bytes = float(T) * (4 * w.merge_hidden + 4) if w.merge_hidden is not None else 0.0
+    (ms_step_mx, ms_e2e_mx), (flops_all, launches) = D.reduce_max_sum(
+        [ms_step, ms_e2e], [flops_step, float(n_kernels * K)], device=dev)
 
     if rank == 0:
         value = flops_all / (ms_step_mx * 1e-3) / 1e12
-        bwd_tf = w.flops(False, True) / (kern_ms["bwd_main"] * 1e-3) / 1e12       # this rank's kernel, per launch
-        fwd_tf = w.flops(True, False) / (kern_ms["fwd"] * 1e-3) / 1e12
-        merge_gbs = merge_bytes / (kern_ms["merge"] * 1e-3) / 1e9
+        fwd_tf = w.flops(True, False) / (kern_ms["fwd"] * 1e-3) / 1e12       # this rank's kernels, per launch
+        breakdown = {"fwd_ms": kern_ms["fwd"], "fwd_tflops": fwd_tf}
+        if w.trained:
+            bwd_tf = w.flops(False, True) / (kern_ms["bwd_main"] * 1e-3) / 1e12
+            breakdown.update({"bwd_main_ms": kern_ms["bwd_main"], "bwd_main_tflops": bwd_tf})
+        if w.merge_hidden is not None and T > 0:
+            merge_gbs = merge_bytes / (kern_ms["merge"] * 1e-3) / 1e9
+            breakdown.update({"merge_ms": kern_ms["merge"], "merge_gbs": merge_gbs,
+                              "merge_frac_of_hbm_peak": merge_gbs / peaks["hbm_gbs"]})
+        breakdown["attn_frac_of_bf16_peak"] = {"measured_sustained": value / world / peaks["bf16_tflops_sustained"],
+                                               "measured_burst": value / world / peaks["bf16_tflops"],
+                                               "nominal_2250": value / world / NOMINAL_BF16_TFLOPS}
         peak_tf = peaks["bf16_tflops_sustained"]
+        top, top_tf = (f"attn_bwd_kernel<{Dh}>", bwd_tf) if w.trained else (f"attn_fwd_kernel<{Dh}>", fwd_tf)
+        traffic = BWD_MAIN_DRAM_BYTES_PER_LAUNCH if (_WORKLOAD_NAME == "vit_l" and w.trained) else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
             "ms_per_step": ms_step_mx, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "vit_l: 32 images of 16..64 x 16..64 patches packed varlen, 16 heads x 64, bf16, "
-                                   "trained (fwd+bwd), + merge of the encoder output into 16 x 8192 LLM tokens at "
-                                   "hidden 1024; one microbatch per GPU",
-                       "tokens_rank0": T, "sum_n2_rank0": w.sum_n2, "l2": "inputs_exceed_l2 (~1 GB touched per step)",
-                       "step": "host plan + upload, attn fwd, attn bwd (prepass, main, convert), merge"},
-            "breakdown": {"fwd_ms": kern_ms["fwd"], "bwd_main_ms": kern_ms["bwd_main"], "merge_ms": kern_ms["merge"],
-                          "fwd_tflops": fwd_tf, "bwd_main_tflops": bwd_tf, "merge_gbs": merge_gbs,
-                          "merge_frac_of_hbm_peak": merge_gbs / peaks["hbm_gbs"],
-                          "attn_frac_of_bf16_peak": {"measured_sustained": value / world / peaks["bf16_tflops_sustained"],
-                                                     "measured_burst": value / world / peaks["bf16_tflops"],
-                                                     "nominal_2250": value / world / NOMINAL_BF16_TFLOPS}},
-            "roofline": {"kernel": "attn_bwd_kernel<64>", "bound": "tensor", "achieved": bwd_tf, "peak": peak_tf,
-                         "unit": "TFLOP/s", "frac": bwd_tf / peak_tf, "peak_kind": f"{peak_kind}, sustained bf16 GEMM",
-                         "traffic": BWD_MAIN_DRAM_BYTES_PER_LAUNCH},
+            "config": {"workload": WORKLOAD_TEXT[_WORKLOAD_NAME] + "; one microbatch per GPU",
+                       "tokens_rank0": T, "sum_n2_rank0": w.sum_n2, "heads": Hh, "head_dim": Dh,
+                       "mode": "trained (fwd+bwd)" if w.trained else "frozen (fwd only)",
+                       "l2": "inputs_exceed_l2" if T * Hh * Dh * 2 * 4 > 126e6 else "inputs_fit_l2 (no flush)",
+                       "step": "host plan + upload, attn fwd" + (", attn bwd (prepass, main, convert)" if w.trained else "")
+                               + (", merge" if w.merge_hidden is not None else "")},
+            "breakdown": breakdown,
+            "roofline": {"kernel": top, "bound": "tensor", "achieved": top_tf, "peak": peak_tf, "unit": "TFLOP/s",
+                         "frac": top_tf / peak_tf, "peak_kind": f"{peak_kind}, sustained bf16 GEMM", "traffic": traffic},
             "e2e": {"value": flops_all / (ms_e2e_mx * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e_mx,
                     "steps": Ke, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
             "gpu_launches": int(launches),
             "clocks": clocks,
         }
-        if world == 1 and not args.profile_mode:
+        if world == 1 and not args.profile_mode and _WORKLOAD_NAME == "vit_l":
             line["cpu_baseline"] = cpu_baseline(w)
         if args.profile_mode:
             line["profile_mode"] = True
@@ -347,10 +384,15 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="vit_l",
+                    help="which synthetic configuration to run (default: vit_l, the one the metric is quoted on; "
+                         "the others are for the per-config results table)")
     ap.add_argument("--profile-mode", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for short runs under a profiler; the line "
                          "such a run prints is not a benchmark value)")
     args = ap.parse_args()
+    global _WORKLOAD_NAME
+    _WORKLOAD_NAME = args.workload
     if args.impl == "reference":
         return reference_arm(args)
     return ours_arm(args)
