@@ -224,6 +224,16 @@ int32_t mpipe_validate_positions(const int32_t* positions, int32_t n, int32_t n_
  */
 int32_t mpipe_set_profile_events(int32_t which, void* start_event, void* stop_event);
 
+/*
+ * Self-test of the bounded waits (the kernel-level counterpart of the paper's argument that an acyclic
+ * order graph cannot dead-lock, Section 4.2: here a wait that would never be satisfied must end by
+ * itself).  Launches one small CTA that waits on a barrier nobody signals, with a budget of
+ * `budget_cycles` SM clock ticks (1 .. 4e9); when the budget runs out the kernel writes
+ * MPIPE_ERR_TIMEOUT to status_buf[0] (device int32[4], required, zeroed by the caller) and returns
+ * normally.  Nothing traps or faults and the CUDA context stays usable.  Enqueues on `stream`.
+ */
+int32_t mpipe_selftest_wait_timeout(int64_t budget_cycles, int32_t* status_buf, void* stream);
+
 const char* mpipe_status_str(int32_t status);
 int32_t mpipe_version(void);
 

@@ -47,6 +47,7 @@ _SIGNATURES = {
     "mpipe_merge_tokens_bwd": (_i32, [_vp, _i64, _vp, _i64, _vp, _i32, _i32, _i32, _i32, _vp, _vp]),
     "mpipe_validate_positions": (_i32, [_vp, _i32, _i32]),
     "mpipe_set_profile_events": (_i32, [_i32, _vp, _vp]),
+    "mpipe_selftest_wait_timeout": (_i32, [_i64, _vp, _vp]),
     "mpipe_status_str": (ctypes.c_char_p, [_i32]),
     "mpipe_version": (_i32, []),
 }
@@ -262,6 +263,12 @@ def merge_tokens_bwd(d_llm_embeds, d_enc, positions_dev, mode: int, status_buf=N
                                        d_enc.stride(0) if n_enc else hidden, _ptr(positions_dev), n_enc, n_llm,
                                        hidden, mode, _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_merge_tokens_bwd")
+
+
+def selftest_wait_timeout(budget_cycles: int, status_buf, stream=None) -> None:
+    """mpipe_selftest_wait_timeout: a wait that nothing satisfies must end with ERR_TIMEOUT in status_buf."""
+    _check(load().mpipe_selftest_wait_timeout(int(budget_cycles), _ptr(status_buf), _stream(stream)),
+           "mpipe_selftest_wait_timeout")
 
 
 PROFILE_FWD, PROFILE_BWD_MAIN, PROFILE_MERGE = 0, 1, 2

@@ -58,7 +58,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // kSleepNs > 0 backs off between polls: roles with slack (producer, staging, reducer) must not compete
 // with the softmax warps of their scheduler for issue slots and shared-memory queue entries.
 template <int kSleepNs = 0>
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_budget(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                 long long budget_cycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
@@ -66,13 +67,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         if (kSleepNs > 0) __nanosleep(kSleepNs);
         if ((++spins & (kSleepNs > 0 ? 0xF : 0xFF)) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > MPIPE_WAIT_BUDGET_CYCLES) {
+            if (clock64() - t0 > budget_cycles) {
                 *abort_flag = 1;
                 return false;
             }
         }
     }
     return true;
+}
+template <int kSleepNs = 0>
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    return mbar_wait_budget<kSleepNs>(bar, parity, abort_flag, MPIPE_WAIT_BUDGET_CYCLES);
 }
 
 // ----------------------------------------------------------------------- TMA
