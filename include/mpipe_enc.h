@@ -225,6 +225,37 @@ int32_t mpipe_validate_positions(const int32_t* positions, int32_t n, int32_t n_
 int32_t mpipe_set_profile_events(int32_t which, void* start_event, void* stop_event);
 
 /*
+ * Cost model of the transpose schedule (Section 4.3) -- host, double arithmetic, nothing on the device.
+ *
+ *   mpipe_event_cost         cost(Fwd) = cost(Bwd) = max(W / F, D / B): W FLOPs at peak rate F, D bytes of
+ *                            HBM traffic at bandwidth B (the roofline of one compute event).
+ *   mpipe_coll_cost          cost(Coll) = cost(DpReduce) = alpha + beta * n for an n-byte payload.
+ *   mpipe_encoder_attn_work  W and D of this library's attention events for one encoder microbatch:
+ *                            forward 4*H*D*sum n_i^2 FLOPs and sum n_i * H * (8*D [+4 LSE if trained]) bytes;
+ *                            backward (trained only, else 0) 10*H*D*sum n_i^2 FLOPs and
+ *                            sum n_i * H * (16*D + 16) bytes.
+ *   mpipe_warmup_slack_1f1b  w_r, the idle time of pipeline rank r before its first LLM forward under
+ *                            1F1B: r * (stage_fwd_cost + seam_cost).  (The paper's figure is missing; this
+ *                            is the reading "rank r waits for r upstream stage forwards and their sends".)
+ *   mpipe_owner_map          the ByMicrobatch owner: microbatches in order of decreasing encoder cost (ties:
+ *                            lower index first), each to the rank with the most warm-up slack left,
+ *                            w_r - E_r (ties: lower rank) -- "heavier encodes to longer warm-up slots".
+ *                            Outputs owner[m], E_r = sum of the costs a rank received,
+ *                            spill_r = max(0, E_r - w_r) and max_r spill_r, the time the encoder adds to
+ *                            the step.
+ * All pointers are HOST pointers.  Negative or NaN inputs, non-positive peaks or rank counts and NULL
+ * outputs give MPIPE_ERR_INVALID_ARG.
+ */
+int32_t mpipe_event_cost(double flops, double bytes, double peak_flops, double peak_bw, double* cost);
+int32_t mpipe_coll_cost(double alpha, double beta, double payload_bytes, double* cost);
+int32_t mpipe_encoder_attn_work(const int32_t* patch_counts, int32_t n_seg, int32_t n_heads, int32_t head_dim,
+                                int32_t mode, double* fwd_flops, double* fwd_bytes, double* bwd_flops,
+                                double* bwd_bytes);
+int32_t mpipe_warmup_slack_1f1b(int32_t n_ranks, double stage_fwd_cost, double seam_cost, double* slack);
+int32_t mpipe_owner_map(const double* enc_cost, int32_t n_microbatches, const double* warmup_slack, int32_t n_ranks,
+                        int32_t* owner, double* enc_work, double* spill, double* max_spill);
+
+/*
  * Self-test of the bounded waits (the kernel-level counterpart of the paper's argument that an acyclic
  * order graph cannot dead-lock, Section 4.2: here a wait that would never be satisfied must end by
  * itself).  Launches one small CTA that waits on a barrier nobody signals, with a budget of

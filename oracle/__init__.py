@@ -222,3 +222,59 @@ def seg_plan(patch_counts: Sequence[int], fwd_tile_rows: int, bwd_tile_rows: int
     fwd = _tile_items(counts, cu, fwd_tile_rows)
     bwd = _tile_items(counts, cu, bwd_tile_rows) if trained else []
     return cu, cu[-1], (max(counts) if counts else 0), fwd, bwd
+
+
+# ---------------------------------------------------------------------------------------------------
+# Cost model of the transpose schedule (Section 4.3), restated plainly
+# ---------------------------------------------------------------------------------------------------
+
+def event_cost(flops: float, nbytes: float, peak_flops: float, peak_bw: float) -> float:
+    """cost(Fwd) = cost(Bwd) = max(W / F, D / B)."""
+    return max(flops / peak_flops, nbytes / peak_bw)
+
+
+def coll_cost(alpha: float, beta: float, payload_bytes: float) -> float:
+    """cost(Coll) = alpha + beta * n."""
+    return alpha + beta * payload_bytes
+
+
+def encoder_attn_work(patch_counts: Sequence[int], n_heads: int, head_dim: int, trained: bool):
+    """FLOPs and HBM bytes of the attention events of one encoder microbatch."""
+    n1 = sum(int(c) for c in patch_counts)
+    n2 = sum(int(c) * int(c) for c in patch_counts)
+    fwd_flops = 4 * n_heads * head_dim * n2
+    fwd_bytes = n1 * n_heads * (8 * head_dim + (4 if trained else 0))
+    bwd_flops = 10 * n_heads * head_dim * n2 if trained else 0
+    bwd_bytes = n1 * n_heads * (16 * head_dim + 16) if trained else 0
+    return float(fwd_flops), float(fwd_bytes), float(bwd_flops), float(bwd_bytes)
+
+
+def spills(owner: Sequence[int], enc_cost: Sequence[float], warmup_slack: Sequence[float]):
+    """E_r = sum of the encoder costs rank r owns; spill_r = max(0, E_r - w_r)."""
+    work = [0.0] * len(warmup_slack)
+    for m, r in enumerate(owner):
+        work[r] += enc_cost[m]
+    sp = [max(0.0, e - w) for e, w in zip(work, warmup_slack)]
+    return work, sp, (max(sp) if sp else 0.0)
+
+
+def owner_map_greedy(enc_cost: Sequence[float], warmup_slack: Sequence[float]):
+    """Heaviest encode first, each to the rank with the most warm-up slack left (ties: lower index / rank)."""
+    work = [0.0] * len(warmup_slack)
+    owner = [0] * len(enc_cost)
+    for m in sorted(range(len(enc_cost)), key=lambda i: -enc_cost[i]):
+        left = [w - e for w, e in zip(warmup_slack, work)]
+        r = max(range(len(left)), key=lambda i: (left[i], -i))
+        owner[m] = r
+        work[r] += enc_cost[m]
+    return owner
+
+
+def owner_map_optimal(enc_cost: Sequence[float], warmup_slack: Sequence[float]):
+    """Brute force over all assignments (tiny inputs only): the smallest achievable max_r spill_r."""
+    import itertools
+    best = None
+    for owner in itertools.product(range(len(warmup_slack)), repeat=len(enc_cost)):
+        mx = spills(owner, enc_cost, warmup_slack)[2]
+        best = mx if best is None or mx < best else best
+    return 0.0 if best is None else best

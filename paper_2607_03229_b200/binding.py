@@ -48,6 +48,11 @@ _SIGNATURES = {
     "mpipe_validate_positions": (_i32, [_vp, _i32, _i32]),
     "mpipe_set_profile_events": (_i32, [_i32, _vp, _vp]),
     "mpipe_selftest_wait_timeout": (_i32, [_i64, _vp, _vp]),
+    "mpipe_event_cost": (_i32, [ctypes.c_double] * 4 + [_vp]),
+    "mpipe_coll_cost": (_i32, [ctypes.c_double] * 3 + [_vp]),
+    "mpipe_encoder_attn_work": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp]),
+    "mpipe_warmup_slack_1f1b": (_i32, [_i32, ctypes.c_double, ctypes.c_double, _vp]),
+    "mpipe_owner_map": (_i32, [_vp, _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
     "mpipe_status_str": (ctypes.c_char_p, [_i32]),
     "mpipe_version": (_i32, []),
 }
@@ -263,6 +268,47 @@ def merge_tokens_bwd(d_llm_embeds, d_enc, positions_dev, mode: int, status_buf=N
                                        d_enc.stride(0) if n_enc else hidden, _ptr(positions_dev), n_enc, n_llm,
                                        hidden, mode, _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_merge_tokens_bwd")
+
+
+def event_cost(flops: float, nbytes: float, peak_flops: float, peak_bw: float) -> float:
+    out = ctypes.c_double()
+    _check(load().mpipe_event_cost(flops, nbytes, peak_flops, peak_bw, ctypes.addressof(out)), "mpipe_event_cost")
+    return out.value
+
+
+def coll_cost(alpha: float, beta: float, payload_bytes: float) -> float:
+    out = ctypes.c_double()
+    _check(load().mpipe_coll_cost(alpha, beta, payload_bytes, ctypes.addressof(out)), "mpipe_coll_cost")
+    return out.value
+
+
+def encoder_attn_work(patch_counts, n_heads: int, head_dim: int, mode: int):
+    """(fwd_flops, fwd_bytes, bwd_flops, bwd_bytes) of one microbatch's attention events."""
+    counts = np.ascontiguousarray(np.asarray(patch_counts, dtype=np.int32).reshape(-1))
+    out = [ctypes.c_double() for _ in range(4)]
+    _check(load().mpipe_encoder_attn_work(_ptr(counts), counts.size, n_heads, head_dim, mode,
+                                          *[ctypes.addressof(x) for x in out]), "mpipe_encoder_attn_work")
+    return tuple(x.value for x in out)
+
+
+def warmup_slack_1f1b(n_ranks: int, stage_fwd_cost: float, seam_cost: float) -> np.ndarray:
+    w = np.zeros(max(n_ranks, 0), dtype=np.float64)
+    _check(load().mpipe_warmup_slack_1f1b(n_ranks, stage_fwd_cost, seam_cost, _ptr(w) if w.size else None),
+           "mpipe_warmup_slack_1f1b")
+    return w
+
+
+def owner_map(enc_cost, warmup_slack):
+    """mpipe_owner_map.  Returns (owner int32[M], E float64[P], spill float64[P], max_spill)."""
+    cost = np.ascontiguousarray(np.asarray(enc_cost, dtype=np.float64).reshape(-1))
+    slack = np.ascontiguousarray(np.asarray(warmup_slack, dtype=np.float64).reshape(-1))
+    owner = np.zeros(cost.size, dtype=np.int32)
+    work = np.zeros(slack.size, dtype=np.float64)
+    spill = np.zeros(slack.size, dtype=np.float64)
+    mx = ctypes.c_double()
+    _check(load().mpipe_owner_map(_ptr(cost), cost.size, _ptr(slack), slack.size, _ptr(owner), _ptr(work), _ptr(spill),
+                                  ctypes.addressof(mx)), "mpipe_owner_map")
+    return owner, work, spill, mx.value
 
 
 def selftest_wait_timeout(budget_cycles: int, status_buf, stream=None) -> None:
