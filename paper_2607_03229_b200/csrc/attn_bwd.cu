@@ -18,8 +18,8 @@
 // dQ_i is read back from TMEM by a reducer warpgroup and added to the global fp32 accumulator with
 // vector atomics; dK (x softmax_scale) and dV leave TMEM once per unit.
 //
-// Warp roles (512 threads): 0 TMA producer, 1 tcgen05 issuer, 2 TMEM allocation + LSE staging,
-// 3 Delta staging, 4-7 / 8-11 softmax on query columns 0-63 / 64-127, 12-15 dQ reducer and epilogue.
+// Warp roles (512 threads): 0 TMA producer, 1 / 3 tcgen05 issuers of TMEM stage 0 / 1, 2 TMEM allocation and
+// LSE/Delta staging, 4-7 / 8-11 softmax of stage 0 / 1, 12-15 dQ reducer and epilogue.
 // Every wait is bounded (see sm100_ptx.cuh); expiry sets status_buf and drains the CTA.
 #include <cuda.h>
 #include <math_constants.h>
@@ -72,6 +72,9 @@ struct BwdCfg {
     static constexpr int kSubTail = kTail ? kQS * 32 : 0;
     static constexpr int kSub = kSubMain + kSubTail;
     static constexpr int kRing = 4;                             // Q/dO sub-tile stages
+    // Issuing warps: two (one per TMEM stage) decouple the warpgroups and gain ~10 % at D = 80; at D = 64 a single
+    // in-order issuer measured ~3 % faster (and keeps dK/dV bit-reproducible), so that is what D = 64 uses.
+    static constexpr int kIssuers = (D == 64) ? 1 : 2;
     static constexpr int kKVBufs = (D == 64) ? 2 : 1;           // D = 64: the next unit's K/V tiles load during the current unit
     static constexpr int kStageBytes = kBT * (D * 4);           // dQ staging for the TMA reduction: [128 q][D fp32]
     static constexpr int kStageBufs = 1;
@@ -102,7 +105,7 @@ struct BwdParams {
 };
 
 struct BwdBarriers {
-    uint64_t kv_full[2], kv_empty[2], dkv_full, dkv_empty;
+    uint64_t kv_full[2], kv_empty[2], dkv_full, dkv_empty, acc_v, acc_k;
     uint64_t qdo_full[4], qdo_empty[4], stat_full[4], stat_empty[4];
     uint64_t s_full[2], p_full[2], dp_full[2], ds_full[2], dq_full, dq_empty;
 };
@@ -116,6 +119,7 @@ __global__ void __maxnreg__(kRegsLaunch)
 attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
     using Cfg = BwdCfg<D>;
     constexpr int NR = Cfg::kRing;
+    constexpr int kIssuers = Cfg::kIssuers;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ BwdBarriers bars;
@@ -133,14 +137,16 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         abort_flag = 0;
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars.kv_full[i], 1);
-            mbar_init(&bars.kv_empty[i], 1);
+            mbar_init(&bars.kv_empty[i], kIssuers);   // one commit from each issuing warp
         }
-        mbar_init(&bars.dkv_full, 1);
+        mbar_init(&bars.acc_v, 1);
+        mbar_init(&bars.acc_k, 1);
+        mbar_init(&bars.dkv_full, kIssuers);
         mbar_init(&bars.dkv_empty, 4);
         for (int s = 0; s < 4; ++s) {
             mbar_init(&bars.qdo_full[s], 1);
             mbar_init(&bars.qdo_empty[s], 1);
-            mbar_init(&bars.stat_full[s], 2);
+            mbar_init(&bars.stat_full[s], 1);
             mbar_init(&bars.stat_empty[s], 4);
         }
         for (int b = 0; b < 2; ++b) {
@@ -205,12 +211,20 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ tcgen05 issuer
+    } else if (warp == 1 || (warp == 3 && kIssuers == 2)) {
+        // ------------------------------------------------------------------ tcgen05 issuers
+        // One issuing warp per TMEM stage (warp 1: even sub-tiles, warp 3: odd sub-tiles), so that neither
+        // warpgroup's MMAs wait behind the other's slowest step; a barrier hop costs ~200 cycles (~340 when it
+        // starts from a tcgen05.commit), and a single in-order issuer made every one of them serial.
         // The whole warp walks the loop (uniform control flow); one elected lane issues and commits.
         // Descriptors are precomputed halves: a K-step only adds a constant to the low word.
+        // Cross-warp ordering on the tensor pipe is needed in two places only: the first (overwriting) dV / dK
+        // MMA of a unit comes from stage 0 and must precede stage 1's first accumulation (acc_v / acc_k), and
+        // the pair's dQ MMA (issued by stage 1) needs both stages' dS^T in shared memory (ds_full[0]).
         setmaxnreg_dec<kRegsService>();
         {
+            const int b0 = (kIssuers == 2) ? (warp >> 1) : 0;   // first TMEM stage served by this warp
+            constexpr int kStep = (kIssuers == 2) ? 2 : 1;      // two issuers: every other sub-tile; one: all, in order
             const bool leader = elect_one();
             const uint32_t sbase = smem_u32(smem);
             constexpr uint32_t hi128 = umma_desc_hi(1024, kSwizzle128);
@@ -225,28 +239,28 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             auto q_lo_of = [&](uint32_t c) { return umma_desc_lo(sbase + Cfg::kSmemQ + (c % NR) * Cfg::kSub, 0); };
             auto do_lo_of = [&](uint32_t c) { return umma_desc_lo(sbase + Cfg::kSmemDO + (c % NR) * Cfg::kSub, 0); };
             // dst[128 keys x 64 q] = A[128 x D] * B[64 x D]^T, both K-major (main 64 columns + optional 16 tail)
-            auto issue_kk = [&](uint32_t dcol, uint32_t a, uint32_t at, uint32_t b) {
+            auto issue_kk = [&](uint32_t dcol, uint32_t a, uint32_t at, uint32_t bq) {
                 if (leader) {
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
-                        umma_ss(tmem + dcol, umma_desc(a + ks * 2, hi128), umma_desc(b + ks * 2, hi128), idesc_s, ks > 0);
-                    if (Cfg::kTail) umma_ss(tmem + dcol, umma_desc(at, hi32), umma_desc(b + kSubTailOff, hi32), idesc_s, 1);
+                        umma_ss(tmem + dcol, umma_desc(a + ks * 2, hi128), umma_desc(bq + ks * 2, hi128), idesc_s, ks > 0);
+                    if (Cfg::kTail) umma_ss(tmem + dcol, umma_desc(at, hi32), umma_desc(bq + kSubTailOff, hi32), idesc_s, 1);
                 }
             };
             // dst[128 keys x D] (+)= A^T-in-TMEM[128 keys x 64 q] * B[64 q x D] (B rows = q, MN-major)
-            auto issue_ts = [&](uint32_t dcol, uint32_t acol, uint32_t b, bool acc) {
+            auto issue_ts = [&](uint32_t dcol, uint32_t acol, uint32_t bq, bool acc) {
                 if (leader) {
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
-                        umma_ts(tmem + dcol, tmem + acol + ks * 8, umma_desc(b + ks * 128, hi128), idesc_ts,
+                        umma_ts(tmem + dcol, tmem + acol + ks * 8, umma_desc(bq + ks * 128, hi128), idesc_ts,
                                 (acc || ks > 0) ? 1u : 0u);
                         if (Cfg::kTail)
-                            umma_ts(tmem + dcol + 64, tmem + acol + ks * 8, umma_desc(b + kSubTailOff + ks * 32, hi32),
+                            umma_ts(tmem + dcol + 64, tmem + acol + ks * 8, umma_desc(bq + kSubTailOff + ks * 32, hi32),
                                     idesc_ts_t, (acc || ks > 0) ? 1u : 0u);
                     }
                 }
             };
-            uint32_t unit_it = 0, sc = 0;
+            uint32_t unit_it = 0, sc = 0;   // sc: global sub-tile counter at the start of the unit (even)
             bool ok = true;
             for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
                 const mpipe_work_item_t it = p.items[u / p.n_heads];
@@ -258,52 +272,74 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 const uint32_t vt_lo = umma_desc_lo(kvb + Cfg::kSmemV + Cfg::kTileMain, 0);
                 ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.kv_full[kb], (unit_it / Cfg::kKVBufs) & 1, &abort_flag);
                 if (!ok) break;
-                for (int s = 0; s < 2; ++s) {   // prologue: S^T and dP^T of the first two sub-tiles
-                    ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[(sc + s) % NR], ((sc + s) / NR) & 1, &abort_flag);
+                for (int s = b0; s < 2; s += kStep) {   // prologue: S^T and dP^T of the first sub-tile of each stage served
+                    const uint32_t c = sc + s;
+                    ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[c % NR], (c / NR) & 1, &abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_kk(Cfg::kColS + 64 * s, k_lo, kt_lo, q_lo_of(sc + s));
+                    issue_kk(Cfg::kColS + 64 * s, k_lo, kt_lo, q_lo_of(c));
                     if (leader) umma_commit(&bars.s_full[s]);
-                    issue_kk(Cfg::kColDP + 64 * s, v_lo, vt_lo, do_lo_of(sc + s));
+                    issue_kk(Cfg::kColDP + 64 * s, v_lo, vt_lo, do_lo_of(c));
                     if (leader) umma_commit(&bars.dp_full[s]);
                 }
                 if (!ok) break;
-                for (int s = 0; s < n2; ++s, ++sc) {
+                for (int s = b0; s < n2; s += kStep) {
                     const int b = s & 1;
-                    const uint32_t ph = (sc >> 1) & 1;   // phase of the per-stage barriers
+                    const uint32_t c = sc + s;
+                    const uint32_t ph = (c >> 1) & 1;   // phase of the per-stage barriers
                     const bool more = (s + 2 < n2);
-                    if (s == 0) {
-                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag);
-                        if (!ok) break;
-                    }
-                    MPIPE_TR(0, sc * 8 + 0);
+                    const bool first = (s < 2);         // the stage's first sub-tile of the unit
+                    MPIPE_TR(0, c * 8 + 0);
                     ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.p_full[b], ph, &abort_flag);
                     if (!ok) break;
-                    MPIPE_TR(0, sc * 8 + 1);
+                    if (first && b == 0) {          // the accumulators are free: the previous unit's epilogue has read them
+                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag);
+                        if (!ok) break;
+                    } else if (first && kIssuers == 2) {   // ... and stage 0's overwriting dV MMA has been issued
+                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.acc_v, unit_it & 1, &abort_flag);
+                        if (!ok) break;
+                    }
+                    MPIPE_TR(0, c * 8 + 1);
                     tc_fence_after();
-                    issue_ts(Cfg::kColDV, Cfg::kColS + 64 * b, do_lo_of(sc), s > 0);          // dV += P^T dO
+                    issue_ts(Cfg::kColDV, Cfg::kColS + 64 * b, do_lo_of(c), !(first && b == 0));         // dV += P^T dO
+                    if (first && b == 0 && kIssuers == 2) {
+                        tc_fence_before();
+                        if (leader) mbar_arrive(&bars.acc_v);
+                    }
                     if (more) {
-                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[(sc + 2) % NR], ((sc + 2) / NR) & 1, &abort_flag);
+                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[(c + 2) % NR], ((c + 2) / NR) & 1, &abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        issue_kk(Cfg::kColS + 64 * b, k_lo, kt_lo, q_lo_of(sc + 2));          // S^T(s+2)
+                        issue_kk(Cfg::kColS + 64 * b, k_lo, kt_lo, q_lo_of(c + 2));                       // S^T(s+2)
                         if (leader) umma_commit(&bars.s_full[b]);
                     }
-                    MPIPE_TR(0, sc * 8 + 2);
+                    MPIPE_TR(0, c * 8 + 2);
                     ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.ds_full[b], ph, &abort_flag);
                     if (!ok) break;
-                    MPIPE_TR(0, sc * 8 + 3);
+                    if (first && b == 1 && kIssuers == 2) {
+                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.acc_k, unit_it & 1, &abort_flag);
+                        if (!ok) break;
+                    }
+                    MPIPE_TR(0, c * 8 + 3);
                     tc_fence_after();
-                    issue_ts(Cfg::kColDK, Cfg::kColDP + 64 * b, q_lo_of(sc), s > 0);          // dK += dS^T Q
-                    if (leader) umma_commit(&bars.qdo_empty[sc % NR]);
+                    issue_ts(Cfg::kColDK, Cfg::kColDP + 64 * b, q_lo_of(c), !(first && b == 0));          // dK += dS^T Q
+                    if (first && b == 0 && kIssuers == 2) {
+                        tc_fence_before();
+                        if (leader) mbar_arrive(&bars.acc_k);
+                    }
+                    if (leader) umma_commit(&bars.qdo_empty[c % NR]);
                     if (more) {
-                        issue_kk(Cfg::kColDP + 64 * b, v_lo, vt_lo, do_lo_of(sc + 2));        // dP^T(s+2)
+                        issue_kk(Cfg::kColDP + 64 * b, v_lo, vt_lo, do_lo_of(c + 2));                     // dP^T(s+2)
                         if (leader) umma_commit(&bars.dp_full[b]);
                     }
                     if (b == 1) {                                                             // dQ of the 128-query pair
-                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.dq_empty, ((sc >> 1) & 1) ^ 1, &abort_flag);
+                        if (kIssuers == 2) {   // the other half of dS^T (a single issuer has already waited for it)
+                            ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.ds_full[0], ph, &abort_flag);
+                            if (!ok) break;
+                        }
+                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.dq_empty, ((c >> 1) & 1) ^ 1, &abort_flag);
                         if (!ok) break;
-                        MPIPE_TR(0, sc * 8 + 4);
+                        MPIPE_TR(0, c * 8 + 4);
                         tc_fence_after();
                         if (leader) {
 #pragma unroll
@@ -316,19 +352,18 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                             umma_commit(&bars.dq_full);
                         }
                     }
-                    MPIPE_TR(0, sc * 8 + 5);
+                    MPIPE_TR(0, c * 8 + 5);
                 }
                 if (!ok) break;
                 if (leader) umma_commit(&bars.dkv_full);
                 if (leader) umma_commit(&bars.kv_empty[kb]);
+                sc += n2;
             }
         }
         __syncwarp();
-    } else if (warp < 4) {
-        // ------------------------------------------------------------------ LSE (warp 2) / Delta (warp 3) staging
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ LSE / Delta staging
         setmaxnreg_dec<kRegsService>();
-        const bool is_lse = (warp == 2);
-        const float* src = is_lse ? p.lse : p.delta;
         uint32_t sc = 0;
         bool ok = true;
         for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
@@ -340,25 +375,28 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 const int rs = sc % NR;
                 ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.stat_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
                 if (!ok) break;
-                float* dst = reinterpret_cast<float*>(smem + Cfg::kSmemStat + rs * (2 * kQS * 4)) + (is_lse ? 0 : kQS);
+                float* dst = reinterpret_cast<float*>(smem + Cfg::kSmemStat + rs * (2 * kQS * 4));
                 const int q0 = it.kv_start + s * kQS;
 #pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int c = lane + 32 * e;
+                for (int e = 0; e < 4; ++e) {   // e = 0, 1: -LSE*log2e of 64 query columns; e = 2, 3: -Delta
+                    const bool is_lse = (e < 2);
+                    const int c = lane + 32 * (e & 1);
                     const int q = q0 + c;
-                    float val;   // stored negated: -LSE*log2e and -Delta are what the softmax warps add
+                    float val;   // stored negated: what the softmax warps add
                     if (q < q_end) {
-                        val = -__ldg(src + int64_t(head) * p.total_tokens + q);
+                        val = -__ldg((is_lse ? p.lse : p.delta) + int64_t(head) * p.total_tokens + q);
                         if (is_lse) val *= 1.4426950408889634f;
                     } else {
                         val = is_lse ? -CUDART_INF_F : 0.f;  // P = exp2(-inf) = 0 for query columns past the segment
                     }
-                    dst[c] = val;
+                    dst[(is_lse ? 0 : kQS) + c] = val;
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars.stat_full[rs]);
             }
         }
+    } else if (warp == 3) {
+        setmaxnreg_dec<kRegsService>();   // spare warp when one issuer is enough
     } else if (warp < 12) {
         // ------------------------------------------------------------------ softmax / dS warps
         // Warpgroup g owns TMEM stage g, i.e. every other 64-query sub-tile; thread = key row.
