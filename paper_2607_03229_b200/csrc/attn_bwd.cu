@@ -168,6 +168,12 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
     const int n_units = p.n_items * p.n_heads;
+    // Units are sorted by decreasing cost; CTAs walk them in boustrophedon order (0..G-1, then G-1..0, ...) so
+    // that the CTA that got the most expensive unit of one round gets the cheapest of the next.
+    auto unit_of = [&](int round) {
+        const int g = int(gridDim.x), i = int(blockIdx.x);
+        return round * g + ((round & 1) ? g - 1 - i : i);
+    };
     // Every unit runs an even number of 64-query sub-tiles (a 128-query tile is two of them); a padding
     // sub-tile past the segment end contributes nothing because its probabilities are forced to zero.
     auto subtiles_of = [](const mpipe_work_item_t& it) { return 2 * ((it.kv_len + kBT - 1) / kBT); };
@@ -178,7 +184,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         if (lane == 0) {
             uint32_t unit_it = 0, sc = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
+            for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
                 const mpipe_work_item_t it = p.items[u / p.n_heads];
                 const int head = u % p.n_heads;
                 const int n2 = subtiles_of(it);
@@ -262,7 +268,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             };
             uint32_t unit_it = 0, sc = 0;   // sc: global sub-tile counter at the start of the unit (even)
             bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
+            for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
                 const mpipe_work_item_t it = p.items[u / p.n_heads];
                 const int n2 = subtiles_of(it);
                 const int kb = unit_it % Cfg::kKVBufs;
@@ -366,7 +372,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         setmaxnreg_dec<kRegsService>();
         uint32_t sc = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
             const mpipe_work_item_t it = p.items[u / p.n_heads];
             const int head = u % p.n_heads;
             const int n2 = subtiles_of(it);
@@ -409,7 +415,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         uint8_t* ds_row = smem + Cfg::kSmemDS + g * (kBT * 128) + r * 128;
         uint32_t sc = 0;   // global sub-tile counter at the start of the unit (always even)
         bool ok = true;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
             const mpipe_work_item_t it = p.items[u / p.n_heads];
             const int n2 = subtiles_of(it);
             const bool key_valid = r < it.row_len;
@@ -531,7 +537,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
         uint32_t pc = 0, unit_it = 0;   // pair counter
         bool ok = true;
-        for (int u = blockIdx.x; u < n_units; u += gridDim.x, ++unit_it) {
+        for (int ur = 0, u = unit_of(0); u < n_units; ++ur, u = unit_of(ur), ++unit_it) {
             const mpipe_work_item_t it = p.items[u / p.n_heads];
             const int head = u % p.n_heads;
             const int npairs = (it.kv_len + kBT - 1) / kBT;

@@ -118,6 +118,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const uint32_t tmem = tmem_base_slot;
     // TMEM columns: S_0 [0,128), S_1 [128,256), O_0 [256,256+D), O_1 [384,384+D); P_w overlays S_w.
     const int n_units = p.n_items * p.n_heads;
+    // Units are sorted by decreasing cost; CTAs walk them in boustrophedon order (0..G-1, then G-1..0, ...) so
+    // that the CTA that got the most expensive unit of one round gets the cheapest of the next.
+    auto unit_of = [&](int round) {
+        const int g = int(gridDim.x), i = int(blockIdx.x);
+        return round * g + ((round & 1) ? g - 1 - i : i);
+    };
 
     if (warp == 0) {
         setmaxnreg_dec<kFwdRegsLight>();
@@ -125,7 +131,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (lane == 0) {
             uint32_t kv_it = 0, unit_it = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
+            for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
                 const mpipe_work_item_t it = p.items[u / p.n_heads];
                 const int head = u % p.n_heads;
                 const bool two = it.row_len > kTileM;
@@ -203,7 +209,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     }
                 }
             };
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++unit_it) {
+            for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
                 const mpipe_work_item_t it = p.items[u / p.n_heads];
                 const bool two = it.row_len > kTileM;
                 const int nkv = (it.kv_len + kTileN - 1) / kTileN;
@@ -283,7 +289,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const uint32_t t_o = tmem + lane_base + 256 + w * 128;
         uint32_t cnt = 0, ocnt = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
             const mpipe_work_item_t it = p.items[u / p.n_heads];
             const int head = u % p.n_heads;
             const int rows_here = it.row_len - w * kTileM;  // valid rows of this tile
