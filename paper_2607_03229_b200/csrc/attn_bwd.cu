@@ -39,13 +39,19 @@ __device__ int g_dbg_flags;   // knock-out switches for experiments: 1 no atomic
     do {                                                                                     \
         if (blockIdx.x == 0 && (idx) < 4096) g_trace[role][(idx)] = clock64();               \
     } while (0)
+__device__ int g_where[16];
+#define MW(call) ((blockIdx.x == (g_dbg_flags >> 16) && (threadIdx.x & 31) == 0 ? (void)(g_where[threadIdx.x >> 5] = __LINE__) : (void)0), call)
 #else
+#define MW(call) call
 #define MPIPE_DBG(bit) false
 #define MPIPE_TR(role, idx) \
     do {                    \
     } while (0)
 #endif
 
+#ifndef MPIPE_STREAM
+#define MPIPE_STREAM 1
+#endif
 #ifndef MPIPE_SLEEP_AUX
 #define MPIPE_SLEEP_AUX 100
 #endif
@@ -76,16 +82,19 @@ struct BwdCfg {
     // in-order issuer measured ~3 % faster (and keeps dK/dV bit-reproducible), so that is what D = 64 uses.
     static constexpr int kIssuers = (D == 64) ? 1 : 2;
     static constexpr int kKVBufs = (D == 64) ? 2 : 1;           // D = 64: the next unit's K/V tiles load during the current unit
-    static constexpr int kStageBytes = kBT * (D * 4);           // dQ staging for the TMA reduction: [128 q][D fp32]
-    static constexpr int kStageBufs = 1;
+    static constexpr int kStatRing = 8;                         // LSE / Delta stages (written well ahead of their use)
+    // dQ staging for the TMA reduction: one [128 q][32 fp32] box (used twice per pair) + the 16-column tail box
+    static constexpr int kStageMain = kBT * 128;
+    static constexpr int kStageBytes = kStageMain + (kTail ? kBT * 64 : 0);
     static constexpr int kSmemK = 0;                            // buffer i at kSmemK + i * 2 * kTile (K then V)
     static constexpr int kSmemV = kTile;
     static constexpr int kSmemQ = kKVBufs * 2 * kTile;
     static constexpr int kSmemDO = kSmemQ + kRing * kSub;
-    static constexpr int kSmemDS = kSmemDO + kRing * kSub;      // dS^T as [key][q]: two 64-query atoms of 16 KB
-    static constexpr int kSmemStage = kSmemDS + 2 * kBT * 128;  // two staging buffers
-    static constexpr int kSmemStat = kSmemStage + kStageBufs * kStageBytes;   // kRing x (LSE[64], Delta[64]) fp32
-    static constexpr int kSmemTotal = kSmemStat + kRing * 2 * kQS * 4;
+    static constexpr int kDSBytes = 2 * kBT * 128;              // dS^T of a pair as [key][q]: two 64-query atoms of 16 KB
+    static constexpr int kSmemDS = kSmemDO + kRing * kSub;      // two of them: pair j writes buffer j & 1 while dQ(j-1) reads the other
+    static constexpr int kSmemStage = kSmemDS + 2 * kDSBytes;
+    static constexpr int kSmemStat = kSmemStage + kStageBytes;  // kStatRing x (LSE[64], Delta[64]) fp32
+    static constexpr int kSmemTotal = kSmemStat + kStatRing * 2 * kQS * 4;
     static constexpr int kSmemAlloc = kSmemTotal + 1024;
     // TMEM columns: S^T stage b at 64*b, dP^T stage b at 128 + 64*b (P^T / dS^T overlay their first 32 columns)
     static constexpr int kColS = 0, kColDP = 128, kColDV = 256, kColDK = 256 + D, kColDQ = 256 + 2 * D;
@@ -106,8 +115,8 @@ struct BwdParams {
 
 struct BwdBarriers {
     uint64_t kv_full[2], kv_empty[2], dkv_full, dkv_empty, acc_v, acc_k;
-    uint64_t qdo_full[4], qdo_empty[4], stat_full[4], stat_empty[4];
-    uint64_t s_full[2], p_full[2], dp_full[2], ds_full[2], dq_full, dq_empty;
+    uint64_t qdo_full[4], qdo_empty[4], stat_full[8], stat_empty[8];
+    uint64_t s_full[2], p_full[2], dp_full[2], ds_full[2], dq_full[2], dq_empty, ds0_seen;
 };
 
 struct BwdMaps {
@@ -119,6 +128,7 @@ __global__ void __maxnreg__(kRegsLaunch)
 attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
     using Cfg = BwdCfg<D>;
     constexpr int NR = Cfg::kRing;
+    constexpr int NS = Cfg::kStatRing;
     constexpr int kIssuers = Cfg::kIssuers;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -146,8 +156,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         for (int s = 0; s < 4; ++s) {
             mbar_init(&bars.qdo_full[s], 1);
             mbar_init(&bars.qdo_empty[s], 1);
+        }
+        for (int s = 0; s < 8; ++s) {
             mbar_init(&bars.stat_full[s], 1);
-            mbar_init(&bars.stat_empty[s], 4);
+            mbar_init(&bars.stat_empty[s], 1);   // released by the issuing warp once the sub-tile's dS^T has arrived
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&bars.s_full[b], 1);
@@ -155,7 +167,9 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             mbar_init(&bars.dp_full[b], 1);
             mbar_init(&bars.ds_full[b], 4);
         }
-        mbar_init(&bars.dq_full, 1);
+        mbar_init(&bars.ds0_seen, 1);
+        mbar_init(&bars.dq_full[0], 1);
+        mbar_init(&bars.dq_full[1], 1);
         mbar_init(&bars.dq_empty, 4);
         fence_mbar_init();
     }
@@ -190,7 +204,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 const int n2 = subtiles_of(it);
                 const int kb = unit_it % Cfg::kKVBufs;            // K/V buffer of this unit
                 uint8_t* kv = smem + kb * (2 * Cfg::kTile);
-                ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.kv_empty[kb], ((unit_it / Cfg::kKVBufs) & 1) ^ 1, &abort_flag);
+                ok = MW(mbar_wait<MPIPE_SLEEP_AUX>(&bars.kv_empty[kb], ((unit_it / Cfg::kKVBufs) & 1) ^ 1, &abort_flag));
                 if (!ok) break;
                 mbar_expect_tx(&bars.kv_full[kb], 2 * Cfg::kTile);
                 tma_load_3d(kv + Cfg::kSmemK, &maps.k, &bars.kv_full[kb], 0, head, it.row_start);
@@ -202,7 +216,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 for (int s = 0; s < n2; ++s, ++sc) {
                     const int rs = sc % NR;
                     const int row = it.kv_start + s * kQS;
-                    ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.qdo_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
+                    ok = MW(mbar_wait<MPIPE_SLEEP_AUX>(&bars.qdo_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag));
                     if (!ok) break;
                     mbar_expect_tx(&bars.qdo_full[rs], 2 * Cfg::kSub);
                     uint8_t* qd = smem + Cfg::kSmemQ + rs * Cfg::kSub;
@@ -236,6 +250,9 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             constexpr uint32_t hi128 = umma_desc_hi(1024, kSwizzle128);
             constexpr uint32_t hi32 = umma_desc_hi(256, kSwizzle32);
             const uint32_t ds_lo = umma_desc_lo(sbase + Cfg::kSmemDS, kBT * 128);   // two 64-query atoms 16 KB apart
+            // LSE / Delta of a sub-tile must be staged before its S^T is issued: the softmax warps then need no
+            // barrier of their own for them (S^T complete implies staged)
+            auto wait_stat = [&](uint32_t c) { return MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.stat_full[c % NS], (c / NS) & 1, &abort_flag)); };
             constexpr uint32_t idesc_s = umma_idesc_bf16(kBT, kQS, 0, 0);      // K-major x K-major, N = 64 queries
             constexpr uint32_t idesc_ts = umma_idesc_bf16(kBT, 64, 0, 1);      // A in TMEM, MN-major B, N = 64
             constexpr uint32_t idesc_ts_t = umma_idesc_bf16(kBT, 16, 0, 1);    // same, 16-wide head-dim tail
@@ -276,33 +293,45 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 const uint32_t k_lo = umma_desc_lo(kvb + Cfg::kSmemK, 0), v_lo = umma_desc_lo(kvb + Cfg::kSmemV, 0);
                 const uint32_t kt_lo = umma_desc_lo(kvb + Cfg::kSmemK + Cfg::kTileMain, 0);
                 const uint32_t vt_lo = umma_desc_lo(kvb + Cfg::kSmemV + Cfg::kTileMain, 0);
-                ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.kv_full[kb], (unit_it / Cfg::kKVBufs) & 1, &abort_flag);
+                // With two K/V buffers the stream of sub-tiles runs on across the unit boundary: the S^T / dP^T MMAs
+                // of the next unit's first two sub-tiles are issued inside this unit's last two iterations, from
+                // the other (prefetched) buffer, so the softmax warps never see the pipeline drain between units.
+                constexpr bool kStream = (Cfg::kKVBufs == 2) && MPIPE_STREAM;
+                const bool has_next = kStream && unit_of(ur + 1) < n_units;
+                const uint32_t kvb_n = sbase + (kb ^ 1) * (2 * Cfg::kTile);
+                const uint32_t k_lo_n = umma_desc_lo(kvb_n + Cfg::kSmemK, 0), v_lo_n = umma_desc_lo(kvb_n + Cfg::kSmemV, 0);
+                ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.kv_full[kb], (unit_it / Cfg::kKVBufs) & 1, &abort_flag));
                 if (!ok) break;
-                for (int s = b0; s < 2; s += kStep) {   // prologue: S^T and dP^T of the first sub-tile of each stage served
-                    const uint32_t c = sc + s;
-                    ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[c % NR], (c / NR) & 1, &abort_flag);
+                if (!kStream || unit_it == 0) {
+                    for (int s = b0; s < 2; s += kStep) {   // prologue: S^T and dP^T of the first sub-tile of each stage served
+                        const uint32_t c = sc + s;
+                        ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[c % NR], (c / NR) & 1, &abort_flag));
+                        if (!ok) break;
+                        ok = wait_stat(c);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_kk(Cfg::kColS + 64 * s, k_lo, kt_lo, q_lo_of(c));
+                        if (leader) umma_commit(&bars.s_full[s]);
+                        issue_kk(Cfg::kColDP + 64 * s, v_lo, vt_lo, do_lo_of(c));
+                        if (leader) umma_commit(&bars.dp_full[s]);
+                    }
                     if (!ok) break;
-                    tc_fence_after();
-                    issue_kk(Cfg::kColS + 64 * s, k_lo, kt_lo, q_lo_of(c));
-                    if (leader) umma_commit(&bars.s_full[s]);
-                    issue_kk(Cfg::kColDP + 64 * s, v_lo, vt_lo, do_lo_of(c));
-                    if (leader) umma_commit(&bars.dp_full[s]);
                 }
-                if (!ok) break;
                 for (int s = b0; s < n2; s += kStep) {
                     const int b = s & 1;
                     const uint32_t c = sc + s;
                     const uint32_t ph = (c >> 1) & 1;   // phase of the per-stage barriers
-                    const bool more = (s + 2 < n2);
+                    const bool cross = (s + 2 >= n2) && has_next;   // sub-tile s+2 is the next unit's
+                    const bool more = (s + 2 < n2) || cross;
                     const bool first = (s < 2);         // the stage's first sub-tile of the unit
                     MPIPE_TR(0, c * 8 + 0);
-                    ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.p_full[b], ph, &abort_flag);
+                    ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.p_full[b], ph, &abort_flag));
                     if (!ok) break;
                     if (first && b == 0) {          // the accumulators are free: the previous unit's epilogue has read them
-                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag);
+                        ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag));
                         if (!ok) break;
                     } else if (first && kIssuers == 2) {   // ... and stage 0's overwriting dV MMA has been issued
-                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.acc_v, unit_it & 1, &abort_flag);
+                        ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.acc_v, unit_it & 1, &abort_flag));
                         if (!ok) break;
                     }
                     MPIPE_TR(0, c * 8 + 1);
@@ -313,17 +342,23 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                         if (leader) mbar_arrive(&bars.acc_v);
                     }
                     if (more) {
-                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[(c + 2) % NR], ((c + 2) / NR) & 1, &abort_flag);
+                        if (cross && b == 0) {   // the next unit's K/V tiles (loaded while this unit ran)
+                            ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.kv_full[kb ^ 1], ((unit_it + 1) / Cfg::kKVBufs) & 1, &abort_flag));
+                            if (!ok) break;
+                        }
+                        ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[(c + 2) % NR], ((c + 2) / NR) & 1, &abort_flag));
+                        if (!ok) break;
+                        ok = wait_stat(c + 2);
                         if (!ok) break;
                         tc_fence_after();
-                        issue_kk(Cfg::kColS + 64 * b, k_lo, kt_lo, q_lo_of(c + 2));                       // S^T(s+2)
+                        issue_kk(Cfg::kColS + 64 * b, cross ? k_lo_n : k_lo, kt_lo, q_lo_of(c + 2));       // S^T(s+2)
                         if (leader) umma_commit(&bars.s_full[b]);
                     }
                     MPIPE_TR(0, c * 8 + 2);
-                    ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.ds_full[b], ph, &abort_flag);
+                    ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.ds_full[b], ph, &abort_flag));
                     if (!ok) break;
                     if (first && b == 1 && kIssuers == 2) {
-                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.acc_k, unit_it & 1, &abort_flag);
+                        ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.acc_k, unit_it & 1, &abort_flag));
                         if (!ok) break;
                     }
                     MPIPE_TR(0, c * 8 + 3);
@@ -333,29 +368,33 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                         tc_fence_before();
                         if (leader) mbar_arrive(&bars.acc_k);
                     }
-                    if (leader) umma_commit(&bars.qdo_empty[c % NR]);
+                    if (leader) {
+                        umma_commit(&bars.qdo_empty[c % NR]);
+                        mbar_arrive(&bars.stat_empty[c % NS]);   // dS^T(c) has arrived: its LSE / Delta stage has been read
+                    }
                     if (more) {
-                        issue_kk(Cfg::kColDP + 64 * b, v_lo, vt_lo, do_lo_of(c + 2));                     // dP^T(s+2)
+                        issue_kk(Cfg::kColDP + 64 * b, cross ? v_lo_n : v_lo, vt_lo, do_lo_of(c + 2));    // dP^T(s+2)
                         if (leader) umma_commit(&bars.dp_full[b]);
                     }
                     if (b == 1) {                                                             // dQ of the 128-query pair
                         if (kIssuers == 2) {   // the other half of dS^T (a single issuer has already waited for it)
-                            ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.ds_full[0], ph, &abort_flag);
+                            ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.ds_full[0], ph, &abort_flag));
                             if (!ok) break;
+                            if (leader) mbar_arrive(&bars.ds0_seen);   // lets stage 0's warpgroup complete the next phase
                         }
-                        ok = mbar_wait<MPIPE_SLEEP_MMA>(&bars.dq_empty, ((c >> 1) & 1) ^ 1, &abort_flag);
+                        ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.dq_empty, ((c >> 1) & 1) ^ 1, &abort_flag));
                         if (!ok) break;
                         MPIPE_TR(0, c * 8 + 4);
                         tc_fence_after();
                         if (leader) {
 #pragma unroll
                             for (int ks = 0; ks < 8; ++ks) {
-                                const uint64_t adesc = umma_desc(ds_lo + ks * 128, hi128);
+                                const uint64_t adesc = umma_desc(ds_lo + ph * (Cfg::kDSBytes >> 4) + ks * 128, hi128);
                                 umma_ss(tmem + Cfg::kColDQ, adesc, umma_desc(k_lo + ks * 128, hi128), idesc_dq, ks > 0);
                                 if (Cfg::kTail)
                                     umma_ss(tmem + Cfg::kColDQ + 64, adesc, umma_desc(kt_lo + ks * 32, hi32), idesc_dq_t, ks > 0);
                             }
-                            umma_commit(&bars.dq_full);
+                            umma_commit(&bars.dq_full[ph]);
                         }
                     }
                     MPIPE_TR(0, c * 8 + 5);
@@ -378,8 +417,8 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             const int n2 = subtiles_of(it);
             const int q_end = it.kv_start + it.kv_len;
             for (int s = 0; s < n2; ++s, ++sc) {
-                const int rs = sc % NR;
-                ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.stat_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
+                const int rs = sc % NS;
+                ok = MW(mbar_wait<MPIPE_SLEEP_AUX>(&bars.stat_empty[rs], ((sc / NS) & 1) ^ 1, &abort_flag));
                 if (!ok) break;
                 float* dst = reinterpret_cast<float*>(smem + Cfg::kSmemStat + rs * (2 * kQS * 4));
                 const int q0 = it.kv_start + s * kQS;
@@ -422,15 +461,14 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             const bool ragged_keys = it.row_len < kBT;
             for (int s = g; s < n2; s += 2) {
                 const uint32_t c = sc + s;
-                const int rs = c % NR;
-                const uint32_t ph = (c >> 1) & 1;
+                const int rs = c % NS;
+                const uint32_t ph = (c >> 1) & 1;   // phase of the per-stage barriers = dS^T buffer of the pair
                 const float* stat = reinterpret_cast<const float*>(smem + Cfg::kSmemStat + rs * (2 * kQS * 4));
                 const float4* lse4 = reinterpret_cast<const float4*>(stat);
                 const float4* dl4 = reinterpret_cast<const float4*>(stat + kQS);
-                ok = mbar_wait(&bars.stat_full[rs], (c / NR) & 1, &abort_flag);
-                if (!ok) break;
                 if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 0);
-                ok = mbar_wait(&bars.s_full[g], ph, &abort_flag);
+                // (the LSE / Delta stage was complete before this S^T was issued)
+                ok = MW(mbar_wait(&bars.s_full[g], ph, &abort_flag));
                 if (!ok) break;
                 if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 1);
                 tc_fence_after();
@@ -471,11 +509,12 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 if (lane == 0) mbar_arrive(&bars.p_full[g]);
                 if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 2);
 
-                ok = mbar_wait(&bars.dp_full[g], ph, &abort_flag);
+                ok = MW(mbar_wait(&bars.dp_full[g], ph, &abort_flag));
                 if (!ok) break;
-                // the dS^T tile in shared memory is free once the previous pair's dQ MMA has completed
-                if ((c >> 1) > 0) {
-                    ok = mbar_wait(&bars.dq_full, ((c >> 1) - 1) & 1, &abort_flag);
+                // dS^T buffer (pair & 1) is free once dQ of pair - 2 has completed. With one issuing warp that is implied
+                // by s_full above (S^T(c) was issued, in order, after that dQ); with two it is waited for.
+                if (kIssuers == 2 && (c >> 1) >= 2) {
+                    ok = MW(mbar_wait(&bars.dq_full[ph], ((c >> 2) + 1) & 1, &abort_flag));
                     if (!ok) break;
                 }
                 if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 3);
@@ -511,7 +550,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     // the same 64 values as 8 x 16 bytes of row r of the [key][q] tile (128-byte swizzle)
 #pragma unroll
                     for (int chunk = 0; chunk < 8; ++chunk) {
-                        if (!MPIPE_DBG(2)) *reinterpret_cast<uint4*>(ds_row + ((chunk ^ (r & 7)) << 4)) =
+                        if (!MPIPE_DBG(2)) *reinterpret_cast<uint4*>(ds_row + ph * Cfg::kDSBytes + ((chunk ^ (r & 7)) << 4)) =
                             make_uint4(pk[4 * chunk], pk[4 * chunk + 1], pk[4 * chunk + 2], pk[4 * chunk + 3]);
                     }
                 }
@@ -519,10 +558,13 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 fence_async_smem();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(&bars.ds_full[g]);
-                    mbar_arrive(&bars.stat_empty[rs]);
+                // With two issuing warps ds_full[0] has two consumers; the second (stage 1's issuer, before dQ) can lag, and
+                // a parity wait cannot tell phase n from n + 2: do not complete a phase before it has seen the last one.
+                if (kIssuers == 2 && g == 0 && (c >> 1) >= 1) {
+                    ok = MW(mbar_wait(&bars.ds0_seen, ((c >> 1) - 1) & 1, &abort_flag));
+                    if (!ok) break;
                 }
+                if (lane == 0) mbar_arrive(&bars.ds_full[g]);
                 if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 4);
             }
             sc += n2;
@@ -545,49 +587,69 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             // they keep walking the (now empty) iterations together instead of leaving one another behind.
             for (int i = 0; i < npairs; ++i, ++pc) {
                 if (lane == 0 && warp == 12) MPIPE_TR(3, pc * 8 + 0);
-                if (ok) ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.dq_full, pc & 1, &abort_flag);
+                if (ok) ok = MW(mbar_wait<MPIPE_SLEEP_AUX>(&bars.dq_full[pc & 1], (pc >> 1) & 1, &abort_flag));
                 if (lane == 0 && warp == 12) MPIPE_TR(3, pc * 8 + 1);
                 tc_fence_after();
-                uint8_t* stage = smem + Cfg::kSmemStage + (pc % Cfg::kStageBufs) * Cfg::kStageBytes;
-                // the staging buffer must have been read by the copy engine before it is overwritten
-                if (rt == 0) bulk_wait_group_read<Cfg::kStageBufs - 1>();
+                uint8_t* stage = smem + Cfg::kSmemStage;
+                const int q0 = it.kv_start + i * kBT;
+                // Two steps through one [128 rows][128 B] staging box (128-byte swizzle): columns 0..31, then 32..63; the
+                // D = 80 tail (columns 64..79, [128 rows][64 B], 64-byte swizzle) rides with the first step. The second
+                // half leaves TMEM before the first is handed to the copy engine, so the next pair's dQ MMA can start.
+                if (rt == 0) bulk_wait_group_read<0>();   // the box must have been read before it is overwritten
                 named_barrier_sync(1, 128);
+                uint32_t v1[2][16];
                 if (ok) {
+                    uint32_t v0[2][16];
+                    tmem_ld16(tmem + lane_base + Cfg::kColDQ, v0[0]);
+                    tmem_ld16(tmem + lane_base + Cfg::kColDQ + 16, v0[1]);
+                    tmem_wait_ld();
 #pragma unroll
-                    for (int c0 = 0; c0 < D; c0 += 16) {
-                        uint32_t v[16];
-                        tmem_ld16(tmem + lane_base + Cfg::kColDQ + c0, v);
+                    for (int chunk = 0; chunk < 8; ++chunk)
+                        *reinterpret_cast<uint4*>(stage + r * 128 + ((chunk ^ (r & 7)) << 4)) =
+                            make_uint4(v0[chunk / 4][4 * (chunk & 3)], v0[chunk / 4][4 * (chunk & 3) + 1],
+                                       v0[chunk / 4][4 * (chunk & 3) + 2], v0[chunk / 4][4 * (chunk & 3) + 3]);
+                    tmem_ld16(tmem + lane_base + Cfg::kColDQ + 32, v1[0]);
+                    tmem_ld16(tmem + lane_base + Cfg::kColDQ + 48, v1[1]);
+                    if (Cfg::kTail) {
+                        uint32_t vt[16];
+                        tmem_ld16(tmem + lane_base + Cfg::kColDQ + 64, vt);
                         tmem_wait_ld();
-                        if (c0 + 16 >= D) {  // last read of this row issued and complete: release dQ in TMEM
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(&bars.dq_empty);
-                        }
-                        // box j = columns [32j, 32j+32): [128 rows][128 B], 128-byte swizzle; the D=80 tail box
-                        // (columns 64..79) is [128 rows][64 B] with 64-byte swizzle
-                        const int box = c0 >> 5;
-                        uint8_t* brow = stage + box * (kBT * 128);
 #pragma unroll
-                        for (int cc = 0; cc < 4; ++cc) {
-                            const int chunk = ((c0 & 31) >> 2) + cc;   // 16-byte chunk inside the box row
-                            uint8_t* dst = (box < 2) ? brow + r * 128 + ((chunk ^ (r & 7)) << 4)
-                                                     : brow + r * 64 + ((chunk ^ ((r >> 1) & 3)) << 4);
-                            *reinterpret_cast<uint4*>(dst) = make_uint4(v[4 * cc], v[4 * cc + 1], v[4 * cc + 2], v[4 * cc + 3]);
-                        }
+                        for (int chunk = 0; chunk < 4; ++chunk)
+                            *reinterpret_cast<uint4*>(stage + Cfg::kStageMain + r * 64 + ((chunk ^ ((r >> 1) & 3)) << 4)) =
+                                make_uint4(vt[4 * chunk], vt[4 * chunk + 1], vt[4 * chunk + 2], vt[4 * chunk + 3]);
+                    } else {
+                        tmem_wait_ld();
                     }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars.dq_empty);   // the whole row has left TMEM
                 }
                 fence_async_smem();
                 named_barrier_sync(1, 128);
                 if (ok && rt == 0 && !MPIPE_DBG(1)) {
-                    const int q0 = it.kv_start + i * kBT;
                     tma_reduce_add_3d(&maps.dq_acc, stage, 0, head, q0);
-                    tma_reduce_add_3d(&maps.dq_acc, stage + kBT * 128, 32, head, q0);
-                    if (Cfg::kTail) tma_reduce_add_3d(&maps.dq_acc_tail, stage + 2 * kBT * 128, 64, head, q0);
+                    if (Cfg::kTail) tma_reduce_add_3d(&maps.dq_acc_tail, stage + Cfg::kStageMain, 64, head, q0);
+                    bulk_commit_group();
+                }
+                if (rt == 0) bulk_wait_group_read<0>();
+                named_barrier_sync(1, 128);
+                if (ok) {
+#pragma unroll
+                    for (int chunk = 0; chunk < 8; ++chunk)
+                        *reinterpret_cast<uint4*>(stage + r * 128 + ((chunk ^ (r & 7)) << 4)) =
+                            make_uint4(v1[chunk / 4][4 * (chunk & 3)], v1[chunk / 4][4 * (chunk & 3) + 1],
+                                       v1[chunk / 4][4 * (chunk & 3) + 2], v1[chunk / 4][4 * (chunk & 3) + 3]);
+                }
+                fence_async_smem();
+                named_barrier_sync(1, 128);
+                if (ok && rt == 0 && !MPIPE_DBG(1)) {
+                    tma_reduce_add_3d(&maps.dq_acc, stage, 32, head, q0);
                     bulk_commit_group();
                 }
                 if (lane == 0 && warp == 12) MPIPE_TR(3, pc * 8 + 2);
             }
-            if (ok) ok = mbar_wait<MPIPE_SLEEP_AUX>(&bars.dkv_full, unit_it & 1, &abort_flag);
+            if (ok) ok = MW(mbar_wait<MPIPE_SLEEP_AUX>(&bars.dkv_full, unit_it & 1, &abort_flag));
             if (!ok) continue;   // keep walking the units so that the named barriers above stay matched
             tc_fence_after();
             const bool store = r < it.row_len;
@@ -600,28 +662,29 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 const float mul = which == 0 ? 1.0f : p.scale;
                 __nv_bfloat16* row = which == 0 ? dv_row : dk_row;
 #pragma unroll
-                for (int c0 = 0; c0 < D; c0 += 16) {
-                    uint32_t v[16];
-                    tmem_ld16(tmem + lane_base + col + c0, v);
+                for (int c0 = 0; c0 < D; c0 += 32) {   // 32 columns per round trip (16 in the D = 80 tail)
+                    uint32_t v[2][16];
+                    const bool two = (c0 + 32 <= D);
+                    tmem_ld16(tmem + lane_base + col + c0, v[0]);
+                    if (two) tmem_ld16(tmem + lane_base + col + c0 + 16, v[1]);
                     tmem_wait_ld();
-                    uint4 a, b;
-                    a.x = pack_bf16(__uint_as_float(v[0]) * mul, __uint_as_float(v[1]) * mul);
-                    a.y = pack_bf16(__uint_as_float(v[2]) * mul, __uint_as_float(v[3]) * mul);
-                    a.z = pack_bf16(__uint_as_float(v[4]) * mul, __uint_as_float(v[5]) * mul);
-                    a.w = pack_bf16(__uint_as_float(v[6]) * mul, __uint_as_float(v[7]) * mul);
-                    b.x = pack_bf16(__uint_as_float(v[8]) * mul, __uint_as_float(v[9]) * mul);
-                    b.y = pack_bf16(__uint_as_float(v[10]) * mul, __uint_as_float(v[11]) * mul);
-                    b.z = pack_bf16(__uint_as_float(v[12]) * mul, __uint_as_float(v[13]) * mul);
-                    b.w = pack_bf16(__uint_as_float(v[14]) * mul, __uint_as_float(v[15]) * mul);
-                    if (store) {
-                        *reinterpret_cast<uint4*>(row + c0) = a;
-                        *reinterpret_cast<uint4*>(row + c0 + 8) = b;
+                    if (which == 1 && c0 + 32 >= D) {   // both accumulators have left TMEM: the next unit may overwrite them
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars.dkv_empty);
+                    }
+#pragma unroll
+                    for (int c8 = 0; c8 < (two ? 4 : 2); ++c8) {
+                        const uint32_t* w = &v[c8 / 2][(c8 & 1) * 8];
+                        uint4 a;
+                        a.x = pack_bf16(__uint_as_float(w[0]) * mul, __uint_as_float(w[1]) * mul);
+                        a.y = pack_bf16(__uint_as_float(w[2]) * mul, __uint_as_float(w[3]) * mul);
+                        a.z = pack_bf16(__uint_as_float(w[4]) * mul, __uint_as_float(w[5]) * mul);
+                        a.w = pack_bf16(__uint_as_float(w[6]) * mul, __uint_as_float(w[7]) * mul);
+                        if (store) *reinterpret_cast<uint4*>(row + c0 + 8 * c8) = a;
                     }
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars.dkv_empty);
         }
         if (rt == 0) bulk_wait_group<0>();   // all reductions have landed before the CTA exits
     }
@@ -745,6 +808,9 @@ extern "C" {
 #ifdef MPIPE_TRACE
 int32_t mpipe_dbg_set_flags(int32_t flags) {
     return cudaMemcpyToSymbol(mpipe::g_dbg_flags, &flags, sizeof(int)) == cudaSuccess ? 0 : 1;
+}
+int32_t mpipe_dbg_read_where(int* host_out) {
+    return cudaMemcpyFromSymbol(host_out, mpipe::g_where, sizeof(int) * 16) == cudaSuccess ? 0 : 1;
 }
 int32_t mpipe_dbg_read_trace(long long* host_out) {
     return cudaMemcpyFromSymbol(host_out, mpipe::g_trace, sizeof(long long) * 4 * 4096) == cudaSuccess ? 0 : 1;
