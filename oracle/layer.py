@@ -1,0 +1,93 @@
+"""CPU oracle for the packed encoder layer -- TEST INFRASTRUCTURE, not product code.
+
+The paper names the relocated computation only as a "ViT-style encoder" (Section 2, "From LLM to
+MLLM Training"); the layer stated here is the pre-norm Transformer block of that family, over a
+packed varlen token matrix x[T, hidden]:
+
+    a  = LayerNorm(x; g1, b1)
+    qkv = a Wqkv^T + bqkv                      -> q, k, v as [T, H, D]   (column block order q | k | v)
+    o  = per-image softmax attention (oracle.attn_fwd, block-diagonal over cu_seqlens)
+    x1 = x + o Wo^T + bo
+    m  = LayerNorm(x1; g2, b2)
+    y  = x1 + GELU(m W1^T + bb1) W2^T + bb2    GELU(u) = u * Phi(u)  (erf form)
+
+Everything is fp64 numpy with no blocking or reordering; weights are nn.Linear-style [out, in].
+Inputs that are bf16 on the GPU side are passed as uint16 bit patterns and widened exactly.
+The GPU path rounds every stored intermediate to bf16; this oracle does not (the tolerance of
+the parity tests covers that, as it does for the attention output).
+
+Pins: ``tests/test_oracle_layer.py`` (torch fp64 functional ops, closed forms, identity cases).
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+
+import numpy as np
+
+from . import _f64, attn_fwd
+
+
+def widen(a) -> np.ndarray:
+    """bf16 bit patterns (uint16) -> fp64, exactly; fp64 passes through."""
+    return _f64(a)
+
+
+def layernorm(x: np.ndarray, gamma: np.ndarray, beta: np.ndarray, eps: float) -> np.ndarray:
+    """Row-wise (x - mean) / sqrt(var + eps) * gamma + beta with the biased variance."""
+    x = np.asarray(x, dtype=np.float64)
+    mean = x.mean(axis=-1, keepdims=True)
+    var = ((x - mean) ** 2).mean(axis=-1, keepdims=True)
+    return (x - mean) / np.sqrt(var + eps) * gamma + beta
+
+
+def linear(x: np.ndarray, w: np.ndarray, b=None) -> np.ndarray:
+    """y = x w^T + b, w as [out, in]."""
+    y = np.asarray(x, dtype=np.float64) @ np.asarray(w, dtype=np.float64).T
+    return y if b is None else y + np.asarray(b, dtype=np.float64)
+
+
+try:   # a library erf as one step of the definition; the fallback is the C library's, element by element
+    from scipy.special import erf as _erf
+except ImportError:   # pragma: no cover
+    _erf = np.vectorize(math.erf, otypes=[np.float64])
+
+
+def gelu(u: np.ndarray) -> np.ndarray:
+    """u * Phi(u) with Phi the standard normal CDF: 0.5 u (1 + erf(u / sqrt 2))."""
+    u = np.asarray(u, dtype=np.float64)
+    return 0.5 * u * (1.0 + _erf(u / math.sqrt(2.0)))
+
+
+@dataclass
+class LayerWeights:
+    """fp64 views of the layer's parameters (nn.Linear layout [out, in])."""
+    g1: np.ndarray
+    b1: np.ndarray
+    wqkv: np.ndarray   # [3*hidden, hidden], rows ordered q | k | v, each head-major
+    bqkv: np.ndarray
+    wo: np.ndarray     # [hidden, hidden]
+    bo: np.ndarray
+    g2: np.ndarray
+    b2: np.ndarray
+    w1: np.ndarray     # [ffn, hidden]
+    bb1: np.ndarray
+    w2: np.ndarray     # [hidden, ffn]
+    bb2: np.ndarray
+
+
+def encoder_layer_fwd(x, w: LayerWeights, cu_seqlens, n_heads: int, scale: float, eps: float):
+    """The whole block.  x: [T, hidden] (uint16 bf16 bits or fp64).  Returns (y, parts) with parts a dict of
+    the intermediates (a, qkv, o, x1, m, f) in fp64 for stage-wise comparisons."""
+    x = widen(x)
+    T, hidden = x.shape
+    D = hidden // n_heads
+    a = layernorm(x, w.g1, w.b1, eps)
+    qkv = linear(a, w.wqkv, w.bqkv)
+    q, k, v = (np.ascontiguousarray(qkv[:, i * hidden:(i + 1) * hidden].reshape(T, n_heads, D)) for i in range(3))
+    o, lse = attn_fwd(q, k, v, cu_seqlens, scale)
+    x1 = x + linear(o.reshape(T, hidden), w.wo, w.bo)
+    m = layernorm(x1, w.g2, w.b2, eps)
+    f = gelu(linear(m, w.w1, w.bb1))
+    y = x1 + linear(f, w.w2, w.bb2)
+    return y, {"a": a, "qkv": qkv, "o": o, "lse": lse, "x1": x1, "m": m, "f": f}

@@ -1,0 +1,107 @@
+"""Pins of the encoder-layer oracle (oracle/layer.py) against what fixes it from outside: torch's fp64
+functional ops (library routines), closed forms, and cases that reduce to something simpler."""
+import math
+
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+import oracle
+from oracle import layer as L
+
+
+def _rand_weights(rng, hidden, ffn, scale=0.2):
+    def r(*s):
+        return rng.standard_normal(s) * scale
+    return L.LayerWeights(g1=1 + r(hidden), b1=r(hidden), wqkv=r(3 * hidden, hidden), bqkv=r(3 * hidden),
+                          wo=r(hidden, hidden), bo=r(hidden), g2=1 + r(hidden), b2=r(hidden),
+                          w1=r(ffn, hidden), bb1=r(ffn), w2=r(hidden, ffn), bb2=r(hidden))
+
+
+def test_layernorm_matches_torch_and_normalises():
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal((7, 48)) * 3 + 1.5
+    g, b = rng.standard_normal(48), rng.standard_normal(48)
+    ref = F.layer_norm(torch.from_numpy(x), (48,), torch.from_numpy(g), torch.from_numpy(b), 1e-6).numpy()
+    np.testing.assert_allclose(L.layernorm(x, g, b, 1e-6), ref, rtol=0, atol=1e-12)
+    z = L.layernorm(x, np.ones(48), np.zeros(48), 1e-6)
+    np.testing.assert_allclose(z.mean(axis=1), 0, atol=1e-13)
+    var = x.var(axis=1)
+    np.testing.assert_allclose(z.var(axis=1), var / (var + 1e-6), rtol=1e-12)
+    # shift / scale invariance of the normalised value (eps -> 0)
+    np.testing.assert_allclose(L.layernorm(5 * x + 3, g, b, 0.0), L.layernorm(x, g, b, 0.0), atol=1e-11)
+
+
+def test_linear_matches_torch_on_non_square_shapes():
+    rng = np.random.default_rng(2)
+    x, w, b = rng.standard_normal((5, 12)), rng.standard_normal((9, 12)), rng.standard_normal(9)
+    ref = F.linear(torch.from_numpy(x), torch.from_numpy(w), torch.from_numpy(b)).numpy()
+    np.testing.assert_allclose(L.linear(x, w, b), ref, atol=1e-13)
+    # one-hot input picks a column of w (catches a transposed operand)
+    e = np.zeros((1, 12)); e[0, 3] = 1
+    np.testing.assert_allclose(L.linear(e, w)[0], w[:, 3], atol=0)
+
+
+def test_gelu_closed_forms_and_torch():
+    phi1 = 0.5 * (1 + math.erf(1 / math.sqrt(2)))   # standard normal CDF at 1 = 0.841344746...
+    assert abs(phi1 - 0.8413447460685429) < 1e-15
+    np.testing.assert_allclose(L.gelu(np.array([0.0, 1.0, -1.0])), [0.0, phi1, -(1 - phi1)], atol=1e-15)
+    u = np.linspace(-6, 6, 241)
+    np.testing.assert_allclose(L.gelu(u) - L.gelu(-u), u, atol=1e-14)          # u Phi(u) + u Phi(-u)... = u
+    np.testing.assert_allclose(L.gelu(u), F.gelu(torch.from_numpy(u)).numpy(), atol=1e-14)
+    assert abs(L.gelu(np.array([30.0]))[0] - 30.0) < 1e-12 and abs(L.gelu(np.array([-30.0]))[0]) < 1e-12
+
+
+def _torch_layer(x, w, counts, H, scale, eps):
+    """The same block from torch fp64 library ops and a dense block-diagonal mask."""
+    t = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float64))
+    T, hidden = x.shape
+    D = hidden // H
+    X = t(x)
+    a = F.layer_norm(X, (hidden,), t(w.g1), t(w.b1), eps)
+    qkv = F.linear(a, t(w.wqkv), t(w.bqkv))
+    q, k, v = (qkv[:, i * hidden:(i + 1) * hidden].reshape(T, H, D).permute(1, 0, 2) for i in range(3))
+    seg = torch.repeat_interleave(torch.arange(len(counts)), torch.tensor(counts))
+    mask = seg[:, None] == seg[None, :]
+    s = (q @ k.transpose(1, 2)) * scale
+    s = s.masked_fill(~mask, float("-inf"))
+    o = (torch.softmax(s, dim=-1) @ v).permute(1, 0, 2).reshape(T, hidden)
+    x1 = X + F.linear(o, t(w.wo), t(w.bo))
+    m = F.layer_norm(x1, (hidden,), t(w.g2), t(w.b2), eps)
+    y = x1 + F.linear(F.gelu(F.linear(m, t(w.w1), t(w.bb1))), t(w.w2), t(w.bb2))
+    return y.numpy()
+
+
+@pytest.mark.parametrize("counts,H,D", [([5, 1, 9], 2, 8), ([16, 7], 3, 16)])
+def test_layer_matches_torch_composite(counts, H, D):
+    rng = np.random.default_rng(3)
+    hidden, ffn = H * D, 3 * H * D
+    w = _rand_weights(rng, hidden, ffn)
+    x = rng.standard_normal((sum(counts), hidden))
+    cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    scale = float(np.float32(1 / math.sqrt(D)))   # the scale is an fp32 input of the attention oracle, as in the C ABI
+    y, parts = L.encoder_layer_fwd(x, w, cu, H, scale, 1e-6)
+    np.testing.assert_allclose(y, _torch_layer(x, w, counts, H, scale, 1e-6), atol=1e-11)
+    assert parts["qkv"].shape == (sum(counts), 3 * hidden) and parts["f"].shape == (sum(counts), ffn)
+
+
+def test_layer_special_cases():
+    rng = np.random.default_rng(4)
+    H, D = 2, 8
+    hidden, ffn = H * D, 32
+    w = _rand_weights(rng, hidden, ffn)
+    x = rng.standard_normal((6, hidden))
+    # zero output projections: both residual branches vanish
+    w0 = L.LayerWeights(**{**w.__dict__, "wo": np.zeros_like(w.wo), "bo": np.zeros_like(w.bo),
+                           "w2": np.zeros_like(w.w2), "bb2": np.zeros_like(w.bb2)})
+    y, _ = L.encoder_layer_fwd(x, w0, np.array([0, 2, 6], dtype=np.int32), H, 0.3, 1e-6)
+    np.testing.assert_allclose(y, x, atol=0)
+    # one-token images: attention returns v, so x1 = x + Wo v + bo
+    cu = np.arange(7, dtype=np.int32)
+    _, parts = L.encoder_layer_fwd(x, w, cu, H, 0.3, 1e-6)
+    v = parts["qkv"][:, 2 * hidden:]
+    np.testing.assert_allclose(parts["x1"], x + v @ w.wo.T + w.bo, atol=1e-12)
+    # bf16 bit patterns widen exactly
+    bits = (np.float32(1.5).view(np.uint32) >> 16).astype(np.uint16)
+    assert L.widen(np.array([[bits]], dtype=np.uint16))[0, 0] == 1.5
