@@ -215,10 +215,58 @@ int32_t mpipe_merge_tokens_bwd(const void* d_llm_embeds, int64_t emb_row_stride,
 int32_t mpipe_validate_positions(const int32_t* positions, int32_t n, int32_t n_llm_tokens);
 
 /*
+ * The rest of the packed encoder layer -- what one Fwd(enc, r, m) event of the transpose schedule executes
+ * besides attention (Section 4.2; the paper says only "ViT-style encoder", Section 2: the block below is the
+ * pre-norm Transformer block of that family).  Forward only: it is the whole layer of a FROZEN encoder
+ * (Lemma 1: no backward events exist then); for a TRAINED one it also writes the LSE that
+ * mpipe_varlen_attn_bwd needs, the backward of the projections and norms is not part of this library yet.
+ *
+ *   mpipe_linear_fwd     C[M, N] = act(A[M, K] W[N, K]^T + bias[N]) + residual[M, N]; all bf16, device, row-major
+ *                        with row strides lda / ldw / ldr / ldc in elements (multiples of 8, bases 16-byte
+ *                        aligned), fp32 accumulation on the tensor cores, act = GELU (u Phi(u), erf form) when
+ *                        flags has MPIPE_LINEAR_GELU, identity otherwise; bias and residual may be NULL.
+ *                        N and K multiples of 8 (MPIPE_ERR_UNSUPPORTED otherwise); M == 0 launches nothing.
+ *   mpipe_layernorm_fwd  y[t, :] = (x[t, :] - mean_t) * rsqrt(var_t + eps) * gamma + beta, biased variance, fp32
+ *                        statistics; bf16 in and out, hidden a multiple of 8 and <= 2048.
+ *   mpipe_encoder_layer_fwd
+ *        a = LN(x; ln1) ; qkv = a Wqkv^T + bqkv (columns q | k | v, each [n_heads][head_dim]) ;
+ *        o = per-image softmax attention (mpipe_varlen_attn_fwd on strided views of qkv, same plan arguments) ;
+ *        x1 = x + o Wo^T + bo ; m = LN(x1; ln2) ; y = x1 + GELU(m W1^T + b1) W2^T + b2.
+ *        x, y: bf16 [n_tokens, hidden] contiguous, device; y may not alias x.  Weights: device bf16, nn.Linear
+ *        layout [out, in], contiguous.  lse: fp32 [n_heads, n_tokens] when TRAINED, ignored when FROZEN.
+ *        workspace: device, 256-byte aligned, >= mpipe_encoder_layer_workspace_bytes (MPIPE_ERR_WORKSPACE);
+ *        caller-owned, contents undefined afterwards.  Seven launches on `stream`, no allocation, no sync.
+ *        head_dim = hidden / n_heads must be one the attention kernels support (64, 80).
+ * Device-side findings (a bounded wait that ran out) are reported through status_buf as for the attention calls.
+ */
+#define MPIPE_LINEAR_GELU 1
+
+typedef struct {
+    const void *ln1_gamma, *ln1_beta;   /* [hidden] */
+    const void *w_qkv, *b_qkv;          /* [3*hidden, hidden], [3*hidden] */
+    const void *w_o, *b_o;              /* [hidden, hidden], [hidden] */
+    const void *ln2_gamma, *ln2_beta;   /* [hidden] */
+    const void *w_fc1, *b_fc1;          /* [ffn, hidden], [ffn] */
+    const void *w_fc2, *b_fc2;          /* [hidden, ffn], [hidden] */
+} mpipe_layer_weights_t;
+
+int32_t mpipe_linear_fwd(const void* a, const void* w, const void* bias, const void* residual, void* c, int32_t M,
+                         int32_t N, int32_t K, int64_t lda, int64_t ldw, int64_t ldr, int64_t ldc, int32_t flags,
+                         int32_t* status_buf, void* stream);
+int32_t mpipe_layernorm_fwd(const void* x, const void* gamma, const void* beta, void* y, int32_t n_tokens,
+                            int32_t hidden, int64_t ldx, int64_t ldy, float eps, void* stream);
+size_t mpipe_encoder_layer_workspace_bytes(int32_t n_tokens, int32_t hidden, int32_t ffn);
+int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weights_t* w, int32_t n_tokens,
+                                int32_t hidden, int32_t n_heads, int32_t ffn, const int32_t* cu_seqlens_dev,
+                                int32_t n_seg, int32_t max_seqlen, const mpipe_work_item_t* fwd_items_dev,
+                                int32_t n_fwd_items, float softmax_scale, float ln_eps, int32_t mode, float* lse,
+                                void* workspace, size_t workspace_bytes, int32_t* status_buf, void* stream);
+
+/*
  * Measurement aid (no counterpart in the paper; its cost model weights each compute event with one
  * duration, Section 4.3, and this is how a benchmark reads that duration for one kernel): while set,
  * the launch of kernel `which` (0 = attention forward, 1 = attention backward main kernel, 2 = merge
- * / merge_bwd) records the two cudaEvent_t handles on the call's stream directly before and after
+ * / merge_bwd, 3 = mpipe_linear_fwd, 4 = mpipe_layernorm_fwd) records the two cudaEvent_t handles on the call's stream directly before and after
  * it.  NULL handles switch it off.  Process-wide, not thread-safe: set it from the thread that makes
  * the calls.  Returns MPIPE_ERR_INVALID_ARG for an unknown `which`.
  */

@@ -32,6 +32,11 @@ ITEM_DTYPE = np.dtype([(n, np.int32) for n in ("seg", "tile", "row_start", "row_
 
 _i32, _i64, _vp, _f32, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float, ctypes.c_size_t
 _SIGNATURES = {
+    "mpipe_linear_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _i32, _vp, _vp]),
+    "mpipe_layernorm_fwd": (_i32, [_vp, _vp, _vp, _vp, _i32, _i32, _i64, _i64, _f32, _vp]),
+    "mpipe_encoder_layer_workspace_bytes": (_sz, [_i32, _i32, _i32]),
+    "mpipe_encoder_layer_fwd": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _i32, _i32, _vp, _i32, _f32, _f32,
+                                       _i32, _vp, _vp, _sz, _vp, _vp]),
     "mpipe_fwd_tile_rows": (_i32, []),
     "mpipe_bwd_tile_rows": (_i32, []),
     "mpipe_seg_plan": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -223,6 +228,69 @@ def varlen_attn_bwd(dout, q, k, v, o, lse, dq, dk, dv, plan: SegPlan, softmax_sc
         _ptr(plan.bwd_items_dev), int(plan.bwd_items.size), H, D, softmax_scale, plan.mode, _ptr(workspace),
         ws_bytes, _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_varlen_attn_bwd")
+
+
+LINEAR_GELU = 1
+
+
+def _rows(t):
+    assert t.dim() == 2 and t.stride(1) == 1 and t.dtype == torch.bfloat16
+    return t.stride(0)
+
+
+def linear_fwd(a, w, c, bias=None, residual=None, gelu: bool = False, status_buf=None, stream=None) -> None:
+    """mpipe_linear_fwd: c[M,N] = act(a[M,K] w[N,K]^T + bias) + residual (bf16 CUDA tensors, rows contiguous)."""
+    M, K = a.shape
+    N = w.shape[0]
+    assert w.shape[1] == K and tuple(c.shape) == (M, N)
+    if bias is not None:
+        assert bias.dtype == torch.bfloat16 and bias.is_contiguous() and bias.numel() == N
+    st = load().mpipe_linear_fwd(_ptr(a), _ptr(w), _ptr(bias), _ptr(residual), _ptr(c), M, N, K, _rows(a), _rows(w),
+                                 0 if residual is None else _rows(residual), _rows(c), LINEAR_GELU if gelu else 0,
+                                 _ptr(status_buf), _stream(stream))
+    _check(st, "mpipe_linear_fwd")
+
+
+def layernorm_fwd(x, gamma, beta, y, eps: float, stream=None) -> None:
+    """mpipe_layernorm_fwd over the rows of x [T, hidden] (bf16 CUDA tensors)."""
+    T, hidden = x.shape
+    assert tuple(y.shape) == (T, hidden) and gamma.numel() == hidden and beta.numel() == hidden
+    assert gamma.dtype == beta.dtype == torch.bfloat16 and gamma.is_contiguous() and beta.is_contiguous()
+    st = load().mpipe_layernorm_fwd(_ptr(x), _ptr(gamma), _ptr(beta), _ptr(y), T, hidden, _rows(x), _rows(y), eps,
+                                    _stream(stream))
+    _check(st, "mpipe_layernorm_fwd")
+
+
+class LayerWeights(ctypes.Structure):
+    """mpipe_layer_weights_t: twelve device pointers.  ``from_tensors`` keeps the tensors alive."""
+    _fields_ = [(n, ctypes.c_void_p) for n in ("ln1_gamma", "ln1_beta", "w_qkv", "b_qkv", "w_o", "b_o", "ln2_gamma",
+                                               "ln2_beta", "w_fc1", "b_fc1", "w_fc2", "b_fc2")]
+
+    @classmethod
+    def from_tensors(cls, **tensors) -> "LayerWeights":
+        w = cls()
+        for name, _ in cls._fields_:
+            t = tensors[name]
+            assert t.dtype == torch.bfloat16 and t.is_cuda and t.is_contiguous(), name
+            setattr(w, name, t.data_ptr())
+        w._keep = tensors
+        return w
+
+
+def encoder_layer_workspace_bytes(n_tokens: int, hidden: int, ffn: int) -> int:
+    return load().mpipe_encoder_layer_workspace_bytes(n_tokens, hidden, ffn)
+
+
+def encoder_layer_fwd(x, y, weights: LayerWeights, n_heads: int, ffn: int, plan: SegPlan, softmax_scale: float,
+                      ln_eps: float, workspace, lse=None, status_buf=None, stream=None) -> None:
+    """mpipe_encoder_layer_fwd: x, y bf16 [T, hidden] contiguous CUDA tensors; lse fp32 [H, T] for a trained plan."""
+    T, hidden = x.shape
+    assert x.is_contiguous() and y.is_contiguous() and tuple(y.shape) == (T, hidden) and x.dtype == y.dtype == torch.bfloat16
+    st = load().mpipe_encoder_layer_fwd(
+        _ptr(x), _ptr(y), ctypes.addressof(weights), T, hidden, n_heads, ffn, _ptr(plan.cu_seqlens_dev), plan.n_seg,
+        plan.max_seqlen, _ptr(plan.fwd_items_dev), int(plan.fwd_items.size), softmax_scale, ln_eps, plan.mode, _ptr(lse),
+        _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status_buf), _stream(stream))
+    _check(st, "mpipe_encoder_layer_fwd")
 
 
 def attn_bwd_static_scratch_bytes() -> int:

@@ -16,7 +16,7 @@ int sm_count();
 struct ProfileEvents {
     cudaEvent_t start = nullptr, stop = nullptr;
 };
-enum { kProfileFwd = 0, kProfileBwdMain = 1, kProfileMerge = 2, kProfileSlots = 3 };
+enum { kProfileFwd = 0, kProfileBwdMain = 1, kProfileMerge = 2, kProfileLinear = 3, kProfileLayerNorm = 4, kProfileSlots = 5 };
 extern ProfileEvents g_profile[kProfileSlots];
 inline void profile_start(int which, cudaStream_t st) {
     if (g_profile[which].start != nullptr) cudaEventRecord(g_profile[which].start, st);

@@ -1,0 +1,258 @@
+// mpipe_linear_fwd: C[M, N] = epilogue(A[M, K] * W[N, K]^T), the dense projections of the packed encoder layer
+// (QKV, attention output, MLP) on the token matrix [T, hidden].  bf16 operands, fp32 accumulation in TMEM.
+//
+// Persistent kernel, one CTA per SM, static round-robin over 128 x 256 output tiles (n fastest, so that the
+// CTAs of a wave share the few weight tiles in L2 and walk down the token rows together).
+//   warp 0      TMA producer: A box [128 rows][64 k], W box [256 rows][64 k] per stage, 128-byte swizzle, 4 stages
+//   warp 1      tcgen05 issuer: 4 x (M 128, N 256, K 16) smem x smem MMAs per stage into one of TWO 256-column
+//               TMEM accumulators, so the epilogue of tile i overlaps the main loop of tile i + 1
+//   warp 2      TMEM allocation
+//   warps 4-11  epilogue: thread = output row = TMEM lane; warpgroup 0 takes columns 0..127, warpgroup 1
+//               columns 128..255; 32 columns per TMEM round trip; + bias, GELU, + residual, bf16, 16-byte stores
+// Every mbarrier wait is bounded (status MPIPE_ERR_TIMEOUT), as in the attention kernels.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "common.h"
+#include "sm100_ptx.cuh"
+#include "tensormap.h"
+
+namespace mpipe {
+
+constexpr int kGemmBM = 128, kGemmBN = 256, kGemmBK = 64, kGemmStages = 4;
+constexpr int kGemmThreads = 384;
+constexpr int kGemmABytes = kGemmBM * kGemmBK * 2;   // 16 KB
+constexpr int kGemmBBytes = kGemmBN * kGemmBK * 2;   // 32 KB
+constexpr int kGemmStageBytes = kGemmABytes + kGemmBBytes;
+constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 1024;
+static_assert(kGemmSmem <= 227 * 1024, "shared memory budget");
+
+struct GemmParams {
+    int32_t M, N, K;
+    int32_t tiles_m, tiles_n;
+    const __nv_bfloat16* bias;       // [N] or null
+    const __nv_bfloat16* residual;   // [M, ldr] or null
+    __nv_bfloat16* C;                // [M, ldc]
+    int64_t ldr, ldc;
+    int32_t gelu;
+    int32_t* status_buf;
+};
+
+struct GemmBarriers {
+    uint64_t full[kGemmStages], empty[kGemmStages], acc_full[2], acc_empty[2];
+};
+
+// erf by the rational-times-Gaussian form of Abramowitz & Stegun 7.1.26 (|error| <= 1.5e-7, far below the bf16
+// rounding of the result): two special-function ops and a degree-5 Horner chain instead of the library routine's branches.
+__device__ __forceinline__ float erf_as(float x) {
+    const float ax = fabsf(x);
+    const float t = __frcp_rn(fmaf(0.3275911f, ax, 1.0f));
+    float p = fmaf(1.061405429f, t, -1.453152027f);
+    p = fmaf(p, t, 1.421413741f);
+    p = fmaf(p, t, -0.284496736f);
+    p = fmaf(p, t, 0.254829592f);
+    p *= t;
+    const float e = ex2_approx(-ax * ax * 1.4426950408889634f);
+    return copysignf(1.0f - p * e, x);
+}
+__device__ __forceinline__ float gelu_erf(float u) { return 0.5f * u * (1.0f + erf_as(u * 0.7071067811865476f)); }
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+linear_fwd_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ GemmBarriers bars;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < kGemmStages; ++s) {
+            mbar_init(&bars.full[s], 1);
+            mbar_init(&bars.empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&bars.acc_full[a], 1);
+            mbar_init(&bars.acc_empty[a], 8);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 2) {
+        tmem_alloc(&tmem_base_slot, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_slot;
+    const int n_tiles = p.tiles_m * p.tiles_n;
+    const int nk = (p.K + kGemmBK - 1) / kGemmBK;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tmap(&map_a);
+            prefetch_tmap(&map_w);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+                const int m0 = (t / p.tiles_n) * kGemmBM, n0 = (t % p.tiles_n) * kGemmBN;
+                for (int kb = 0; kb < nk; ++kb, ++it) {
+                    const int s = it % kGemmStages;
+                    ok = mbar_wait<100>(&bars.empty[s], ((it / kGemmStages) & 1) ^ 1, &abort_flag);
+                    if (!ok) break;
+                    uint8_t* st = smem + s * kGemmStageBytes;
+                    mbar_expect_tx(&bars.full[s], kGemmStageBytes);   // out-of-range rows / columns are zero-filled, still counted
+                    tma_load_3d(st, &map_a, &bars.full[s], kb * kGemmBK, 0, m0);
+                    tma_load_3d(st + kGemmABytes, &map_w, &bars.full[s], kb * kGemmBK, 0, n0);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        const bool leader = elect_one();
+        const uint32_t sbase = smem_u32(smem);
+        constexpr uint32_t hi128 = umma_desc_hi(1024, kSwizzle128);
+        constexpr uint32_t idesc = umma_idesc_bf16(kGemmBM, kGemmBN, 0, 0);
+        uint32_t it = 0, tile_it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_it) {
+            const uint32_t acc = tile_it & 1;
+            ok = mbar_wait(&bars.acc_empty[acc], ((tile_it >> 1) & 1) ^ 1, &abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            for (int kb = 0; kb < nk; ++kb, ++it) {
+                const int s = it % kGemmStages;
+                ok = mbar_wait(&bars.full[s], (it / kGemmStages) & 1, &abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_lo = umma_desc_lo(sbase + s * kGemmStageBytes, 0);
+                const uint32_t b_lo = umma_desc_lo(sbase + s * kGemmStageBytes + kGemmABytes, 0);
+                if (leader) {
+#pragma unroll
+                    for (int ks = 0; ks < kGemmBK / 16; ++ks)
+                        umma_ss(tmem + acc * kGemmBN, umma_desc(a_lo + ks * 2, hi128), umma_desc(b_lo + ks * 2, hi128), idesc,
+                                (kb > 0 || ks > 0) ? 1u : 0u);
+                    umma_commit(&bars.empty[s]);
+                }
+            }
+            if (!ok) break;
+            if (leader) umma_commit(&bars.acc_full[acc]);
+        }
+        __syncwarp();
+    } else if (warp >= 4) {
+        const int wg = (warp - 4) >> 2;                 // column half of the tile
+        const int r = ((warp & 3) << 5) | lane;         // output row inside the tile = TMEM lane
+        const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
+        uint32_t tile_it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_it) {
+            const uint32_t acc = tile_it & 1;
+            const int m = (t / p.tiles_n) * kGemmBM + r;
+            const int n_base = (t % p.tiles_n) * kGemmBN + wg * (kGemmBN / 2);
+            ok = mbar_wait(&bars.acc_full[acc], (tile_it >> 1) & 1, &abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const bool row_ok = m < p.M;
+            __nv_bfloat16* crow = p.C + int64_t(m) * p.ldc;
+            const __nv_bfloat16* rrow = p.residual != nullptr ? p.residual + int64_t(m) * p.ldr : nullptr;
+#pragma unroll 1
+            for (int c0 = 0; c0 < kGemmBN / 2; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tmem + lane_base + acc * kGemmBN + wg * (kGemmBN / 2) + c0, v);
+                tmem_wait_ld();
+                if (c0 + 32 == kGemmBN / 2) {   // this thread's part of the accumulator is in registers
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars.acc_empty[acc]);
+                }
+#pragma unroll
+                for (int g8 = 0; g8 < 4; ++g8) {   // 8 columns = 16 bytes of output
+                    const int n = n_base + c0 + 8 * g8;
+                    if (n >= p.N) break;            // N is a multiple of 8
+                    float f[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[8 * g8 + i]);
+                    if (p.bias != nullptr) {
+                        const uint4 b4 = __ldg(reinterpret_cast<const uint4*>(p.bias + n));
+                        const uint32_t bw[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            f[2 * i] += __uint_as_float(bw[i] << 16);
+                            f[2 * i + 1] += __uint_as_float(bw[i] & 0xffff0000u);
+                        }
+                    }
+                    if (p.gelu) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
+                    }
+                    if (rrow != nullptr && row_ok) {
+                        const uint4 r4 = *reinterpret_cast<const uint4*>(rrow + n);
+                        const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            f[2 * i] += __uint_as_float(rw[i] << 16);
+                            f[2 * i + 1] += __uint_as_float(rw[i] & 0xffff0000u);
+                        }
+                    }
+                    if (row_ok)
+                        *reinterpret_cast<uint4*>(crow + n) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]),
+                                                                         pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) tmem_dealloc(tmem, 512);
+    if (tid == 0 && abort_flag) report_status(p.status_buf, MPIPE_ERR_TIMEOUT, int32_t(blockIdx.x));
+}
+
+}  // namespace mpipe
+
+extern "C" {
+
+int32_t mpipe_linear_fwd(const void* a, const void* w, const void* bias, const void* residual, void* c, int32_t M,
+                         int32_t N, int32_t K, int64_t lda, int64_t ldw, int64_t ldr, int64_t ldc, int32_t flags,
+                         int32_t* status_buf, void* stream) {
+    using namespace mpipe;
+    if (M < 0 || N <= 0 || K <= 0) return MPIPE_ERR_INVALID_ARG;
+    if (M == 0) return MPIPE_OK;
+    if (a == nullptr || w == nullptr || c == nullptr) return MPIPE_ERR_INVALID_ARG;
+    if ((flags & ~(MPIPE_LINEAR_GELU)) != 0) return MPIPE_ERR_INVALID_ARG;
+    if ((N % 8) != 0 || (K % 8) != 0) return MPIPE_ERR_UNSUPPORTED;
+    if (lda < K || ldw < K || ldc < N || (residual != nullptr && ldr < N)) return MPIPE_ERR_INVALID_ARG;
+    if ((lda % 8) != 0 || (ldw % 8) != 0 || (ldc % 8) != 0 || (residual != nullptr && (ldr % 8) != 0)) return MPIPE_ERR_UNSUPPORTED;
+    if (!aligned16(a) || !aligned16(w) || !aligned16(c) || !aligned16(bias) || !aligned16(residual)) return MPIPE_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CUtensorMap map_a, map_w;
+    if (!make_tensor_map_thd(&map_a, a, M, 1, K, lda, lda, kGemmBK, kGemmBM, 128) ||
+        !make_tensor_map_thd(&map_w, w, N, 1, K, ldw, ldw, kGemmBK, kGemmBN, 128))
+        return MPIPE_ERR_CUDA;
+    GemmParams p;
+    p.M = M; p.N = N; p.K = K;
+    p.tiles_m = cdiv(M, kGemmBM);
+    p.tiles_n = cdiv(N, kGemmBN);
+    p.bias = static_cast<const __nv_bfloat16*>(bias);
+    p.residual = static_cast<const __nv_bfloat16*>(residual);
+    p.C = static_cast<__nv_bfloat16*>(c);
+    p.ldr = ldr; p.ldc = ldc;
+    p.gelu = (flags & MPIPE_LINEAR_GELU) ? 1 : 0;
+    p.status_buf = status_buf;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(linear_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem) != cudaSuccess)
+            return MPIPE_ERR_CUDA;
+        attr_set = true;
+    }
+    const long long tiles = (long long)p.tiles_m * p.tiles_n;
+    const int grid = int(tiles < sm_count() ? tiles : sm_count());
+    profile_start(kProfileLinear, st);
+    linear_fwd_kernel<<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, p);
+    profile_stop(kProfileLinear, st);
+    return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -98,6 +98,34 @@ def normal_bf16(seed: int, stream: int, shape) -> np.ndarray:
     return out[:n].reshape(shape)
 
 
+def scaled_normal_bf16(seed: int, stream: int, shape, std: float, mean: float = 0.0) -> np.ndarray:
+    """mean + std * N(0,1), rounded to bf16 bits (for synthetic weights, biases and norm parameters)."""
+    z = bf16_bits_to_f32(normal_bf16(seed, stream, shape))
+    return f32_to_bf16_bits((np.float32(mean) + np.float32(std) * z).astype(np.float32))
+
+
+LAYER_PARAMS = ("ln1_gamma", "ln1_beta", "w_qkv", "b_qkv", "w_o", "b_o", "ln2_gamma", "ln2_beta", "w_fc1", "b_fc1",
+                "w_fc2", "b_fc2")
+
+
+def layer_params_bf16(seed: int, hidden: int, ffn: int) -> dict:
+    """Random-init parameters of one encoder layer as bf16 bits: weights N(0, 1/fan_in) so that activations stay
+    O(1), biases N(0, 0.1^2), norm scales 1 + N(0, 0.1^2).  Streams 100.. keep them apart from the activations."""
+    shapes = {"ln1_gamma": (hidden,), "ln1_beta": (hidden,), "w_qkv": (3 * hidden, hidden), "b_qkv": (3 * hidden,),
+              "w_o": (hidden, hidden), "b_o": (hidden,), "ln2_gamma": (hidden,), "ln2_beta": (hidden,),
+              "w_fc1": (ffn, hidden), "b_fc1": (ffn,), "w_fc2": (hidden, ffn), "b_fc2": (hidden,)}
+    out = {}
+    for i, name in enumerate(LAYER_PARAMS):
+        shp = shapes[name]
+        if name.startswith("w_"):
+            out[name] = scaled_normal_bf16(seed, 100 + i, shp, std=float(shp[1]) ** -0.5)
+        elif name.endswith("gamma"):
+            out[name] = scaled_normal_bf16(seed, 100 + i, shp, std=0.1, mean=1.0)
+        else:
+            out[name] = scaled_normal_bf16(seed, 100 + i, shp, std=0.1)
+    return out
+
+
 # --------------------------------------------------------------------------------------
 # Structure recipes
 # --------------------------------------------------------------------------------------

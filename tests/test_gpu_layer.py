@@ -1,0 +1,120 @@
+"""GPU parity of the encoder-layer entry points (linear, layernorm, whole layer) against oracle/layer.py."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import layer as OL
+from paper_2607_03229_b200 import binding as B, workloads as W
+from _util import to_dev, to_f64, rel_l2, status_buf
+
+pytestmark = pytest.mark.gpu
+
+# A bf16 result of an fp32-accumulated dot product: half an ulp of bf16 (2^-9 relative) plus the accumulation error.
+ELEM_REL = 2.0 ** -8
+LAYER_REL_L2 = 1e-2     # several bf16-rounded stages in a row (same bound as the attention gradients)
+
+
+def _check_close(got, ref, atol):
+    err = np.abs(got - ref)
+    bound = atol + ELEM_REL * np.abs(ref)
+    assert (err <= bound).all(), f"max excess {(err - bound).max():.3e} at {np.unravel_index((err - bound).argmax(), err.shape)}"
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 8, 8), (300, 264, 72), (257, 512, 1024), (1000, 1024, 1280), (129, 3072, 64)])
+@pytest.mark.parametrize("bias,res,gelu", [(False, False, False), (True, False, True), (True, True, False)])
+def test_linear_matches_oracle(M, N, K, bias, res, gelu):
+    a = W.normal_bf16(11, 0, (M, K))
+    w = W.scaled_normal_bf16(11, 1, (N, K), std=K ** -0.5)
+    b = W.scaled_normal_bf16(11, 2, (N,), std=0.5) if bias else None
+    r = W.normal_bf16(11, 3, (M, N)) if res else None
+    c = torch.full((M, N), 7.0, dtype=torch.bfloat16, device="cuda")
+    st = status_buf()
+    B.linear_fwd(to_dev(a), to_dev(w), c, None if b is None else to_dev(b), None if r is None else to_dev(r), gelu, st)
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[0] == 0
+    ref = OL.linear(OL.widen(a), OL.widen(w), None if b is None else OL.widen(b))
+    if gelu:
+        ref = OL.gelu(ref)
+    if res:
+        ref = ref + OL.widen(r)
+    _check_close(to_f64(c), ref, atol=2e-3)
+
+
+def test_linear_strided_rows_and_untouched_padding():
+    M, N, K = 200, 256, 128
+    a_full = to_dev(W.normal_bf16(12, 0, (M, K + 8)))
+    c_full = torch.full((M + 3, N + 16), 5.0, dtype=torch.bfloat16, device="cuda")
+    w = W.scaled_normal_bf16(12, 1, (N, K), std=K ** -0.5)
+    B.linear_fwd(a_full[:, :K], to_dev(w), c_full[:M, :N])
+    torch.cuda.synchronize()
+    ref = OL.linear(to_f64(a_full[:, :K]), OL.widen(w))
+    _check_close(to_f64(c_full[:M, :N]), ref, atol=2e-3)
+    assert (c_full[M:, :] == 5.0).all() and (c_full[:, N:] == 5.0).all()
+
+
+@pytest.mark.parametrize("T,hidden", [(1, 8), (37, 256), (1000, 1024), (513, 1280), (9, 2048)])
+def test_layernorm_matches_oracle(T, hidden):
+    x = W.scaled_normal_bf16(13, 0, (T, hidden), std=2.0, mean=0.7)
+    g = W.scaled_normal_bf16(13, 1, (hidden,), std=0.1, mean=1.0)
+    b = W.scaled_normal_bf16(13, 2, (hidden,), std=0.1)
+    y = torch.empty((T, hidden), dtype=torch.bfloat16, device="cuda")
+    B.layernorm_fwd(to_dev(x), to_dev(g), to_dev(b), y, 1e-6)
+    torch.cuda.synchronize()
+    ref = OL.layernorm(OL.widen(x), OL.widen(g), OL.widen(b), 1e-6)
+    _check_close(to_f64(y), ref, atol=1e-4)
+
+
+def _run_layer(counts, H, D, ffn, mode, seed=21):
+    hidden = H * D
+    T = sum(counts)
+    pb = W.layer_params_bf16(seed, hidden, ffn)
+    x = W.normal_bf16(seed, 0, (T, hidden))
+    plan = B.seg_plan(counts, mode).to_device()
+    weights = B.LayerWeights.from_tensors(**{k: to_dev(v) for k, v in pb.items()})
+    y = torch.empty((T, hidden), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((H, T), dtype=torch.float32, device="cuda") if mode == B.TRAINED else None
+    ws = torch.empty(B.encoder_layer_workspace_bytes(T, hidden, ffn), dtype=torch.uint8, device="cuda")
+    st = status_buf()
+    scale = float(np.float32(1 / math.sqrt(D)))
+    B.encoder_layer_fwd(to_dev(x), y, weights, H, ffn, plan, scale, 1e-6, ws, lse, st)
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[0] == 0
+    ow = OL.LayerWeights(g1=OL.widen(pb["ln1_gamma"]), b1=OL.widen(pb["ln1_beta"]), wqkv=OL.widen(pb["w_qkv"]),
+                         bqkv=OL.widen(pb["b_qkv"]), wo=OL.widen(pb["w_o"]), bo=OL.widen(pb["b_o"]),
+                         g2=OL.widen(pb["ln2_gamma"]), b2=OL.widen(pb["ln2_beta"]), w1=OL.widen(pb["w_fc1"]),
+                         bb1=OL.widen(pb["b_fc1"]), w2=OL.widen(pb["w_fc2"]), bb2=OL.widen(pb["b_fc2"]))
+    cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    ref, parts = OL.encoder_layer_fwd(x, ow, cu, H, scale, 1e-6)
+    return to_f64(y), ref, (None if lse is None else lse.cpu().double().numpy()), parts
+
+
+@pytest.mark.parametrize("counts,H,D,ffn", [([16, 49, 64, 100], 4, 64, 1024), ([300, 1, 129], 2, 80, 328),
+                                            ([1024, 256, 777], 16, 64, 4096)])
+def test_layer_matches_oracle(counts, H, D, ffn):
+    y, ref, lse, parts = _run_layer(counts, H, D, ffn, B.TRAINED)
+    assert rel_l2(y, ref) <= LAYER_REL_L2
+    assert np.abs(y - ref).max() <= 0.05 + 2.0 ** -6 * np.abs(ref).max()
+    assert np.abs(lse - parts["lse"]).max() <= 2e-2   # LSE of bf16-rounded q, k (the projections are stored as bf16)
+
+
+def test_layer_frozen_equals_trained_output():
+    y_t, ref, _, _ = _run_layer([200, 56], 4, 64, 512, B.TRAINED)
+    y_f, _, lse, _ = _run_layer([200, 56], 4, 64, 512, B.FROZEN)
+    assert lse is None and np.array_equal(y_t, y_f)
+
+
+def test_layer_argument_checks():
+    T, hidden, ffn = 64, 256, 512
+    ws = torch.empty(B.encoder_layer_workspace_bytes(T, hidden, ffn) - 256, dtype=torch.uint8, device="cuda")
+    pb = W.layer_params_bf16(5, hidden, ffn)
+    weights = B.LayerWeights.from_tensors(**{k: to_dev(v) for k, v in pb.items()})
+    x = to_dev(W.normal_bf16(5, 0, (T, hidden)))
+    y = torch.empty_like(x)
+    plan = B.seg_plan([T], B.FROZEN).to_device()
+    with pytest.raises(B.MpipeError) as e:
+        B.encoder_layer_fwd(x, y, weights, 4, ffn, plan, 0.125, 1e-6, ws)
+    assert e.value.status == B.ERR_WORKSPACE
+    with pytest.raises(B.MpipeError):
+        B.linear_fwd(x, to_dev(W.normal_bf16(5, 1, (12, hidden))), torch.empty((T, 12), dtype=torch.bfloat16, device="cuda"))
