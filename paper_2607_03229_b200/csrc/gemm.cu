@@ -8,7 +8,9 @@
 //               TMEM accumulators, so the epilogue of tile i overlaps the main loop of tile i + 1
 //   warp 2      TMEM allocation
 //   warps 4-11  epilogue: thread = output row = TMEM lane; warpgroup 0 takes columns 0..127, warpgroup 1
-//               columns 128..255; 32 columns per TMEM round trip; + bias, GELU, + residual, bf16, 16-byte stores
+//               columns 128..255; 32 columns per TMEM round trip; + bias, GELU, + residual in fp32, bf16 into a
+//               64-byte-swizzled [128 rows][32 columns] staging box (two per warpgroup), one TMA store per box --
+//               row-per-thread global stores cost 32 L1 wavefronts per instruction and bound the K = 1024 cases
 // Every mbarrier wait is bounded (status MPIPE_ERR_TIMEOUT), as in the attention kernels.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -25,7 +27,9 @@ constexpr int kGemmThreads = 384;
 constexpr int kGemmABytes = kGemmBM * kGemmBK * 2;   // 16 KB
 constexpr int kGemmBBytes = kGemmBN * kGemmBK * 2;   // 32 KB
 constexpr int kGemmStageBytes = kGemmABytes + kGemmBBytes;
-constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 1024;
+constexpr int kGemmOutBox = kGemmBM * 64;            // [128 rows][32 bf16] staging box
+constexpr int kGemmSmemOut = kGemmStages * kGemmStageBytes;   // 2 warpgroups x 2 boxes
+constexpr int kGemmSmem = kGemmSmemOut + 4 * kGemmOutBox + 1024;
 static_assert(kGemmSmem <= 227 * 1024, "shared memory budget");
 
 struct GemmParams {
@@ -47,7 +51,8 @@ struct GemmBarriers {
 // rounding of the result): two special-function ops and a degree-5 Horner chain instead of the library routine's branches.
 __device__ __forceinline__ float erf_as(float x) {
     const float ax = fabsf(x);
-    const float t = __frcp_rn(fmaf(0.3275911f, ax, 1.0f));
+    float t;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, ax, 1.0f)));
     float p = fmaf(1.061405429f, t, -1.453152027f);
     p = fmaf(p, t, 1.421413741f);
     p = fmaf(p, t, -0.284496736f);
@@ -59,7 +64,8 @@ __device__ __forceinline__ float erf_as(float x) {
 __device__ __forceinline__ float gelu_erf(float u) { return 0.5f * u * (1.0f + erf_as(u * 0.7071067811865476f)); }
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
-linear_fwd_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p) {
+linear_fwd_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
+                  const __grid_constant__ CUtensorMap map_c, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ GemmBarriers bars;
@@ -145,63 +151,98 @@ linear_fwd_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const int wg = (warp - 4) >> 2;                 // column half of the tile
         const int r = ((warp & 3) << 5) | lane;         // output row inside the tile = TMEM lane
         const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
-        uint32_t tile_it = 0;
+        const int wt = tid - (4 + 4 * wg) * 32;         // thread index inside the warpgroup
+        uint8_t* boxes = smem + kGemmSmemOut + wg * 2 * kGemmOutBox;
+        uint32_t tile_it = 0, box_it = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_it) {
+        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_it) {
+            // no early exit: the warpgroup meets at named barriers, so after a time-out it keeps walking empty tiles
             const uint32_t acc = tile_it & 1;
-            const int m = (t / p.tiles_n) * kGemmBM + r;
+            const int m0 = (t / p.tiles_n) * kGemmBM;
+            const int m = m0 + r;
             const int n_base = (t % p.tiles_n) * kGemmBN + wg * (kGemmBN / 2);
-            ok = mbar_wait(&bars.acc_full[acc], (tile_it >> 1) & 1, &abort_flag);
-            if (!ok) break;
-            tc_fence_after();
             const bool row_ok = m < p.M;
-            __nv_bfloat16* crow = p.C + int64_t(m) * p.ldc;
-            const __nv_bfloat16* rrow = p.residual != nullptr ? p.residual + int64_t(m) * p.ldr : nullptr;
-#pragma unroll 1
-            for (int c0 = 0; c0 < kGemmBN / 2; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(tmem + lane_base + acc * kGemmBN + wg * (kGemmBN / 2) + c0, v);
-                tmem_wait_ld();
-                if (c0 + 32 == kGemmBN / 2) {   // this thread's part of the accumulator is in registers
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars.acc_empty[acc]);
-                }
+            const __nv_bfloat16* rrow = (p.residual != nullptr && row_ok) ? p.residual + int64_t(m) * p.ldr : nullptr;
+            // the residual row is fetched one 32-column chunk ahead (each thread reads its own row: latency, not bandwidth)
+            uint4 res[4];
+            auto load_res = [&](int c0) {
 #pragma unroll
-                for (int g8 = 0; g8 < 4; ++g8) {   // 8 columns = 16 bytes of output
+                for (int g8 = 0; g8 < 4; ++g8) {
                     const int n = n_base + c0 + 8 * g8;
-                    if (n >= p.N) break;            // N is a multiple of 8
-                    float f[8];
+                    res[g8] = (rrow != nullptr && n < p.N) ? __ldg(reinterpret_cast<const uint4*>(rrow + n)) : make_uint4(0u, 0u, 0u, 0u);
+                }
+            };
+            if (p.residual != nullptr) load_res(0);
+            if (ok) ok = mbar_wait(&bars.acc_full[acc], (tile_it >> 1) & 1, &abort_flag);
+            tc_fence_after();
+#pragma unroll 1
+            for (int c0 = 0; c0 < kGemmBN / 2; c0 += 32, ++box_it) {
+                uint32_t v[32];
+                uint32_t out[16];
+                uint4 rcur[4];
+                if (p.residual != nullptr) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[8 * g8 + i]);
-                    if (p.bias != nullptr) {
-                        const uint4 b4 = __ldg(reinterpret_cast<const uint4*>(p.bias + n));
-                        const uint32_t bw[4] = {b4.x, b4.y, b4.z, b4.w};
+                    for (int g8 = 0; g8 < 4; ++g8) rcur[g8] = res[g8];
+                    if (c0 + 32 < kGemmBN / 2) load_res(c0 + 32);
+                }
+                if (ok) {
+                    tmem_ld32(tmem + lane_base + acc * kGemmBN + wg * (kGemmBN / 2) + c0, v);
+                    tmem_wait_ld();
+                    if (c0 + 32 == kGemmBN / 2) {   // this thread's part of the accumulator is in registers
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars.acc_empty[acc]);
+                    }
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            f[2 * i] += __uint_as_float(bw[i] << 16);
-                            f[2 * i + 1] += __uint_as_float(bw[i] & 0xffff0000u);
+                    for (int g8 = 0; g8 < 4; ++g8) {   // 8 columns = 16 bytes of output
+                        const int n = n_base + c0 + 8 * g8;
+                        const bool col_ok = n < p.N;     // N is a multiple of 8; the store clips what lies outside
+                        float f[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[8 * g8 + i]);
+                        if (p.bias != nullptr && col_ok) {
+                            const uint4 b4 = __ldg(reinterpret_cast<const uint4*>(p.bias + n));
+                            const uint32_t bw[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                f[2 * i] += __uint_as_float(bw[i] << 16);
+                                f[2 * i + 1] += __uint_as_float(bw[i] & 0xffff0000u);
+                            }
                         }
-                    }
-                    if (p.gelu) {
+                        if (p.gelu) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
-                    }
-                    if (rrow != nullptr && row_ok) {
-                        const uint4 r4 = *reinterpret_cast<const uint4*>(rrow + n);
-                        const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            f[2 * i] += __uint_as_float(rw[i] << 16);
-                            f[2 * i + 1] += __uint_as_float(rw[i] & 0xffff0000u);
+                            for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
                         }
+                        if (p.residual != nullptr) {
+                            const uint32_t rw[4] = {rcur[g8].x, rcur[g8].y, rcur[g8].z, rcur[g8].w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                f[2 * i] += __uint_as_float(rw[i] << 16);
+                                f[2 * i + 1] += __uint_as_float(rw[i] & 0xffff0000u);
+                            }
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) out[4 * g8 + i] = pack_bf16(f[2 * i], f[2 * i + 1]);
                     }
-                    if (row_ok)
-                        *reinterpret_cast<uint4*>(crow + n) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]),
-                                                                         pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+                }
+                uint8_t* box = boxes + (box_it & 1) * kGemmOutBox;
+                if (wt == 0) bulk_wait_group_read<1>();   // the store issued two boxes ago has read this box
+                named_barrier_sync(1 + wg, 128);
+                if (ok) {
+#pragma unroll
+                    for (int g8 = 0; g8 < 4; ++g8)
+                        *reinterpret_cast<uint4*>(box + r * 64 + ((g8 ^ ((r >> 1) & 3)) << 4)) =
+                            make_uint4(out[4 * g8], out[4 * g8 + 1], out[4 * g8 + 2], out[4 * g8 + 3]);
+                }
+                fence_async_smem();
+                named_barrier_sync(1 + wg, 128);
+                if (ok && wt == 0) {
+                    tma_store_3d(&map_c, box, n_base + c0, 0, m0);
+                    bulk_commit_group();
                 }
             }
         }
+        if (wt == 0) bulk_wait_group<0>();   // shared memory must outlive the copy engine's reads
     }
 
     tc_fence_before();
@@ -227,9 +268,10 @@ int32_t mpipe_linear_fwd(const void* a, const void* w, const void* bias, const v
     if ((lda % 8) != 0 || (ldw % 8) != 0 || (ldc % 8) != 0 || (residual != nullptr && (ldr % 8) != 0)) return MPIPE_ERR_UNSUPPORTED;
     if (!aligned16(a) || !aligned16(w) || !aligned16(c) || !aligned16(bias) || !aligned16(residual)) return MPIPE_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    CUtensorMap map_a, map_w;
+    CUtensorMap map_a, map_w, map_c;
     if (!make_tensor_map_thd(&map_a, a, M, 1, K, lda, lda, kGemmBK, kGemmBM, 128) ||
-        !make_tensor_map_thd(&map_w, w, N, 1, K, ldw, ldw, kGemmBK, kGemmBN, 128))
+        !make_tensor_map_thd(&map_w, w, N, 1, K, ldw, ldw, kGemmBK, kGemmBN, 128) ||
+        !make_tensor_map_thd(&map_c, c, M, 1, N, ldc, ldc, 32, kGemmBM, 64))
         return MPIPE_ERR_CUDA;
     GemmParams p;
     p.M = M; p.N = N; p.K = K;
@@ -250,7 +292,7 @@ int32_t mpipe_linear_fwd(const void* a, const void* w, const void* bias, const v
     const long long tiles = (long long)p.tiles_m * p.tiles_n;
     const int grid = int(tiles < sm_count() ? tiles : sm_count());
     profile_start(kProfileLinear, st);
-    linear_fwd_kernel<<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, p);
+    linear_fwd_kernel<<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, p);
     profile_stop(kProfileLinear, st);
     return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
 }
