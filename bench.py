@@ -393,6 +393,181 @@ def ours_arm(args):
     return 0
 
 
+# ----------------------------------------------------------------------------- encoder-layer line (--workload *_layer)
+LAYER_WORKLOADS = {"vit_l_layer": "vit_l", "qwen2vl_layer": "qwen2vl_frozen"}
+
+
+def layer_flops(w, ffn):
+    """Algorithmic FLOPs of one layer forward: the four projections (2 * T * in * out each) + attention 4 * H * D * sum n^2."""
+    hidden = w.n_heads * w.head_dim
+    gemm = 2.0 * w.total_tokens * hidden * (3 * hidden + hidden + 2 * ffn)
+    return gemm, gemm + w.flops(True, False)
+
+
+def layer_arm(args):
+    """The whole packed encoder layer forward (frozen mode: the layer a frozen encoder executes per microbatch) through
+    mpipe_encoder_layer_fwd.  Same line format; `roofline` covers linear_fwd_kernel over the layer's four projections."""
+    import torch
+    from paper_2607_03229_b200 import binding as B
+    from paper_2607_03229_b200 import dist as D
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    rank, local_rank, world = D.init("nccl")
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch N>1 with torchrun, one rank per GPU")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    B.load()
+    peaks, peak_kind = load_peaks()
+    base = LAYER_WORKLOADS[_WORKLOAD_NAME]
+    w = WORKLOADS[base](D.rank_seed(W.BASE_SEED + 2, rank))
+    T, Hh, Dh = w.total_tokens, w.n_heads, w.head_dim
+    hidden, ffn = Hh * Dh, 4 * Hh * Dh
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(w.seed)
+
+    def rnd(shape, std, mean=0.0):
+        return (torch.randn(shape, device=dev, generator=gen) * std + mean).to(torch.bfloat16)
+
+    params = {"ln1_gamma": rnd((hidden,), 0.1, 1.0), "ln1_beta": rnd((hidden,), 0.1), "w_qkv": rnd((3 * hidden, hidden), hidden ** -0.5),
+              "b_qkv": rnd((3 * hidden,), 0.1), "w_o": rnd((hidden, hidden), hidden ** -0.5), "b_o": rnd((hidden,), 0.1),
+              "ln2_gamma": rnd((hidden,), 0.1, 1.0), "ln2_beta": rnd((hidden,), 0.1), "w_fc1": rnd((ffn, hidden), hidden ** -0.5),
+              "b_fc1": rnd((ffn,), 0.1), "w_fc2": rnd((hidden, ffn), ffn ** -0.5), "b_fc2": rnd((hidden,), 0.1)}
+    weights = B.LayerWeights.from_tensors(**params)
+    x = rnd((T, hidden), 1.0)
+    y = torch.empty_like(x)
+    plan = B.seg_plan(w.patch_counts, B.FROZEN).to_device(dev)
+    ws = torch.empty(B.encoder_layer_workspace_bytes(T, hidden, ffn), dtype=torch.uint8, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+    step = lambda xin=x, yout=y, st=None: B.encoder_layer_fwd(xin, yout, weights, Hh, ffn, plan, w.softmax_scale, 1e-6, ws, None,
+                                                             status, st)
+    K, Wm = args.steps, max(args.warmup, 3)
+    for _ in range(Wm):
+        step()
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0, f"device status {status.tolist()}"
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid) if hasattr(
+        torch.cuda.get_device_properties(dev), "uuid") else str(local_rank)
+    sampler = ClockSampler(uuid)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    D.barrier()
+    sampler.start()
+    time.sleep(0.15)
+    torch.cuda.synchronize()
+    t_begin = time.perf_counter()
+    e0.record()
+    for _ in range(K):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    t_end = time.perf_counter()
+    D.barrier()
+    clocks = sampler.stop(t_begin, t_end)
+    ms_step = e0.elapsed_time(e1) / K
+
+    # ---- per-kernel durations: the same launches, one at a time, each between its own pair of events
+    norm = torch.empty_like(x); qkv = torch.empty((T, 3 * hidden), dtype=torch.bfloat16, device=dev)
+    attn = torch.empty_like(x); x1 = torch.empty_like(x); fc1 = torch.empty((T, ffn), dtype=torch.bfloat16, device=dev)
+    q3 = qkv.view(T, 3, Hh, Dh)
+    stages = [
+        ("layernorm", lambda: B.layernorm_fwd(x, params["ln1_gamma"], params["ln1_beta"], norm, 1e-6)),
+        ("linear_qkv", lambda: B.linear_fwd(norm, params["w_qkv"], qkv, params["b_qkv"], None, False, status)),
+        ("attn_fwd", lambda: B.varlen_attn_fwd(q3[:, 0], q3[:, 1], q3[:, 2], attn.view(T, Hh, Dh), None, plan, w.softmax_scale, status)),
+        ("linear_out", lambda: B.linear_fwd(attn, params["w_o"], x1, params["b_o"], x, False, status)),
+        ("linear_fc1", lambda: B.linear_fwd(norm, params["w_fc1"], fc1, params["b_fc1"], None, True, status)),
+        ("linear_fc2", lambda: B.linear_fwd(fc1, params["w_fc2"], y, params["b_fc2"], x1, False, status)),
+    ]
+    Kk = min(K, 20)
+    kern_ms = {}
+    for name, fn in stages:
+        fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(Kk):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        kern_ms[name] = a.elapsed_time(b) / Kk
+    assert int(status[0]) == 0
+
+    # ---- end to end: x from pinned host memory, y back to the host, every step
+    Ke = 1 if args.profile_mode else min(K, 20)
+    hx = torch.empty(tuple(x.shape), dtype=torch.bfloat16).pin_memory()
+    hx.copy_(x)
+    hy = torch.empty(tuple(y.shape), dtype=torch.bfloat16).pin_memory()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    f0.record()
+    for _ in range(Ke):
+        x.copy_(hx, non_blocking=True)
+        step()
+        hy.copy_(y, non_blocking=True)
+    f1.record()
+    torch.cuda.synchronize()
+    ms_e2e = f0.elapsed_time(f1) / Ke
+
+    gemm_flops, flops_step = layer_flops(w, ffn)
+    (ms_step_mx, ms_e2e_mx), (flops_all, launches) = D.reduce_max_sum([ms_step, ms_e2e], [flops_step, float(7 * K)], device=dev)
+    if rank == 0:
+        value = flops_all / (ms_step_mx * 1e-3) / 1e12
+        lin_ms = sum(v for k_, v in kern_ms.items() if k_.startswith("linear"))
+        lin_tf = gemm_flops / (lin_ms * 1e-3) / 1e12
+        peak_tf = peaks["bf16_tflops_sustained"]
+        line = {
+            "metric": "packed encoder layer forward (norms, QKV/out/MLP projections, varlen attention) TFLOP/s (1 B200)",
+            "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": ms_step_mx,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": _WORKLOAD_NAME + ": one pre-norm encoder layer over the packed microbatch of " +
+                       WORKLOAD_TEXT[base].split(":")[0] + f", hidden {hidden}, ffn {ffn}, frozen (forward only); one microbatch per GPU",
+                       "tokens_rank0": T, "sum_n2_rank0": w.sum_n2, "heads": Hh, "head_dim": Dh,
+                       "l2": "inputs_exceed_l2", "step": "mpipe_encoder_layer_fwd: LN, QKV, attention, out-proj + residual, LN, fc1 + GELU, fc2 + residual"},
+            "breakdown": {"kernel_ms": kern_ms, "linear_tflops": lin_tf,
+                          "attn_fwd_tflops": w.flops(True, False) / (kern_ms["attn_fwd"] * 1e-3) / 1e12,
+                          "layernorm_gbs": 4.0 * T * hidden / (kern_ms["layernorm"] * 1e-3) / 1e9,
+                          "frac_of_bf16_peak": {"measured_sustained": value / world / peak_tf, "measured_burst": value / world / peaks["bf16_tflops"],
+                                                "nominal_2250": value / world / NOMINAL_BF16_TFLOPS}},
+            "roofline": {"kernel": "linear_fwd_kernel (4 launches per step)", "bound": "tensor", "achieved": lin_tf, "peak": peak_tf,
+                         "unit": "TFLOP/s", "frac": lin_tf / peak_tf, "peak_kind": f"{peak_kind}, sustained bf16 GEMM", "traffic": None},
+            "e2e": {"value": flops_all / (ms_e2e_mx * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e_mx, "steps": Ke,
+                    "h2d_bytes_per_step": int(hx.numel() * 2), "d2h_bytes_per_step": int(hy.numel() * 2)},
+            "gpu_launches": int(launches), "clocks": clocks,
+        }
+        if world == 1 and not args.profile_mode:
+            line["cpu_baseline"] = layer_cpu_baseline(w, hidden, ffn)
+        if args.profile_mode:
+            line["profile_mode"] = True
+        print(json.dumps(line))
+    D.shutdown()
+    return 0
+
+
+def layer_cpu_baseline(w, hidden, ffn):
+    """The layer oracle on the first segments of the workload (a few thousand tokens), one pass on the host cores."""
+    import oracle
+    from oracle import layer as OL
+    m, tok = 0, 0
+    while m < len(w.patch_counts) and (m == 0 or tok + w.patch_counts[m] <= 20000):
+        tok += w.patch_counts[m]
+        m += 1
+    counts = w.patch_counts[:m]
+    pb = W.layer_params_bf16(w.seed, hidden, ffn)
+    ow = OL.LayerWeights(g1=OL.widen(pb["ln1_gamma"]), b1=OL.widen(pb["ln1_beta"]), wqkv=OL.widen(pb["w_qkv"]), bqkv=OL.widen(pb["b_qkv"]),
+                         wo=OL.widen(pb["w_o"]), bo=OL.widen(pb["b_o"]), g2=OL.widen(pb["ln2_gamma"]), b2=OL.widen(pb["ln2_beta"]),
+                         w1=OL.widen(pb["w_fc1"]), bb1=OL.widen(pb["b_fc1"]), w2=OL.widen(pb["w_fc2"]), bb2=OL.widen(pb["b_fc2"]))
+    x = W.normal_bf16(w.seed, 0, (tok, hidden))
+    cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    oracle.build()
+    t0 = time.perf_counter()
+    OL.encoder_layer_fwd(x, ow, cu, w.n_heads, w.softmax_scale, 1e-6)
+    dt = time.perf_counter() - t0
+    flops = 2.0 * tok * hidden * (4 * hidden + 2 * ffn) + 4.0 * hidden * float(sum(n * n for n in counts))
+    return {"value": flops / dt / 1e12, "unit": UNIT, "cores": oracle.n_threads(), "kind": "oracle", "seconds": dt,
+            "sample": f"first {m} of {len(w.patch_counts)} segments ({tok} tokens, {flops:.3g} algorithmic FLOPs), one pass"}
+
+
+
 def cpu_baseline(w):
     """The oracle as it stands on the host cores, on a bounded sample (about 10-20 s of CPU work)."""
     import oracle
@@ -410,7 +585,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
-    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="vit_l",
+    ap.add_argument("--workload", choices=sorted(WORKLOADS) + sorted(LAYER_WORKLOADS), default="vit_l",
                     help="which synthetic configuration to run (default: vit_l, the one the metric is quoted on; "
                          "the others are for the per-config results table)")
     ap.add_argument("--profile-mode", action="store_true",
@@ -419,6 +594,11 @@ def main():
     args = ap.parse_args()
     global _WORKLOAD_NAME
     _WORKLOAD_NAME = args.workload
+    if args.workload in LAYER_WORKLOADS:
+        if args.impl == "reference":
+            print(json.dumps({"impl": "reference", "unavailable": "the reference arm covers the attention metric only (default workload)"}))
+            return 0
+        return layer_arm(args)
     if args.impl == "reference":
         return reference_arm(args)
     return ours_arm(args)

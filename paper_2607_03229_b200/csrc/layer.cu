@@ -101,10 +101,16 @@ int32_t mpipe_layernorm_fwd(const void* x, const void* gamma, const void* beta, 
     const auto* bp = static_cast<const __nv_bfloat16*>(beta);
     auto* yp = static_cast<__nv_bfloat16*>(y);
     profile_start(kProfileLayerNorm, st);
-    if (hidden <= 4 * 256)
-        layernorm_kernel<4><<<grid, 256, 0, st>>>(xp, gp, bp, yp, n_tokens, hidden, ldx, ldy, eps);
-    else
-        layernorm_kernel<kLnMaxChunks><<<grid, 256, 0, st>>>(xp, gp, bp, yp, n_tokens, hidden, ldx, ldy, eps);
+    const int chunks = cdiv(hidden, 256);   // 16-byte chunks per lane: instantiate what the row length needs, not the maximum
+#define MPIPE_LN_LAUNCH(C) layernorm_kernel<C><<<grid, 256, 0, st>>>(xp, gp, bp, yp, n_tokens, hidden, ldx, ldy, eps)
+    if (chunks <= 1) MPIPE_LN_LAUNCH(1);
+    else if (chunks <= 2) MPIPE_LN_LAUNCH(2);
+    else if (chunks <= 3) MPIPE_LN_LAUNCH(3);
+    else if (chunks <= 4) MPIPE_LN_LAUNCH(4);
+    else if (chunks <= 5) MPIPE_LN_LAUNCH(5);
+    else if (chunks <= 6) MPIPE_LN_LAUNCH(6);
+    else MPIPE_LN_LAUNCH(kLnMaxChunks);
+#undef MPIPE_LN_LAUNCH
     profile_stop(kProfileLayerNorm, st);
     return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
 }
