@@ -440,8 +440,11 @@ def layer_arm(args):
     plan = B.seg_plan(w.patch_counts, B.FROZEN).to_device(dev)
     ws = torch.empty(B.encoder_layer_workspace_bytes(T, hidden, ffn), dtype=torch.uint8, device=dev)
     status = torch.zeros(4, dtype=torch.int32, device=dev)
+    rope = None
+    if base.startswith("qwen2vl"):   # the Qwen2-VL-like configuration carries a 2-D rotary encoding of q and k
+        rope = tuple(torch.from_numpy(t).to(dev) for t in W.rope2d_tables(w.patch_counts, Dh))
     step = lambda xin=x, yout=y, st=None: B.encoder_layer_fwd(xin, yout, weights, Hh, ffn, plan, w.softmax_scale, 1e-6, ws, None,
-                                                             status, st)
+                                                             status, st, rope)
     K, Wm = args.steps, max(args.warmup, 3)
     for _ in range(Wm):
         step()
@@ -473,6 +476,7 @@ def layer_arm(args):
     stages = [
         ("layernorm", lambda: B.layernorm_fwd(x, params["ln1_gamma"], params["ln1_beta"], norm, 1e-6)),
         ("linear_qkv", lambda: B.linear_fwd(norm, params["w_qkv"], qkv, params["b_qkv"], None, False, status)),
+        ("rope", (lambda: B.rope_apply(qkv, rope[0], rope[1], Hh, Dh)) if rope is not None else None),
         ("attn_fwd", lambda: B.varlen_attn_fwd(q3[:, 0], q3[:, 1], q3[:, 2], attn.view(T, Hh, Dh), None, plan, w.softmax_scale, status)),
         ("linear_out", lambda: B.linear_fwd(attn, params["w_o"], x1, params["b_o"], x, False, status)),
         ("linear_fc1", lambda: B.linear_fwd(norm, params["w_fc1"], fc1, params["b_fc1"], None, True, status)),
@@ -481,6 +485,8 @@ def layer_arm(args):
     Kk = min(K, 20)
     kern_ms = {}
     for name, fn in stages:
+        if fn is None:
+            continue
         fn()
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -509,7 +515,8 @@ def layer_arm(args):
     ms_e2e = f0.elapsed_time(f1) / Ke
 
     gemm_flops, flops_step = layer_flops(w, ffn)
-    (ms_step_mx, ms_e2e_mx), (flops_all, launches) = D.reduce_max_sum([ms_step, ms_e2e], [flops_step, float(7 * K)], device=dev)
+    (ms_step_mx, ms_e2e_mx), (flops_all, launches) = D.reduce_max_sum(
+        [ms_step, ms_e2e], [flops_step, float((8 if rope is not None else 7) * K)], device=dev)
     if rank == 0:
         value = flops_all / (ms_step_mx * 1e-3) / 1e12
         lin_ms = sum(v for k_, v in kern_ms.items() if k_.startswith("linear"))
@@ -522,7 +529,7 @@ def layer_arm(args):
             "config": {"workload": _WORKLOAD_NAME + ": one pre-norm encoder layer over the packed microbatch of " +
                        WORKLOAD_TEXT[base].split(":")[0] + f", hidden {hidden}, ffn {ffn}, frozen (forward only); one microbatch per GPU",
                        "tokens_rank0": T, "sum_n2_rank0": w.sum_n2, "heads": Hh, "head_dim": Dh,
-                       "l2": "inputs_exceed_l2", "step": "mpipe_encoder_layer_fwd: LN, QKV, attention, out-proj + residual, LN, fc1 + GELU, fc2 + residual"},
+                       "l2": "inputs_exceed_l2", "step": "mpipe_encoder_layer_fwd: LN, QKV" + (", 2-D rope" if rope is not None else "") + ", attention, out-proj + residual, LN, fc1 + GELU, fc2 + residual"},
             "breakdown": {"kernel_ms": kern_ms, "linear_tflops": lin_tf,
                           "attn_fwd_tflops": w.flops(True, False) / (kern_ms["attn_fwd"] * 1e-3) / 1e12,
                           "layernorm_gbs": 4.0 * T * hidden / (kern_ms["layernorm"] * 1e-3) / 1e9,

@@ -228,14 +228,23 @@ int32_t mpipe_validate_positions(const int32_t* positions, int32_t n, int32_t n_
  *                        N and K multiples of 8 (MPIPE_ERR_UNSUPPORTED otherwise); M == 0 launches nothing.
  *   mpipe_layernorm_fwd  y[t, :] = (x[t, :] - mean_t) * rsqrt(var_t + eps) * gamma + beta, biased variance, fp32
  *                        statistics; bf16 in and out, hidden a multiple of 8 and <= 2048.
+ *   mpipe_rope_apply     rotary position encoding, rotate-half form, in place on q and k of a packed projection:
+ *                        for each token t, head h and pair j < head_dim/2:
+ *                          (x[j], x[j + head_dim/2]) <- (x[j] cos[t,j] - x[j+hd/2] sin[t,j], x[j+hd/2] cos[t,j] + x[j] sin[t,j]).
+ *                        qk: bf16 device, q of token t at qk + t*tok_stride, its k at + k_offset, heads contiguous
+ *                        (head stride = head_dim); cos/sin: fp32 device [n_tokens, head_dim/2] -- the caller builds
+ *                        them (1-D, or 2-D with one half of the pairs per image axis); head_dim a multiple of 16.
+ *                        The paper does not name a position encoding; this is the one the Qwen2-VL-like
+ *                        configuration implies.  fp32 arithmetic, one rounding to bf16.
  *   mpipe_encoder_layer_fwd
  *        a = LN(x; ln1) ; qkv = a Wqkv^T + bqkv (columns q | k | v, each [n_heads][head_dim]) ;
+ *        q, k <- rope(q, k) when rope_cos / rope_sin are given (both NULL: none) ;
  *        o = per-image softmax attention (mpipe_varlen_attn_fwd on strided views of qkv, same plan arguments) ;
  *        x1 = x + o Wo^T + bo ; m = LN(x1; ln2) ; y = x1 + GELU(m W1^T + b1) W2^T + b2.
  *        x, y: bf16 [n_tokens, hidden] contiguous, device; y may not alias x.  Weights: device bf16, nn.Linear
  *        layout [out, in], contiguous.  lse: fp32 [n_heads, n_tokens] when TRAINED, ignored when FROZEN.
  *        workspace: device, 256-byte aligned, >= mpipe_encoder_layer_workspace_bytes (MPIPE_ERR_WORKSPACE);
- *        caller-owned, contents undefined afterwards.  Seven launches on `stream`, no allocation, no sync.
+ *        caller-owned, contents undefined afterwards.  Seven launches (eight with rope) on `stream`, no allocation, no sync.
  *        head_dim = hidden / n_heads must be one the attention kernels support (64, 80).
  * Device-side findings (a bounded wait that ran out) are reported through status_buf as for the attention calls.
  */
@@ -255,12 +264,15 @@ int32_t mpipe_linear_fwd(const void* a, const void* w, const void* bias, const v
                          int32_t* status_buf, void* stream);
 int32_t mpipe_layernorm_fwd(const void* x, const void* gamma, const void* beta, void* y, int32_t n_tokens,
                             int32_t hidden, int64_t ldx, int64_t ldy, float eps, void* stream);
+int32_t mpipe_rope_apply(void* qk, int64_t tok_stride, int64_t k_offset, const float* cos_table, const float* sin_table,
+                         int32_t n_tokens, int32_t n_heads, int32_t head_dim, void* stream);
 size_t mpipe_encoder_layer_workspace_bytes(int32_t n_tokens, int32_t hidden, int32_t ffn);
 int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weights_t* w, int32_t n_tokens,
                                 int32_t hidden, int32_t n_heads, int32_t ffn, const int32_t* cu_seqlens_dev,
                                 int32_t n_seg, int32_t max_seqlen, const mpipe_work_item_t* fwd_items_dev,
-                                int32_t n_fwd_items, float softmax_scale, float ln_eps, int32_t mode, float* lse,
-                                void* workspace, size_t workspace_bytes, int32_t* status_buf, void* stream);
+                                int32_t n_fwd_items, float softmax_scale, float ln_eps, const float* rope_cos,
+                                const float* rope_sin, int32_t mode, float* lse, void* workspace,
+                                size_t workspace_bytes, int32_t* status_buf, void* stream);
 
 /*
  * Measurement aid (no counterpart in the paper; its cost model weights each compute event with one

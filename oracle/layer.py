@@ -6,6 +6,7 @@ packed varlen token matrix x[T, hidden]:
 
     a  = LayerNorm(x; g1, b1)
     qkv = a Wqkv^T + bqkv                      -> q, k, v as [T, H, D]   (column block order q | k | v)
+    q, k = rope(q), rope(k)                    optional rotate-half rotary encoding, angles given per token and pair
     o  = per-image softmax attention (oracle.attn_fwd, block-diagonal over cu_seqlens)
     x1 = x + o Wo^T + bo
     m  = LayerNorm(x1; g2, b2)
@@ -59,6 +60,16 @@ def gelu(u: np.ndarray) -> np.ndarray:
     return 0.5 * u * (1.0 + _erf(u / math.sqrt(2.0)))
 
 
+def rope(x: np.ndarray, cos: np.ndarray, sin: np.ndarray) -> np.ndarray:
+    """Rotate-half rotary encoding.  x: [T, H, D]; cos, sin: [T, D/2] (angle of pair j of token t).  The pair is
+    (x[..., j], x[..., j + D/2]) and it is rotated by that angle: a plain 2-D rotation per pair."""
+    x = np.asarray(x, dtype=np.float64)
+    half = x.shape[-1] // 2
+    x1, x2 = x[..., :half], x[..., half:]
+    c, s = np.asarray(cos, dtype=np.float64)[:, None, :], np.asarray(sin, dtype=np.float64)[:, None, :]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
 @dataclass
 class LayerWeights:
     """fp64 views of the layer's parameters (nn.Linear layout [out, in])."""
@@ -76,7 +87,7 @@ class LayerWeights:
     bb2: np.ndarray
 
 
-def encoder_layer_fwd(x, w: LayerWeights, cu_seqlens, n_heads: int, scale: float, eps: float):
+def encoder_layer_fwd(x, w: LayerWeights, cu_seqlens, n_heads: int, scale: float, eps: float, rope_tables=None):
     """The whole block.  x: [T, hidden] (uint16 bf16 bits or fp64).  Returns (y, parts) with parts a dict of
     the intermediates (a, qkv, o, x1, m, f) in fp64 for stage-wise comparisons."""
     x = widen(x)
@@ -85,6 +96,8 @@ def encoder_layer_fwd(x, w: LayerWeights, cu_seqlens, n_heads: int, scale: float
     a = layernorm(x, w.g1, w.b1, eps)
     qkv = linear(a, w.wqkv, w.bqkv)
     q, k, v = (np.ascontiguousarray(qkv[:, i * hidden:(i + 1) * hidden].reshape(T, n_heads, D)) for i in range(3))
+    if rope_tables is not None:   # (cos, sin) [T, D/2]: q and k are rotated, v is not
+        q, k = rope(q, *rope_tables), rope(k, *rope_tables)
     o, lse = attn_fwd(q, k, v, cu_seqlens, scale)
     x1 = x + linear(o.reshape(T, hidden), w.wo, w.bo)
     m = layernorm(x1, w.g2, w.b2, eps)

@@ -36,7 +36,8 @@ _SIGNATURES = {
     "mpipe_layernorm_fwd": (_i32, [_vp, _vp, _vp, _vp, _i32, _i32, _i64, _i64, _f32, _vp]),
     "mpipe_encoder_layer_workspace_bytes": (_sz, [_i32, _i32, _i32]),
     "mpipe_encoder_layer_fwd": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _i32, _i32, _vp, _i32, _f32, _f32,
-                                       _i32, _vp, _vp, _sz, _vp, _vp]),
+                                       _vp, _vp, _i32, _vp, _vp, _sz, _vp, _vp]),
+    "mpipe_rope_apply": (_i32, [_vp, _i64, _i64, _vp, _vp, _i32, _i32, _i32, _vp]),
     "mpipe_fwd_tile_rows": (_i32, []),
     "mpipe_bwd_tile_rows": (_i32, []),
     "mpipe_seg_plan": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -281,14 +282,28 @@ def encoder_layer_workspace_bytes(n_tokens: int, hidden: int, ffn: int) -> int:
     return load().mpipe_encoder_layer_workspace_bytes(n_tokens, hidden, ffn)
 
 
+def rope_apply(qkv, cos, sin, n_heads: int, head_dim: int, stream=None) -> None:
+    """mpipe_rope_apply in place on the q and k column blocks of a packed projection qkv [T, 3*hidden] (bf16, CUDA);
+    cos, sin: fp32 [T, head_dim/2] contiguous CUDA tensors."""
+    T = qkv.shape[0]
+    hidden = n_heads * head_dim
+    assert qkv.shape[1] == 3 * hidden and qkv.dtype == torch.bfloat16 and qkv.stride(1) == 1
+    for t in (cos, sin):
+        assert t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == (T, head_dim // 2)
+    st = load().mpipe_rope_apply(_ptr(qkv), qkv.stride(0), hidden, _ptr(cos), _ptr(sin), T, n_heads, head_dim, _stream(stream))
+    _check(st, "mpipe_rope_apply")
+
+
 def encoder_layer_fwd(x, y, weights: LayerWeights, n_heads: int, ffn: int, plan: SegPlan, softmax_scale: float,
-                      ln_eps: float, workspace, lse=None, status_buf=None, stream=None) -> None:
-    """mpipe_encoder_layer_fwd: x, y bf16 [T, hidden] contiguous CUDA tensors; lse fp32 [H, T] for a trained plan."""
+                      ln_eps: float, workspace, lse=None, status_buf=None, stream=None, rope=None) -> None:
+    """mpipe_encoder_layer_fwd: x, y bf16 [T, hidden] contiguous CUDA tensors; lse fp32 [H, T] for a trained plan;
+    rope = (cos, sin) fp32 [T, head_dim/2] CUDA tensors or None."""
     T, hidden = x.shape
     assert x.is_contiguous() and y.is_contiguous() and tuple(y.shape) == (T, hidden) and x.dtype == y.dtype == torch.bfloat16
     st = load().mpipe_encoder_layer_fwd(
         _ptr(x), _ptr(y), ctypes.addressof(weights), T, hidden, n_heads, ffn, _ptr(plan.cu_seqlens_dev), plan.n_seg,
-        plan.max_seqlen, _ptr(plan.fwd_items_dev), int(plan.fwd_items.size), softmax_scale, ln_eps, plan.mode, _ptr(lse),
+        plan.max_seqlen, _ptr(plan.fwd_items_dev), int(plan.fwd_items.size), softmax_scale, ln_eps,
+        _ptr(None if rope is None else rope[0]), _ptr(None if rope is None else rope[1]), plan.mode, _ptr(lse),
         _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_encoder_layer_fwd")
 

@@ -80,6 +80,42 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const __nv_bfloat16* __r
     }
 }
 
+// Rotary position encoding in the rotate-half form, in place on q and k inside the packed projection:
+// (x1, x2) -> (x1 cos - x2 sin, x2 cos + x1 sin) for x1 = x[0 .. D/2), x2 = x[D/2 .. D), angles per token and pair.
+// One thread per (token, q|k, head, 8-pair chunk): 2 x 16 bytes in, 2 x 16 bytes out, 2 x 32 bytes of table.
+__global__ void __launch_bounds__(256) rope_kernel(__nv_bfloat16* __restrict__ qk, int64_t tok_stride, int64_t k_offset,
+                                                   const float* __restrict__ cos_t, const float* __restrict__ sin_t, int32_t T,
+                                                   int32_t n_heads, int32_t head_dim) {
+    const int half = head_dim >> 1, chunks = half >> 3;
+    const int64_t idx = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int64_t total = int64_t(T) * 2 * n_heads * chunks;
+    if (idx >= total) return;
+    const int c = int(idx % chunks);
+    const int h = int((idx / chunks) % n_heads);
+    const int which = int((idx / (int64_t(chunks) * n_heads)) & 1);
+    const int64_t t = idx / (int64_t(chunks) * n_heads * 2);
+    __nv_bfloat16* x = qk + t * tok_stride + which * k_offset + int64_t(h) * head_dim + c * 8;
+    const uint4 a = *reinterpret_cast<const uint4*>(x), b = *reinterpret_cast<const uint4*>(x + half);
+    const float4* cp = reinterpret_cast<const float4*>(cos_t + t * half + c * 8);
+    const float4* sp = reinterpret_cast<const float4*>(sin_t + t * half + c * 8);
+    const float4 c0 = __ldg(cp), c1 = __ldg(cp + 1), s0 = __ldg(sp), s1 = __ldg(sp + 1);
+    const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+    const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+    uint32_t oa[4], ob[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float x1l = __uint_as_float(aw[j] << 16), x1h = __uint_as_float(aw[j] & 0xffff0000u);
+        const float x2l = __uint_as_float(bw[j] << 16), x2h = __uint_as_float(bw[j] & 0xffff0000u);
+        const __nv_bfloat162 o1 = __floats2bfloat162_rn(x1l * cs[2 * j] - x2l * sn[2 * j], x1h * cs[2 * j + 1] - x2h * sn[2 * j + 1]);
+        const __nv_bfloat162 o2 = __floats2bfloat162_rn(x2l * cs[2 * j] + x1l * sn[2 * j], x2h * cs[2 * j + 1] + x1h * sn[2 * j + 1]);
+        oa[j] = *reinterpret_cast<const uint32_t*>(&o1);
+        ob[j] = *reinterpret_cast<const uint32_t*>(&o2);
+    }
+    *reinterpret_cast<uint4*>(x) = make_uint4(oa[0], oa[1], oa[2], oa[3]);
+    *reinterpret_cast<uint4*>(x + half) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+}
+
 static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 
 }  // namespace mpipe
@@ -115,6 +151,22 @@ int32_t mpipe_layernorm_fwd(const void* x, const void* gamma, const void* beta, 
     return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
 }
 
+int32_t mpipe_rope_apply(void* qk, int64_t tok_stride, int64_t k_offset, const float* cos_table, const float* sin_table,
+                         int32_t n_tokens, int32_t n_heads, int32_t head_dim, void* stream) {
+    using namespace mpipe;
+    if (n_tokens < 0 || n_heads <= 0 || head_dim <= 0) return MPIPE_ERR_INVALID_ARG;
+    if (n_tokens == 0) return MPIPE_OK;
+    if (qk == nullptr || cos_table == nullptr || sin_table == nullptr) return MPIPE_ERR_INVALID_ARG;
+    if ((head_dim % 16) != 0 || (tok_stride % 8) != 0 || (k_offset % 8) != 0) return MPIPE_ERR_UNSUPPORTED;
+    if (!aligned16(qk) || !aligned16(cos_table) || !aligned16(sin_table)) return MPIPE_ERR_UNSUPPORTED;
+    const int64_t total = int64_t(n_tokens) * 2 * n_heads * (head_dim / 16);
+    const int64_t blocks = (total + 255) / 256;
+    if (blocks > 0x7fffffffLL) return MPIPE_ERR_UNSUPPORTED;
+    rope_kernel<<<int(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<__nv_bfloat16*>(qk), tok_stride, k_offset, cos_table,
+                                                                           sin_table, n_tokens, n_heads, head_dim);
+    return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
+}
+
 size_t mpipe_encoder_layer_workspace_bytes(int32_t n_tokens, int32_t hidden, int32_t ffn) {
     using namespace mpipe;
     if (n_tokens <= 0 || hidden <= 0 || ffn <= 0) return 0;
@@ -127,8 +179,8 @@ size_t mpipe_encoder_layer_workspace_bytes(int32_t n_tokens, int32_t hidden, int
 int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weights_t* w, int32_t n_tokens, int32_t hidden,
                                 int32_t n_heads, int32_t ffn, const int32_t* cu_seqlens_dev, int32_t n_seg, int32_t max_seqlen,
                                 const mpipe_work_item_t* fwd_items_dev, int32_t n_fwd_items, float softmax_scale, float ln_eps,
-                                int32_t mode, float* lse, void* workspace, size_t workspace_bytes, int32_t* status_buf,
-                                void* stream) {
+                                const float* rope_cos, const float* rope_sin, int32_t mode, float* lse, void* workspace,
+                                size_t workspace_bytes, int32_t* status_buf, void* stream) {
     using namespace mpipe;
     if (n_tokens < 0 || hidden <= 0 || n_heads <= 0 || ffn <= 0 || w == nullptr) return MPIPE_ERR_INVALID_ARG;
     if (mode != MPIPE_ENC_FROZEN && mode != MPIPE_ENC_TRAINED) return MPIPE_ERR_INVALID_ARG;
@@ -148,6 +200,10 @@ int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weight
     if ((rc = mpipe_layernorm_fwd(x, w->ln1_gamma, w->ln1_beta, norm, n_tokens, hidden, hidden, hidden, ln_eps, stream)) != MPIPE_OK) return rc;
     if ((rc = mpipe_linear_fwd(norm, w->w_qkv, w->b_qkv, nullptr, qkv, n_tokens, 3 * hidden, hidden, hidden, hidden, 0,
                                3 * int64_t(hidden), 0, status_buf, stream)) != MPIPE_OK) return rc;
+    if ((rope_cos == nullptr) != (rope_sin == nullptr)) return MPIPE_ERR_INVALID_ARG;
+    if (rope_cos != nullptr &&
+        (rc = mpipe_rope_apply(qkv, 3 * int64_t(hidden), hidden, rope_cos, rope_sin, n_tokens, n_heads, head_dim, stream)) != MPIPE_OK)
+        return rc;
     const uint8_t* q = qkv;
     const uint8_t* k = qkv + size_t(hidden) * 2;
     const uint8_t* v = qkv + size_t(hidden) * 4;

@@ -126,6 +126,25 @@ def layer_params_bf16(seed: int, hidden: int, ffn: int) -> dict:
     return out
 
 
+def rope2d_tables(patch_counts, head_dim: int, theta: float = 10000.0):
+    """cos / sin tables fp32 [T, head_dim/2] of a 2-D rotary encoding for packed images: image i is laid out as a
+    grid of width ceil(sqrt(n_i)) (row-major, last row ragged); the first head_dim/4 pairs turn with the row
+    index, the other head_dim/4 with the column index, frequencies theta^(-k / (head_dim/4)).  Input recipe only:
+    the tables are inputs of both the kernel and the oracle."""
+    quarter = head_dim // 4
+    inv = (theta ** (-np.arange(quarter, dtype=np.float64) / quarter))
+    rows, cols = [], []
+    for n in patch_counts:
+        wdt = int(np.ceil(np.sqrt(n)))
+        idx = np.arange(n)
+        rows.append(idx // wdt)
+        cols.append(idx % wdt)
+    r = np.concatenate(rows).astype(np.float64)[:, None] * inv[None, :]
+    c = np.concatenate(cols).astype(np.float64)[:, None] * inv[None, :]
+    ang = np.concatenate([r, c], axis=1)
+    return np.cos(ang).astype(np.float32), np.sin(ang).astype(np.float32)
+
+
 # --------------------------------------------------------------------------------------
 # Structure recipes
 # --------------------------------------------------------------------------------------

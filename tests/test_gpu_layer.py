@@ -66,7 +66,24 @@ def test_layernorm_matches_oracle(T, hidden):
     _check_close(to_f64(y), ref, atol=1e-4)
 
 
-def _run_layer(counts, H, D, ffn, mode, seed=21):
+@pytest.mark.parametrize("counts,H,D", [([5, 1, 30], 2, 64), ([300, 77], 3, 80), ([1000], 16, 64)])
+def test_rope_matches_oracle(counts, H, D):
+    T, hidden = sum(counts), H * D
+    qkv = W.normal_bf16(14, 0, (T, 3 * hidden))
+    cos, sin = W.rope2d_tables(counts, D)
+    dev = to_dev(qkv)
+    B.rope_apply(dev, torch.from_numpy(cos).cuda(), torch.from_numpy(sin).cuda(), H, D)
+    torch.cuda.synchronize()
+    got = to_f64(dev)
+    ref = OL.widen(qkv).copy()
+    for i in range(2):   # q and k are rotated, v stays
+        blk = ref[:, i * hidden:(i + 1) * hidden].reshape(T, H, D)
+        ref[:, i * hidden:(i + 1) * hidden] = OL.rope(blk, cos.astype(np.float64), sin.astype(np.float64)).reshape(T, hidden)
+    _check_close(got, ref, atol=1e-6)
+    assert np.array_equal(got[:, 2 * hidden:], OL.widen(qkv)[:, 2 * hidden:])
+
+
+def _run_layer(counts, H, D, ffn, mode, seed=21, rope=False):
     hidden = H * D
     T = sum(counts)
     pb = W.layer_params_bf16(seed, hidden, ffn)
@@ -78,7 +95,9 @@ def _run_layer(counts, H, D, ffn, mode, seed=21):
     ws = torch.empty(B.encoder_layer_workspace_bytes(T, hidden, ffn), dtype=torch.uint8, device="cuda")
     st = status_buf()
     scale = float(np.float32(1 / math.sqrt(D)))
-    B.encoder_layer_fwd(to_dev(x), y, weights, H, ffn, plan, scale, 1e-6, ws, lse, st)
+    tabs = W.rope2d_tables(counts, D) if rope else None
+    rope_dev = None if tabs is None else tuple(torch.from_numpy(t).cuda() for t in tabs)
+    B.encoder_layer_fwd(to_dev(x), y, weights, H, ffn, plan, scale, 1e-6, ws, lse, st, rope=rope_dev)
     torch.cuda.synchronize()
     assert st.cpu().tolist()[0] == 0
     ow = OL.LayerWeights(g1=OL.widen(pb["ln1_gamma"]), b1=OL.widen(pb["ln1_beta"]), wqkv=OL.widen(pb["w_qkv"]),
@@ -86,7 +105,8 @@ def _run_layer(counts, H, D, ffn, mode, seed=21):
                          g2=OL.widen(pb["ln2_gamma"]), b2=OL.widen(pb["ln2_beta"]), w1=OL.widen(pb["w_fc1"]),
                          bb1=OL.widen(pb["b_fc1"]), w2=OL.widen(pb["w_fc2"]), bb2=OL.widen(pb["b_fc2"]))
     cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
-    ref, parts = OL.encoder_layer_fwd(x, ow, cu, H, scale, 1e-6)
+    ref, parts = OL.encoder_layer_fwd(x, ow, cu, H, scale, 1e-6,
+                                      rope_tables=None if tabs is None else tuple(t.astype(np.float64) for t in tabs))
     return to_f64(y), ref, (None if lse is None else lse.cpu().double().numpy()), parts
 
 
@@ -97,6 +117,12 @@ def test_layer_matches_oracle(counts, H, D, ffn):
     assert rel_l2(y, ref) <= LAYER_REL_L2
     assert np.abs(y - ref).max() <= 0.05 + 2.0 ** -6 * np.abs(ref).max()
     assert np.abs(lse - parts["lse"]).max() <= 2e-2   # LSE of bf16-rounded q, k (the projections are stored as bf16)
+
+
+def test_layer_with_rope_matches_oracle():
+    y, ref, lse, parts = _run_layer([300, 1, 129, 640], 4, 80, 1280, B.TRAINED, rope=True)
+    assert rel_l2(y, ref) <= LAYER_REL_L2
+    assert np.abs(lse - parts["lse"]).max() <= 2e-2
 
 
 def test_layer_frozen_equals_trained_output():

@@ -105,3 +105,48 @@ def test_layer_special_cases():
     # bf16 bit patterns widen exactly
     bits = (np.float32(1.5).view(np.uint32) >> 16).astype(np.uint16)
     assert L.widen(np.array([[bits]], dtype=np.uint16))[0, 0] == 1.5
+
+
+def test_rope_is_a_rotation_and_matches_complex_form():
+    rng = np.random.default_rng(5)
+    T, H, D = 9, 2, 16
+    x = rng.standard_normal((T, H, D))
+    ang = rng.uniform(-3, 3, (T, D // 2))
+    y = L.rope(x, np.cos(ang), np.sin(ang))
+    # the same thing as a complex multiplication of (x1 + i x2) by exp(i angle)
+    z = (x[..., :D // 2] + 1j * x[..., D // 2:]) * np.exp(1j * ang)[:, None, :]
+    np.testing.assert_allclose(y, np.concatenate([z.real, z.imag], axis=-1), atol=1e-14)
+    np.testing.assert_allclose((y ** 2).sum(-1), (x ** 2).sum(-1), rtol=1e-13)          # norms are kept
+    np.testing.assert_allclose(L.rope(x, np.ones((T, D // 2)), np.zeros((T, D // 2))), x, atol=0)   # angle 0
+    back = L.rope(y, np.cos(-ang), np.sin(-ang))
+    np.testing.assert_allclose(back, x, atol=1e-13)
+
+
+def test_rope_scores_depend_on_relative_position_only():
+    rng = np.random.default_rng(6)
+    D = 8
+    q, k = rng.standard_normal((1, 1, D)), rng.standard_normal((1, 1, D))
+    inv = 10000.0 ** (-np.arange(D // 2) / (D // 2))
+
+    def score(m, n):
+        qa = L.rope(q, np.cos(m * inv)[None], np.sin(m * inv)[None])
+        ka = L.rope(k, np.cos(n * inv)[None], np.sin(n * inv)[None])
+        return float((qa * ka).sum())
+    assert abs(score(5, 2) - score(13, 10)) < 1e-12 and abs(score(5, 2) - score(5, 3)) > 1e-6
+
+
+def test_layer_with_rope_matches_manual_composition():
+    rng = np.random.default_rng(7)
+    H, D = 2, 8
+    hidden, ffn = H * D, 24
+    w = _rand_weights(rng, hidden, ffn)
+    x = rng.standard_normal((7, hidden))
+    cu = np.array([0, 3, 7], dtype=np.int32)
+    ang = rng.uniform(-2, 2, (7, D // 2))
+    tabs = (np.cos(ang), np.sin(ang))
+    _, parts = L.encoder_layer_fwd(x, w, cu, H, 0.25, 1e-6, rope_tables=tabs)
+    qkv = parts["qkv"]
+    q, k, v = (qkv[:, i * hidden:(i + 1) * hidden].reshape(7, H, D) for i in range(3))
+    o_ref, _ = oracle.attn_fwd(np.ascontiguousarray(L.rope(q, *tabs)), np.ascontiguousarray(L.rope(k, *tabs)),
+                               np.ascontiguousarray(v), cu, 0.25)
+    np.testing.assert_allclose(parts["o"], o_ref, atol=1e-14)
