@@ -275,6 +275,77 @@ int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weight
                                 size_t workspace_bytes, int32_t* status_buf, void* stream);
 
 /*
+ * derive : cut x schedule x model -> placement x collectives x order  (Section 4.1, "Schedule Algebra") -- host only.
+ *
+ * A model of n_layers layers is cut into k contiguous regions by k-1 interior boundaries cut[0] < ... < cut[k-2]
+ * in (0, n_layers); skeletons[j] in {1f1b, gpipe, transpose} is region j+1's skeleton and trainable[j] its
+ * trainable bit.  layout(transpose) = Replicated, layout(1f1b) = layout(gpipe) = Sharded.  Regions, microbatches
+ * and events' `mb` are 1-based as in the paper; ranks are 0-based.
+ *
+ *   mpipe_schedule_valid      MPIPE_OK iff the cut tiles the model and no two adjacent regions are Replicated
+ *                             (normal form), MPIPE_ERR_INVALID_ARG otherwise.
+ *   mpipe_schedule_normalize  collapses runs of adjacent transpose regions into one (their seam is the identity):
+ *                             <transpose, transpose> -> <transpose>.  out_skeletons[k], out_cut[k-1], *out_k.
+ *   mpipe_stage_index         rank + (region - 1) * n_ranks.
+ *   mpipe_derive              for a VALID schedule:
+ *     regions[k]      layout, first layer, layer count, skeleton of each region (placement);
+ *     slabs[k][P][2]  the owner's table: Sharded = ByLayer, contiguous slabs (first layer, count), the remainder of
+ *                     count / P going to the first ranks; Replicated = the whole region on every rank, with
+ *                     ByMicrobatch given by owner[mb-1] (NULL: (mb-1) mod P);
+ *     seams[k-1]      Table 2: forward comm of (j, j+1) from the layout pair, backward comm present (else
+ *                     MPIPE_COMM_NONE) iff some region <= j is trainable (Lemma 1 (ii) at j = (i) at j+1);
+ *     reduces         (region, group) of every trainable region: ReplicaGroup if Replicated, DataGroup if Sharded;
+ *     events / edges  the order graph.  Per microbatch: Fwd(j, r, m) on every rank of a Sharded region (r = 0..P-1 in
+ *                     turn) or on owner(m) for a Replicated one; Coll(fwd comm, seam j, m) between regions, placed
+ *                     on the receiving rank; Loss(m) on the last rank of the last region; Bwd(j, r, m) for every
+ *                     region with some trainable region <= j, in reverse; Coll(bwd comm, seam j-1, m) iff some region
+ *                     < j is trainable.  Then one DpReduce per entry of `reduces` and one StepBarrier (rank -1).
+ *                     Edges: Activation along the forward chain and from each Fwd to its own Bwd (the saved
+ *                     activation), Turnaround Loss -> first Bwd, Gradient along the backward chain, Accumulate
+ *                     Bwd -> DpReduce, Sequence DpReduce -> StepBarrier (Loss -> StepBarrier when nothing is
+ *                     trainable), Sequence for the skeleton's order inside a stage (1f1b: as many forwards as there are
+ *                     stages downstream -- P-1-r in the region, P per later Sharded and 1 per later Replicated
+ *                     region --, then forward/backward pairs, then backwards; gpipe: forwards then backwards in reverse; transpose:
+ *                     forwards then backwards by microbatch) and between neighbours of nodes(r);
+ *     node_order / node_offsets[P+1]   nodes(r): rank r's events in execution order, from unit-cost list scheduling
+ *                     in which a rank prefers (0) forwards of a Replicated region ahead of the first Sharded region
+ *                     (the warm-up bubble), (1) Sharded-region events, collectives and losses, (2) other
+ *                     Replicated-region events (cool-down); ties by event index.  The paper's figure for this is
+ *                     missing; this is the reading taken.
+ *     Capacities: events_cap / edges_cap entries; when too small the counts are still written and
+ *     MPIPE_ERR_WORKSPACE is returned.  MPIPE_ERR_INVALID_ARG for an invalid schedule or a Sharded region with
+ *     fewer layers than ranks; MPIPE_ERR_INDEX for an owner outside [0, P).
+ *   mpipe_order_makespan      Section 4.3: with cost[e] >= 0 per event, T = longest path of the graph (each rank's
+ *                             events follow nodes(r) through the Sequence edges), start[e] the earliest start times,
+ *                             bubble[r] = T - sum of the costs of rank r's events.  start and bubble may be NULL.
+ */
+enum { MPIPE_SK_1F1B = 0, MPIPE_SK_GPIPE = 1, MPIPE_SK_TRANSPOSE = 2 };
+enum { MPIPE_LAYOUT_SHARDED = 0, MPIPE_LAYOUT_REPLICATED = 1 };
+enum { MPIPE_COMM_NONE = 0, MPIPE_COMM_GATHER = 1, MPIPE_COMM_SCATTER = 2, MPIPE_COMM_SEND = 3, MPIPE_COMM_RECVGRAD = 4 };
+enum { MPIPE_GROUP_REPLICA = 0, MPIPE_GROUP_DATA = 1 };
+enum { MPIPE_EV_FWD = 0, MPIPE_EV_BWD = 1, MPIPE_EV_COLL = 2, MPIPE_EV_DPREDUCE = 3, MPIPE_EV_LOSS = 4, MPIPE_EV_STEPBARRIER = 5 };
+enum { MPIPE_EDGE_ACTIVATION = 0, MPIPE_EDGE_GRADIENT = 1, MPIPE_EDGE_TURNAROUND = 2, MPIPE_EDGE_ACCUMULATE = 3, MPIPE_EDGE_SEQUENCE = 4 };
+
+typedef struct { int32_t layout, first_layer, n_layers, skeleton; } mpipe_region_t;
+typedef struct { int32_t left_region, fwd_comm, bwd_comm; } mpipe_seam_t;          /* seam (left_region, left_region + 1) */
+typedef struct { int32_t region, group; } mpipe_reduce_t;
+/* kind; region (Coll: the seam's left region; StepBarrier: 0); rank (-1: all ranks); mb (0: none); comm (Coll only); group (DpReduce only, else -1) */
+typedef struct { int32_t kind, region, rank, mb, comm, group; } mpipe_event_t;
+typedef struct { int32_t src, dst, type; } mpipe_edge_t;
+
+int32_t mpipe_stage_index(int32_t rank, int32_t region, int32_t n_ranks);
+int32_t mpipe_schedule_valid(const int32_t* skeletons, const int32_t* cut, int32_t k, int32_t n_layers);
+int32_t mpipe_schedule_normalize(const int32_t* skeletons, const int32_t* cut, int32_t k, int32_t n_layers,
+                                 int32_t* out_skeletons, int32_t* out_cut, int32_t* out_k);
+int32_t mpipe_derive(const int32_t* skeletons, const int32_t* cut, int32_t k, int32_t n_layers, const int32_t* trainable,
+                     int32_t n_ranks, int32_t n_microbatches, const int32_t* owner, mpipe_region_t* regions,
+                     int32_t* slabs, mpipe_seam_t* seams, mpipe_reduce_t* reduces, int32_t* n_reduces,
+                     mpipe_event_t* events, int32_t events_cap, int32_t* n_events, mpipe_edge_t* edges,
+                     int32_t edges_cap, int32_t* n_edges, int32_t* node_order, int32_t* node_offsets);
+int32_t mpipe_order_makespan(const mpipe_event_t* events, int32_t n_events, const mpipe_edge_t* edges, int32_t n_edges,
+                             const double* cost, int32_t n_ranks, double* makespan, double* start, double* bubble);
+
+/*
  * Measurement aid (no counterpart in the paper; its cost model weights each compute event with one
  * duration, Section 4.3, and this is how a benchmark reads that duration for one kernel): while set,
  * the launch of kernel `which` (0 = attention forward, 1 = attention backward main kernel, 2 = merge

@@ -10,7 +10,7 @@ from __future__ import annotations
 import ctypes
 import os
 from dataclasses import dataclass
-from typing import Optional
+from typing import List, Optional
 
 import numpy as np
 import torch
@@ -32,6 +32,12 @@ ITEM_DTYPE = np.dtype([(n, np.int32) for n in ("seg", "tile", "row_start", "row_
 
 _i32, _i64, _vp, _f32, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float, ctypes.c_size_t
 _SIGNATURES = {
+    "mpipe_stage_index": (_i32, [_i32, _i32, _i32]),
+    "mpipe_schedule_valid": (_i32, [_vp, _vp, _i32, _i32]),
+    "mpipe_schedule_normalize": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp]),
+    "mpipe_derive": (_i32, [_vp, _vp, _i32, _i32, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _i32,
+                            _vp, _vp, _vp]),
+    "mpipe_order_makespan": (_i32, [_vp, _i32, _vp, _i32, _vp, _i32, _vp, _vp, _vp]),
     "mpipe_linear_fwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _i32, _vp, _vp]),
     "mpipe_layernorm_fwd": (_i32, [_vp, _vp, _vp, _vp, _i32, _i32, _i64, _i64, _f32, _vp]),
     "mpipe_encoder_layer_workspace_bytes": (_sz, [_i32, _i32, _i32]),
@@ -416,3 +422,90 @@ def set_profile_events(which: int, start: Optional[torch.cuda.Event], stop: Opti
 def validate_positions(positions, n_llm_tokens: int) -> int:
     pos = np.ascontiguousarray(np.asarray(positions, dtype=np.int32))
     return load().mpipe_validate_positions(_ptr(pos), pos.size, n_llm_tokens)
+
+
+# ------------------------------------------------------------------------------------------------
+# derive (Section 4.1) and the makespan read off its order graph (Section 4.3): host only
+# ------------------------------------------------------------------------------------------------
+SK_1F1B, SK_GPIPE, SK_TRANSPOSE = 0, 1, 2
+LAYOUT_SHARDED, LAYOUT_REPLICATED = 0, 1
+COMM_NONE, COMM_GATHER, COMM_SCATTER, COMM_SEND, COMM_RECVGRAD = range(5)
+GROUP_REPLICA, GROUP_DATA = 0, 1
+EV_FWD, EV_BWD, EV_COLL, EV_DPREDUCE, EV_LOSS, EV_STEPBARRIER = range(6)
+EDGE_ACTIVATION, EDGE_GRADIENT, EDGE_TURNAROUND, EDGE_ACCUMULATE, EDGE_SEQUENCE = range(5)
+
+
+def _i32arr(x):
+    return np.ascontiguousarray(np.asarray(x, dtype=np.int32).reshape(-1))
+
+
+def stage_index(rank: int, region: int, n_ranks: int) -> int:
+    return load().mpipe_stage_index(rank, region, n_ranks)
+
+
+def schedule_valid(skeletons, cut, n_layers: int) -> bool:
+    sk, c = _i32arr(skeletons), _i32arr(cut)
+    assert c.size == max(sk.size - 1, 0)
+    return load().mpipe_schedule_valid(sk.ctypes.data, c.ctypes.data if c.size else None, sk.size, n_layers) == OK
+
+
+def schedule_normalize(skeletons, cut, n_layers: int):
+    """-> (skeletons, cut) with runs of adjacent transpose regions collapsed into one."""
+    sk, c = _i32arr(skeletons), _i32arr(cut)
+    out_sk, out_c, out_k = np.zeros(sk.size, np.int32), np.zeros(max(sk.size - 1, 1), np.int32), ctypes.c_int32(0)
+    st = load().mpipe_schedule_normalize(sk.ctypes.data, c.ctypes.data if c.size else None, sk.size, n_layers,
+                                         out_sk.ctypes.data, out_c.ctypes.data, ctypes.addressof(out_k))
+    _check(st, "mpipe_schedule_normalize")
+    return out_sk[:out_k.value].tolist(), out_c[:out_k.value - 1].tolist()
+
+
+@dataclass
+class Derived:
+    """Output of mpipe_derive as numpy arrays (column meaning as in the header's structs)."""
+    regions: np.ndarray       # [k, 4]  layout, first_layer, n_layers, skeleton
+    slabs: np.ndarray         # [k, P, 2]
+    seams: np.ndarray         # [k-1, 3] left_region, fwd_comm, bwd_comm
+    reduces: np.ndarray       # [n, 2]  region, group
+    events: np.ndarray        # [n, 6]  kind, region, rank, mb, comm, group
+    edges: np.ndarray         # [n, 3]  src, dst, type
+    nodes: List[List[int]]    # per rank, event indices in execution order
+
+
+def derive(skeletons, cut, n_layers: int, trainable, n_ranks: int, n_microbatches: int, owner=None) -> Derived:
+    sk, c, tr = _i32arr(skeletons), _i32arr(cut), _i32arr(trainable)
+    k, P = sk.size, n_ranks
+    assert tr.size == k and c.size == max(k - 1, 0)
+    ow = None if owner is None else _i32arr(owner)
+    regions, slabs = np.zeros((k, 4), np.int32), np.zeros((k, max(P, 1), 2), np.int32)
+    seams, reduces = np.zeros((max(k - 1, 1), 3), np.int32), np.zeros((k, 2), np.int32)
+    n_red, n_ev, n_ed = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
+    offsets = np.zeros(max(P, 1) + 1, np.int32)
+    lib = load()
+
+    def call(events, edges, order, ecap, dcap):
+        return lib.mpipe_derive(sk.ctypes.data, c.ctypes.data if c.size else None, k, n_layers, tr.ctypes.data, P,
+                                n_microbatches, None if ow is None else ow.ctypes.data, regions.ctypes.data,
+                                slabs.ctypes.data, seams.ctypes.data, reduces.ctypes.data, ctypes.addressof(n_red),
+                                None if events is None else events.ctypes.data, ecap, ctypes.addressof(n_ev),
+                                None if edges is None else edges.ctypes.data, dcap, ctypes.addressof(n_ed),
+                                None if order is None else order.ctypes.data, offsets.ctypes.data)
+    st = call(None, None, None, 0, 0)          # first pass: sizes
+    if st != ERR_WORKSPACE:
+        _check(st, "mpipe_derive")
+    events, edges = np.zeros((max(n_ev.value, 1), 6), np.int32), np.zeros((max(n_ed.value, 1), 3), np.int32)
+    order = np.zeros(max(n_ev.value, 1), np.int32)
+    _check(call(events, edges, order, n_ev.value, n_ed.value), "mpipe_derive")
+    nodes = [order[offsets[r]:offsets[r + 1]].tolist() for r in range(P)]
+    return Derived(regions, slabs, seams[:k - 1], reduces[:n_red.value], events[:n_ev.value], edges[:n_ed.value], nodes)
+
+
+def order_makespan(events: np.ndarray, edges: np.ndarray, cost, n_ranks: int):
+    """-> (T, start[n_events], bubble[n_ranks])."""
+    ev, ed = np.ascontiguousarray(events, dtype=np.int32), np.ascontiguousarray(edges, dtype=np.int32)
+    cs = np.ascontiguousarray(cost, dtype=np.float64)
+    assert cs.size == ev.shape[0]
+    T, start, bub = ctypes.c_double(0.0), np.zeros(ev.shape[0], np.float64), np.zeros(n_ranks, np.float64)
+    st = load().mpipe_order_makespan(ev.ctypes.data, ev.shape[0], ed.ctypes.data if ed.size else None, ed.shape[0],
+                                     cs.ctypes.data, n_ranks, ctypes.addressof(T), start.ctypes.data, bub.ctypes.data)
+    _check(st, "mpipe_order_makespan")
+    return T.value, start, bub
