@@ -82,7 +82,10 @@ struct BwdCfg {
     // in-order issuer measured ~3 % faster (and keeps dK/dV bit-reproducible), so that is what D = 64 uses.
     static constexpr int kIssuers = (D == 64) ? 1 : 2;
     static constexpr int kKVBufs = (D == 64) ? 2 : 1;           // D = 64: the next unit's K/V tiles load during the current unit
-    static constexpr int kStatRing = 8;                         // LSE / Delta stages (written well ahead of their use)
+    // LSE / Delta stages.  One issuing warp: they travel with the Q / dO stages (same ring, same full / empty barriers:
+    // the issuer has no waits to spare).  Two issuing warps: a ring of 8 with barriers of its own, staged far ahead.
+    static constexpr bool kStatFolded = (kIssuers == 1);
+    static constexpr int kStatRing = kStatFolded ? kRing : 8;
     // dQ staging for the TMA reduction: one [128 q][32 fp32] box (used twice per pair) + the 16-column tail box
     static constexpr int kStageMain = kBT * 128;
     static constexpr int kStageBytes = kStageMain + (kTail ? kBT * 64 : 0);
@@ -154,7 +157,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         mbar_init(&bars.dkv_full, kIssuers);
         mbar_init(&bars.dkv_empty, 4);
         for (int s = 0; s < 4; ++s) {
-            mbar_init(&bars.qdo_full[s], 1);
+            mbar_init(&bars.qdo_full[s], Cfg::kStatFolded ? 2 : 1);   // the producer's expect_tx arrival (+ the staging warp)
             mbar_init(&bars.qdo_empty[s], 1);
         }
         for (int s = 0; s < 8; ++s) {
@@ -250,9 +253,12 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             constexpr uint32_t hi128 = umma_desc_hi(1024, kSwizzle128);
             constexpr uint32_t hi32 = umma_desc_hi(256, kSwizzle32);
             const uint32_t ds_lo = umma_desc_lo(sbase + Cfg::kSmemDS, kBT * 128);   // two 64-query atoms 16 KB apart
-            // LSE / Delta of a sub-tile must be staged before its S^T is issued: the softmax warps then need no
-            // barrier of their own for them (S^T complete implies staged)
-            auto wait_stat = [&](uint32_t c) { return MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.stat_full[c % NS], (c / NS) & 1, &abort_flag)); };
+            // LSE / Delta of a sub-tile must be staged before its S^T is issued: the softmax warps then need no barrier
+            // of their own for them (S^T complete implies staged).  Folded: qdo_full completes only when the staging
+            // warp has arrived too, so there is nothing more to wait for here.
+            auto wait_stat = [&](uint32_t c) {
+                return Cfg::kStatFolded ? true : MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.stat_full[c % NS], (c / NS) & 1, &abort_flag));
+            };
             constexpr uint32_t idesc_s = umma_idesc_bf16(kBT, kQS, 0, 0);      // K-major x K-major, N = 64 queries
             constexpr uint32_t idesc_ts = umma_idesc_bf16(kBT, 64, 0, 1);      // A in TMEM, MN-major B, N = 64
             constexpr uint32_t idesc_ts_t = umma_idesc_bf16(kBT, 16, 0, 1);    // same, 16-wide head-dim tail
@@ -369,8 +375,8 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                         if (leader) mbar_arrive(&bars.acc_k);
                     }
                     if (leader) {
-                        umma_commit(&bars.qdo_empty[c % NR]);
-                        mbar_arrive(&bars.stat_empty[c % NS]);   // dS^T(c) has arrived: its LSE / Delta stage has been read
+                        umma_commit(&bars.qdo_empty[c % NR]);   // folded: also frees the LSE / Delta stage (dS^T(c) has arrived)
+                        if (!Cfg::kStatFolded) mbar_arrive(&bars.stat_empty[c % NS]);
                     }
                     if (more) {
                         issue_kk(Cfg::kColDP + 64 * b, cross ? v_lo_n : v_lo, vt_lo, do_lo_of(c + 2));    // dP^T(s+2)
@@ -418,26 +424,29 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             const int q_end = it.kv_start + it.kv_len;
             for (int s = 0; s < n2; ++s, ++sc) {
                 const int rs = sc % NS;
-                ok = MW(mbar_wait<MPIPE_SLEEP_AUX>(&bars.stat_empty[rs], ((sc / NS) & 1) ^ 1, &abort_flag));
-                if (!ok) break;
                 float* dst = reinterpret_cast<float*>(smem + Cfg::kSmemStat + rs * (2 * kQS * 4));
                 const int q0 = it.kv_start + s * kQS;
+                float val[4];   // read from global memory before the stage is known to be free: the latency overlaps the wait
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {   // e = 0, 1: -LSE*log2e of 64 query columns; e = 2, 3: -Delta
                     const bool is_lse = (e < 2);
-                    const int c = lane + 32 * (e & 1);
-                    const int q = q0 + c;
-                    float val;   // stored negated: what the softmax warps add
-                    if (q < q_end) {
-                        val = -__ldg((is_lse ? p.lse : p.delta) + int64_t(head) * p.total_tokens + q);
-                        if (is_lse) val *= 1.4426950408889634f;
+                    const int q = q0 + lane + 32 * (e & 1);
+                    if (q < q_end) {   // stored negated: what the softmax warps add
+                        val[e] = -__ldg((is_lse ? p.lse : p.delta) + int64_t(head) * p.total_tokens + q);
+                        if (is_lse) val[e] *= 1.4426950408889634f;
                     } else {
-                        val = is_lse ? -CUDART_INF_F : 0.f;  // P = exp2(-inf) = 0 for query columns past the segment
+                        val[e] = is_lse ? -CUDART_INF_F : 0.f;  // P = exp2(-inf) = 0 for query columns past the segment
                     }
-                    dst[(is_lse ? 0 : kQS) + c] = val;
                 }
+                // the stage is free when the MMAs that read the Q / dO sub-tile of four sub-tiles ago have completed
+                // (that commit follows the arrival of its dS^T, i.e. the softmax warps' last read of the stage)
+                ok = MW(mbar_wait<MPIPE_SLEEP_AUX>(Cfg::kStatFolded ? &bars.qdo_empty[rs] : &bars.stat_empty[rs],
+                                                   ((sc / NS) & 1) ^ 1, &abort_flag));
+                if (!ok) break;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) dst[((e < 2) ? 0 : kQS) + lane + 32 * (e & 1)] = val[e];
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bars.stat_full[rs]);
+                if (lane == 0) mbar_arrive(Cfg::kStatFolded ? &bars.qdo_full[rs] : &bars.stat_full[rs]);
             }
         }
     } else if (warp == 3) {
