@@ -144,3 +144,59 @@ def test_layer_argument_checks():
     assert e.value.status == B.ERR_WORKSPACE
     with pytest.raises(B.MpipeError):
         B.linear_fwd(x, to_dev(W.normal_bf16(5, 1, (12, hidden))), torch.empty((T, 12), dtype=torch.bfloat16, device="cuda"))
+
+
+def test_linear_full_size_sampled_rows():
+    """The bench's largest projection shapes (ViT-L layer: fc1 and fc2 on the 50 439-token microbatch), checked on sampled
+    output rows that the oracle computes one by one."""
+    w = W.vit_l()
+    T, hidden, ffn = w.total_tokens, 1024, 4096
+    g = torch.Generator(device="cuda")
+    g.manual_seed(3)
+    a = torch.randn((T, hidden), device="cuda", generator=g).to(torch.bfloat16)
+    w1 = (torch.randn((ffn, hidden), device="cuda", generator=g) * hidden ** -0.5).to(torch.bfloat16)
+    b1 = (torch.randn((ffn,), device="cuda", generator=g) * 0.5).to(torch.bfloat16)
+    w2 = (torch.randn((hidden, ffn), device="cuda", generator=g) * ffn ** -0.5).to(torch.bfloat16)
+    res = torch.randn((T, hidden), device="cuda", generator=g).to(torch.bfloat16)
+    h = torch.empty((T, ffn), dtype=torch.bfloat16, device="cuda")
+    y = torch.empty((T, hidden), dtype=torch.bfloat16, device="cuda")
+    st = status_buf()
+    B.linear_fwd(a, w1, h, b1, None, True, st)
+    B.linear_fwd(h, w2, y, None, res, False, st)
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[0] == 0
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, T - 1, T - 2, (T // 128) * 128],
+                                     np.random.default_rng(0).integers(0, T, 40)]))
+    idx = torch.from_numpy(rows).cuda()
+    h_ref = OL.gelu(OL.linear(to_f64(a[idx]), to_f64(w1), to_f64(b1)))
+    _check_close(to_f64(h[idx]), h_ref, atol=2e-3)
+    y_ref = OL.linear(to_f64(h[idx]), to_f64(w2)) + to_f64(res[idx])      # from the GPU's own bf16 h: one stage at a time
+    _check_close(to_f64(y[idx]), y_ref, atol=2e-3)
+
+
+def test_layer_full_size_sampled_segments():
+    """The bench's ViT-L layer microbatch through mpipe_encoder_layer_fwd; attention is block-diagonal, so the rows of
+    any image depend on that image alone: the oracle recomputes the three shortest images and compares those rows."""
+    w = W.vit_l()
+    H, D = w.n_heads, w.head_dim
+    hidden, ffn, T = H * D, 4 * H * D, w.total_tokens
+    pb = W.layer_params_bf16(31, hidden, ffn)
+    x = W.normal_bf16(31, 0, (T, hidden))
+    plan = B.seg_plan(w.patch_counts, B.FROZEN).to_device()
+    weights = B.LayerWeights.from_tensors(**{k: to_dev(v) for k, v in pb.items()})
+    y = torch.empty((T, hidden), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(B.encoder_layer_workspace_bytes(T, hidden, ffn), dtype=torch.uint8, device="cuda")
+    st = status_buf()
+    B.encoder_layer_fwd(to_dev(x), y, weights, H, ffn, plan, w.softmax_scale, 1e-6, ws, None, st)
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[0] == 0
+    ow = OL.LayerWeights(g1=OL.widen(pb["ln1_gamma"]), b1=OL.widen(pb["ln1_beta"]), wqkv=OL.widen(pb["w_qkv"]),
+                         bqkv=OL.widen(pb["b_qkv"]), wo=OL.widen(pb["w_o"]), bo=OL.widen(pb["b_o"]),
+                         g2=OL.widen(pb["ln2_gamma"]), b2=OL.widen(pb["ln2_beta"]), w1=OL.widen(pb["w_fc1"]),
+                         bb1=OL.widen(pb["b_fc1"]), w2=OL.widen(pb["w_fc2"]), bb2=OL.widen(pb["b_fc2"]))
+    got = to_f64(y)
+    cu = w.cu_seqlens
+    for seg in np.argsort(w.patch_counts)[:3]:
+        lo, hi = int(cu[seg]), int(cu[seg + 1])
+        ref, _ = OL.encoder_layer_fwd(x[lo:hi], ow, np.array([0, hi - lo], dtype=np.int32), H, w.softmax_scale, 1e-6)
+        assert rel_l2(got[lo:hi], ref) <= LAYER_REL_L2, (seg, rel_l2(got[lo:hi], ref))
