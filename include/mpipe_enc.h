@@ -275,6 +275,22 @@ int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weight
                                 size_t workspace_bytes, int32_t* status_buf, void* stream);
 
 /*
+ * The Replicated -> Sharded seam across ranks (Table 2: Gather forward, Scatter backward).  The encoder output of
+ * microbatch m is produced on ByMicrobatch(m); the LLM input sequence lives on the first pipeline stage.  The seam is
+ * run as ONE kernel: mpipe_merge_tokens on the owner with `llm_embeds` pointing into the first stage's buffer through
+ * a peer mapping (plain stores over NVLink), and mpipe_merge_tokens_bwd reading the gradient rows the same way.
+ * These three host calls provide the mapping (CUDA IPC; the exporting allocation must come from cudaMalloc and stay
+ * alive while mapped).  handle buffers are mpipe_ipc_handle_bytes() bytes of host memory.  An opened pointer is valid
+ * in the opening process only and must be closed there.  Ordering between ranks (the first stage may read the rows
+ * only after the owner's kernel has completed) is the caller's: a stream synchronisation on the owner followed by any
+ * host-level message.  MPIPE_ERR_CUDA when the runtime refuses (e.g. same process as the exporter).
+ */
+int32_t mpipe_ipc_handle_bytes(void);
+int32_t mpipe_ipc_export(const void* dev_ptr, void* handle_out);
+int32_t mpipe_ipc_open(const void* handle, void** dev_ptr_out);
+int32_t mpipe_ipc_close(void* dev_ptr);
+
+/*
  * derive : cut x schedule x model -> placement x collectives x order  (Section 4.1, "Schedule Algebra") -- host only.
  *
  * A model of n_layers layers is cut into k contiguous regions by k-1 interior boundaries cut[0] < ... < cut[k-2]

@@ -32,6 +32,10 @@ ITEM_DTYPE = np.dtype([(n, np.int32) for n in ("seg", "tile", "row_start", "row_
 
 _i32, _i64, _vp, _f32, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float, ctypes.c_size_t
 _SIGNATURES = {
+    "mpipe_ipc_handle_bytes": (_i32, []),
+    "mpipe_ipc_export": (_i32, [_vp, _vp]),
+    "mpipe_ipc_open": (_i32, [_vp, _vp]),
+    "mpipe_ipc_close": (_i32, [_vp]),
     "mpipe_stage_index": (_i32, [_i32, _i32, _i32]),
     "mpipe_schedule_valid": (_i32, [_vp, _vp, _i32, _i32]),
     "mpipe_schedule_normalize": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp]),
@@ -356,6 +360,49 @@ def merge_tokens_bwd(d_llm_embeds, d_enc, positions_dev, mode: int, status_buf=N
     st = load().mpipe_merge_tokens_bwd(_ptr(d_llm_embeds), d_llm_embeds.stride(0), _ptr(d_enc),
                                        d_enc.stride(0) if n_enc else hidden, _ptr(positions_dev), n_enc, n_llm,
                                        hidden, mode, _ptr(status_buf), _stream(stream))
+    _check(st, "mpipe_merge_tokens_bwd")
+
+
+class PeerRows:
+    """A [n_rows, hidden] bf16 matrix in ANOTHER process's device memory (opened from an IPC handle), usable as the
+    `llm_embeds` of merge_tokens / the `d_llm_embeds` of merge_tokens_bwd: the cross-rank seam as one kernel."""
+
+    def __init__(self, handle: bytes, n_rows: int, hidden: int, row_stride: int):
+        self.n_rows, self.hidden, self.row_stride = n_rows, hidden, row_stride
+        ptr = ctypes.c_void_p()
+        buf = ctypes.create_string_buffer(handle, len(handle))
+        _check(load().mpipe_ipc_open(ctypes.addressof(buf), ctypes.addressof(ptr)), "mpipe_ipc_open")
+        self.ptr = ptr.value
+
+    def close(self) -> None:
+        if self.ptr:
+            _check(load().mpipe_ipc_close(self.ptr), "mpipe_ipc_close")
+            self.ptr = None
+
+
+def ipc_export(t) -> bytes:
+    """IPC handle of the allocation behind CUDA tensor t (which must start at the allocation's base: allocate it with
+    `torch.empty` of at least 1 MiB or through a dedicated allocation so that it is not packed into a shared block)."""
+    n = load().mpipe_ipc_handle_bytes()
+    buf = ctypes.create_string_buffer(n)
+    _check(load().mpipe_ipc_export(_ptr(t), ctypes.addressof(buf)), "mpipe_ipc_export")
+    return buf.raw
+
+
+def merge_tokens_peer(enc_tokens, peer: PeerRows, positions_dev, mode: int = TRAINED, status_buf=None, stream=None) -> None:
+    """mpipe_merge_tokens with the destination in a peer's memory: the Gather seam (Table 2) as one kernel."""
+    n_enc = int(positions_dev.numel())
+    assert enc_tokens.dtype == torch.bfloat16 and enc_tokens.shape[1] == peer.hidden and enc_tokens.stride(1) == 1
+    st = load().mpipe_merge_tokens(_ptr(enc_tokens), enc_tokens.stride(0), peer.ptr, peer.row_stride, _ptr(positions_dev),
+                                   n_enc, peer.n_rows, peer.hidden, mode, _ptr(status_buf), _stream(stream))
+    _check(st, "mpipe_merge_tokens")
+
+
+def merge_tokens_bwd_peer(peer: PeerRows, d_enc, positions_dev, mode: int, status_buf=None, stream=None) -> None:
+    """mpipe_merge_tokens_bwd reading the gradient rows from a peer's memory: the reverse (Scatter) seam."""
+    n_enc = int(positions_dev.numel())
+    st = load().mpipe_merge_tokens_bwd(peer.ptr, peer.row_stride, _ptr(d_enc), d_enc.stride(0), _ptr(positions_dev), n_enc,
+                                       peer.n_rows, peer.hidden, mode, _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_merge_tokens_bwd")
 
 

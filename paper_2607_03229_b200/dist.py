@@ -45,6 +45,35 @@ def reduce_max_sum(max_vals: Sequence[float], sum_vals: Sequence[float], device=
     return mx.tolist(), sm.tolist()
 
 
+def seam_targets(owner: Sequence[int], first_stage_rank: int = 0):
+    """For the Replicated -> Sharded seam (Table 2): which microbatches rank r must ship, per rank.  `owner[m]` is the
+    ByMicrobatch owner of microbatch m (0-based); every microbatch goes to `first_stage_rank`, and a microbatch that
+    is already there needs no transfer (its merge is local)."""
+    world = (max(owner) + 1) if len(owner) else 1
+    world = max(world, first_stage_rank + 1)
+    ship = {r: [] for r in range(world)}
+    local = []
+    for m, r in enumerate(owner):
+        (local if r == first_stage_rank else ship[r]).append(m)
+    return ship, local
+
+
+def share_rows(t: "torch.Tensor", src_rank: int):
+    """Export `t` ([rows, hidden] bf16 CUDA tensor owned by `src_rank`, alone in its allocation) to every other rank of
+    the default process group.  Returns the tensor itself on `src_rank` and a binding.PeerRows elsewhere."""
+    from . import binding as B
+    rank = dist.get_rank() if dist.is_initialized() else 0
+    payload = [None]
+    if rank == src_rank:
+        payload = [(B.ipc_export(t), int(t.shape[0]), int(t.shape[1]), int(t.stride(0)))]
+    if dist.is_initialized():
+        dist.broadcast_object_list(payload, src=src_rank)
+    if rank == src_rank:
+        return t
+    handle, rows, hidden, stride = payload[0]
+    return B.PeerRows(handle, rows, hidden, stride)
+
+
 def shutdown() -> None:
     if dist.is_initialized():
         dist.destroy_process_group()

@@ -50,3 +50,16 @@ def test_single_process_defaults():
     assert D.env_world() == (0, 0, 1)
     assert D.reduce_max_sum([3.0], [4.0]) == ([3.0], [4.0])
     assert D.rank_seed(7, 0) == 7 and D.rank_seed(7, 3) == 3007
+
+
+def test_seam_targets_route_every_microbatch_to_the_first_stage():
+    from paper_2607_03229_b200 import dist as D
+    ship, local = D.seam_targets([3, 0, 1, 3, 0, 2], first_stage_rank=0)
+    assert local == [1, 4] and ship == {0: [], 1: [2], 2: [5], 3: [0, 3]}
+    ship, local = D.seam_targets([], first_stage_rank=0)
+    assert local == [] and ship == {0: []}
+    # every microbatch is either local to the first stage or shipped by exactly its owner
+    owner = [1, 1, 0, 2]
+    ship, local = D.seam_targets(owner, first_stage_rank=1)
+    assert sorted(local + [m for v in ship.values() for m in v]) == list(range(len(owner)))
+    assert all(owner[m] == r for r, v in ship.items() for m in v) and all(owner[m] == 1 for m in local)
