@@ -191,7 +191,7 @@ def _every_element(w):
 
 _FULL = pytest.mark.skipif(__import__("os").environ.get("MPIPE_FULL_PARITY") != "1",
                            reason="full-tensor oracle pass of the two largest configs takes minutes of CPU; "
-                                  "set MPIPE_FULL_PARITY=1 (done once per release, results in DESIGN.md)")
+                                  "set MPIPE_FULL_PARITY=1 (done once per release)")
 
 
 @_FULL
