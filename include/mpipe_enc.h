@@ -262,6 +262,13 @@ typedef struct {
 int32_t mpipe_linear_fwd(const void* a, const void* w, const void* bias, const void* residual, void* c, int32_t M,
                          int32_t N, int32_t K, int64_t lda, int64_t ldw, int64_t ldr, int64_t ldc, int32_t flags,
                          int32_t* status_buf, void* stream);
+/* Input gradient of a projection y = x W^T (W [N, K]):  dx[M, K] = (dy[M, N] W[N, K]) o GELU'(gelu_input[M, K]) + residual[M, K].
+ * gelu_input (the pre-activation u of the layer in front, whose output x = GELU(u) fed this projection) and residual
+ * may be NULL; GELU'(u) = Phi(u) + u phi(u).  Same layout, alignment and error rules as mpipe_linear_fwd; W is read
+ * as stored (no transposed copy). */
+int32_t mpipe_linear_dgrad(const void* dy, const void* w, const void* gelu_input, const void* residual, void* dx, int32_t M,
+                           int32_t N, int32_t K, int64_t lddy, int64_t ldw, int64_t ldu, int64_t ldr, int64_t lddx,
+                           int32_t* status_buf, void* stream);
 int32_t mpipe_layernorm_fwd(const void* x, const void* gamma, const void* beta, void* y, int32_t n_tokens,
                             int32_t hidden, int64_t ldx, int64_t ldy, float eps, void* stream);
 int32_t mpipe_rope_apply(void* qk, int64_t tok_stride, int64_t k_offset, const float* cos_table, const float* sin_table,

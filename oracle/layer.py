@@ -60,6 +60,23 @@ def gelu(u: np.ndarray) -> np.ndarray:
     return 0.5 * u * (1.0 + _erf(u / math.sqrt(2.0)))
 
 
+def gelu_grad(u: np.ndarray) -> np.ndarray:
+    """d/du [u Phi(u)] = Phi(u) + u phi(u) with phi the standard normal density."""
+    u = np.asarray(u, dtype=np.float64)
+    return 0.5 * (1.0 + _erf(u / math.sqrt(2.0))) + u * np.exp(-0.5 * u * u) / math.sqrt(2.0 * math.pi)
+
+
+def linear_dgrad(dy: np.ndarray, w: np.ndarray) -> np.ndarray:
+    """Input gradient of y = x w^T: dx = dy w."""
+    return np.asarray(dy, dtype=np.float64) @ np.asarray(w, dtype=np.float64)
+
+
+def linear_wgrad(dy: np.ndarray, x: np.ndarray):
+    """Parameter gradients of y = x w^T + b: dw = dy^T x, db = column sums of dy."""
+    dy = np.asarray(dy, dtype=np.float64)
+    return dy.T @ np.asarray(x, dtype=np.float64), dy.sum(axis=0)
+
+
 def rope(x: np.ndarray, cos: np.ndarray, sin: np.ndarray) -> np.ndarray:
     """Rotate-half rotary encoding.  x: [T, H, D]; cos, sin: [T, D/2] (angle of pair j of token t).  The pair is
     (x[..., j], x[..., j + D/2]) and it is rotated by that angle: a plain 2-D rotation per pair."""

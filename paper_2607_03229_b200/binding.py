@@ -32,6 +32,7 @@ ITEM_DTYPE = np.dtype([(n, np.int32) for n in ("seg", "tile", "row_start", "row_
 
 _i32, _i64, _vp, _f32, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float, ctypes.c_size_t
 _SIGNATURES = {
+    "mpipe_linear_dgrad": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _i64, _vp, _vp]),
     "mpipe_ipc_handle_bytes": (_i32, []),
     "mpipe_ipc_export": (_i32, [_vp, _vp]),
     "mpipe_ipc_open": (_i32, [_vp, _vp]),
@@ -260,6 +261,17 @@ def linear_fwd(a, w, c, bias=None, residual=None, gelu: bool = False, status_buf
                                  0 if residual is None else _rows(residual), _rows(c), LINEAR_GELU if gelu else 0,
                                  _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_linear_fwd")
+
+
+def linear_dgrad(dy, w, dx, gelu_input=None, residual=None, status_buf=None, stream=None) -> None:
+    """mpipe_linear_dgrad: dx[M,K] = (dy[M,N] w[N,K]) o GELU'(gelu_input) + residual (bf16 CUDA tensors)."""
+    M, N = dy.shape
+    K = w.shape[1]
+    assert w.shape[0] == N and tuple(dx.shape) == (M, K)
+    st = load().mpipe_linear_dgrad(_ptr(dy), _ptr(w), _ptr(gelu_input), _ptr(residual), _ptr(dx), M, N, K, _rows(dy), _rows(w),
+                                   0 if gelu_input is None else _rows(gelu_input), 0 if residual is None else _rows(residual),
+                                   _rows(dx), _ptr(status_buf), _stream(stream))
+    _check(st, "mpipe_linear_dgrad")
 
 
 def layernorm_fwd(x, gamma, beta, y, eps: float, stream=None) -> None:

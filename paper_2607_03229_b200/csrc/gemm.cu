@@ -1,5 +1,7 @@
 // mpipe_linear_fwd: C[M, N] = epilogue(A[M, K] * W[N, K]^T), the dense projections of the packed encoder layer
 // (QKV, attention output, MLP) on the token matrix [T, hidden].  bf16 operands, fp32 accumulation in TMEM.
+// mpipe_linear_dgrad: dX[M, K] = epilogue(dY[M, N] * W[N, K]) -- the same kernel with the second operand read as
+// [contraction][output] (an MN-major B: four 64-column atoms per stage, loaded as four TMA boxes).
 //
 // Persistent kernel, one CTA per SM, static round-robin over 128 x 256 output tiles (n fastest, so that the
 // CTAs of a wave share the few weight tiles in L2 and walk down the token rows together).
@@ -37,6 +39,8 @@ struct GemmParams {
     int32_t tiles_m, tiles_n;
     const __nv_bfloat16* bias;       // [N] or null
     const __nv_bfloat16* residual;   // [M, ldr] or null
+    const __nv_bfloat16* aux;        // [M, ldx] or null: pre-activation u; the result is multiplied by GELU'(u)
+    int64_t ldx;
     __nv_bfloat16* C;                // [M, ldc]
     int64_t ldr, ldc;
     int32_t gelu;
@@ -62,9 +66,18 @@ __device__ __forceinline__ float erf_as(float x) {
     return copysignf(1.0f - p * e, x);
 }
 __device__ __forceinline__ float gelu_erf(float u) { return 0.5f * u * (1.0f + erf_as(u * 0.7071067811865476f)); }
+// d/du [u Phi(u)] = Phi(u) + u phi(u), phi the standard normal density
+__device__ __forceinline__ float gelu_erf_grad(float u) {
+    const float cdf = 0.5f * (1.0f + erf_as(u * 0.7071067811865476f));
+    const float pdf = 0.3989422804014327f * ex2_approx(-0.5f * u * u * 1.4426950408889634f);
+    return fmaf(u, pdf, cdf);
+}
 
+// kBMode 0: W tile [256 output rows][64 k], K-major (forward).  kBMode 1: W tile [64 contraction rows][256 output
+// columns], MN-major: four [64][64] atoms 8 KB apart (input gradient).
+template <int kBMode>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-linear_fwd_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
+linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
                   const __grid_constant__ CUtensorMap map_c, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -111,7 +124,13 @@ linear_fwd_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     uint8_t* st = smem + s * kGemmStageBytes;
                     mbar_expect_tx(&bars.full[s], kGemmStageBytes);   // out-of-range rows / columns are zero-filled, still counted
                     tma_load_3d(st, &map_a, &bars.full[s], kb * kGemmBK, 0, m0);
-                    tma_load_3d(st + kGemmABytes, &map_w, &bars.full[s], kb * kGemmBK, 0, n0);
+                    if (kBMode == 0) {
+                        tma_load_3d(st + kGemmABytes, &map_w, &bars.full[s], kb * kGemmBK, 0, n0);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < kGemmBN / 64; ++i)
+                            tma_load_3d(st + kGemmABytes + i * (kGemmBK * 128), &map_w, &bars.full[s], n0 + 64 * i, 0, kb * kGemmBK);
+                    }
                 }
             }
         }
@@ -120,7 +139,7 @@ linear_fwd_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const bool leader = elect_one();
         const uint32_t sbase = smem_u32(smem);
         constexpr uint32_t hi128 = umma_desc_hi(1024, kSwizzle128);
-        constexpr uint32_t idesc = umma_idesc_bf16(kGemmBM, kGemmBN, 0, 0);
+        constexpr uint32_t idesc = umma_idesc_bf16(kGemmBM, kGemmBN, 0, kBMode);
         uint32_t it = 0, tile_it = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_it) {
@@ -134,11 +153,12 @@ linear_fwd_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t a_lo = umma_desc_lo(sbase + s * kGemmStageBytes, 0);
-                const uint32_t b_lo = umma_desc_lo(sbase + s * kGemmStageBytes + kGemmABytes, 0);
+                const uint32_t b_lo = umma_desc_lo(sbase + s * kGemmStageBytes + kGemmABytes, kBMode == 0 ? 0 : kGemmBK * 128);
+                constexpr uint32_t b_step = kBMode == 0 ? 2 : 128;   // one K-step: 32 bytes along a row, or 16 rows of 128 bytes
                 if (leader) {
 #pragma unroll
                     for (int ks = 0; ks < kGemmBK / 16; ++ks)
-                        umma_ss(tmem + acc * kGemmBN, umma_desc(a_lo + ks * 2, hi128), umma_desc(b_lo + ks * 2, hi128), idesc,
+                        umma_ss(tmem + acc * kGemmBN, umma_desc(a_lo + ks * 2, hi128), umma_desc(b_lo + ks * b_step, hi128), idesc,
                                 (kb > 0 || ks > 0) ? 1u : 0u);
                     umma_commit(&bars.empty[s]);
                 }
@@ -172,7 +192,17 @@ linear_fwd_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     res[g8] = (rrow != nullptr && n < p.N) ? __ldg(reinterpret_cast<const uint4*>(rrow + n)) : make_uint4(0u, 0u, 0u, 0u);
                 }
             };
+            const __nv_bfloat16* xrow = (p.aux != nullptr && row_ok) ? p.aux + int64_t(m) * p.ldx : nullptr;
+            uint4 aux[4];
+            auto load_aux = [&](int c0) {
+#pragma unroll
+                for (int g8 = 0; g8 < 4; ++g8) {
+                    const int n = n_base + c0 + 8 * g8;
+                    aux[g8] = (xrow != nullptr && n < p.N) ? __ldg(reinterpret_cast<const uint4*>(xrow + n)) : make_uint4(0u, 0u, 0u, 0u);
+                }
+            };
             if (p.residual != nullptr) load_res(0);
+            if (p.aux != nullptr) load_aux(0);
             if (ok) ok = mbar_wait(&bars.acc_full[acc], (tile_it >> 1) & 1, &abort_flag);
             tc_fence_after();
 #pragma unroll 1
@@ -180,10 +210,16 @@ linear_fwd_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 uint32_t v[32];
                 uint32_t out[16];
                 uint4 rcur[4];
+                uint4 xcur[4];
                 if (p.residual != nullptr) {
 #pragma unroll
                     for (int g8 = 0; g8 < 4; ++g8) rcur[g8] = res[g8];
                     if (c0 + 32 < kGemmBN / 2) load_res(c0 + 32);
+                }
+                if (p.aux != nullptr) {
+#pragma unroll
+                    for (int g8 = 0; g8 < 4; ++g8) xcur[g8] = aux[g8];
+                    if (c0 + 32 < kGemmBN / 2) load_aux(c0 + 32);
                 }
                 if (ok) {
                     tmem_ld32(tmem + lane_base + acc * kGemmBN + wg * (kGemmBN / 2) + c0, v);
@@ -212,6 +248,14 @@ linear_fwd_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                         if (p.gelu) {
 #pragma unroll
                             for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
+                        }
+                        if (p.aux != nullptr) {
+                            const uint32_t xw[4] = {xcur[g8].x, xcur[g8].y, xcur[g8].z, xcur[g8].w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                f[2 * i] *= gelu_erf_grad(__uint_as_float(xw[i] << 16));
+                                f[2 * i + 1] *= gelu_erf_grad(__uint_as_float(xw[i] & 0xffff0000u));
+                            }
                         }
                         if (p.residual != nullptr) {
                             const uint32_t rw[4] = {rcur[g8].x, rcur[g8].y, rcur[g8].z, rcur[g8].w};
@@ -253,48 +297,74 @@ linear_fwd_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
 }  // namespace mpipe
 
+namespace mpipe {
+
+// Shared host side of the two entry points.  n_out / n_contract are the output columns and the contraction length.
+static int32_t launch_linear(int b_mode, const void* a, const void* w, const void* bias, const void* residual, const void* aux,
+                             void* c, int32_t M, int32_t n_out, int32_t n_contract, int64_t lda, int64_t ldw, int64_t ldr,
+                             int64_t ldx, int64_t ldc, int32_t gelu, int32_t* status_buf, void* stream) {
+    if (M < 0 || n_out <= 0 || n_contract <= 0) return MPIPE_ERR_INVALID_ARG;
+    if (M == 0) return MPIPE_OK;
+    if (a == nullptr || w == nullptr || c == nullptr) return MPIPE_ERR_INVALID_ARG;
+    if ((n_out % 8) != 0 || (n_contract % 8) != 0) return MPIPE_ERR_UNSUPPORTED;
+    const int64_t w_cols = b_mode == 0 ? n_contract : n_out;
+    if (lda < n_contract || ldw < w_cols || ldc < n_out || (residual != nullptr && ldr < n_out) || (aux != nullptr && ldx < n_out))
+        return MPIPE_ERR_INVALID_ARG;
+    if ((lda % 8) != 0 || (ldw % 8) != 0 || (ldc % 8) != 0 || (residual != nullptr && (ldr % 8) != 0) || (aux != nullptr && (ldx % 8) != 0))
+        return MPIPE_ERR_UNSUPPORTED;
+    if (!aligned16(a) || !aligned16(w) || !aligned16(c) || !aligned16(bias) || !aligned16(residual) || !aligned16(aux))
+        return MPIPE_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CUtensorMap map_a, map_w, map_c;
+    bool ok = make_tensor_map_thd(&map_a, a, M, 1, n_contract, lda, lda, kGemmBK, kGemmBM, 128) &&
+              make_tensor_map_thd(&map_c, c, M, 1, n_out, ldc, ldc, 32, kGemmBM, 64);
+    if (b_mode == 0)   // W[n_out rows, n_contract columns]: boxes of 256 rows x 64 k
+        ok = ok && make_tensor_map_thd(&map_w, w, n_out, 1, n_contract, ldw, ldw, kGemmBK, kGemmBN, 128);
+    else               // W[n_contract rows, n_out columns]: boxes of 64 contraction rows x 64 output columns
+        ok = ok && make_tensor_map_thd(&map_w, w, n_contract, 1, n_out, ldw, ldw, 64, kGemmBK, 128);
+    if (!ok) return MPIPE_ERR_CUDA;
+    GemmParams p;
+    p.M = M; p.N = n_out; p.K = n_contract;
+    p.tiles_m = cdiv(M, kGemmBM);
+    p.tiles_n = cdiv(n_out, kGemmBN);
+    p.bias = static_cast<const __nv_bfloat16*>(bias);
+    p.residual = static_cast<const __nv_bfloat16*>(residual);
+    p.aux = static_cast<const __nv_bfloat16*>(aux);
+    p.C = static_cast<__nv_bfloat16*>(c);
+    p.ldr = ldr; p.ldx = ldx; p.ldc = ldc;
+    p.gelu = gelu;
+    p.status_buf = status_buf;
+    const long long tiles = (long long)p.tiles_m * p.tiles_n;
+    const int grid = int(tiles < sm_count() ? tiles : sm_count());
+    profile_start(kProfileLinear, st);
+    if (b_mode == 0) {
+        if (cudaFuncSetAttribute(linear_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem) != cudaSuccess) return MPIPE_ERR_CUDA;
+        linear_kernel<0><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, p);
+    } else {
+        if (cudaFuncSetAttribute(linear_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem) != cudaSuccess) return MPIPE_ERR_CUDA;
+        linear_kernel<1><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, p);
+    }
+    profile_stop(kProfileLinear, st);
+    return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
+}
+
+}  // namespace mpipe
+
 extern "C" {
 
 int32_t mpipe_linear_fwd(const void* a, const void* w, const void* bias, const void* residual, void* c, int32_t M,
                          int32_t N, int32_t K, int64_t lda, int64_t ldw, int64_t ldr, int64_t ldc, int32_t flags,
                          int32_t* status_buf, void* stream) {
-    using namespace mpipe;
-    if (M < 0 || N <= 0 || K <= 0) return MPIPE_ERR_INVALID_ARG;
-    if (M == 0) return MPIPE_OK;
-    if (a == nullptr || w == nullptr || c == nullptr) return MPIPE_ERR_INVALID_ARG;
     if ((flags & ~(MPIPE_LINEAR_GELU)) != 0) return MPIPE_ERR_INVALID_ARG;
-    if ((N % 8) != 0 || (K % 8) != 0) return MPIPE_ERR_UNSUPPORTED;
-    if (lda < K || ldw < K || ldc < N || (residual != nullptr && ldr < N)) return MPIPE_ERR_INVALID_ARG;
-    if ((lda % 8) != 0 || (ldw % 8) != 0 || (ldc % 8) != 0 || (residual != nullptr && (ldr % 8) != 0)) return MPIPE_ERR_UNSUPPORTED;
-    if (!aligned16(a) || !aligned16(w) || !aligned16(c) || !aligned16(bias) || !aligned16(residual)) return MPIPE_ERR_UNSUPPORTED;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    CUtensorMap map_a, map_w, map_c;
-    if (!make_tensor_map_thd(&map_a, a, M, 1, K, lda, lda, kGemmBK, kGemmBM, 128) ||
-        !make_tensor_map_thd(&map_w, w, N, 1, K, ldw, ldw, kGemmBK, kGemmBN, 128) ||
-        !make_tensor_map_thd(&map_c, c, M, 1, N, ldc, ldc, 32, kGemmBM, 64))
-        return MPIPE_ERR_CUDA;
-    GemmParams p;
-    p.M = M; p.N = N; p.K = K;
-    p.tiles_m = cdiv(M, kGemmBM);
-    p.tiles_n = cdiv(N, kGemmBN);
-    p.bias = static_cast<const __nv_bfloat16*>(bias);
-    p.residual = static_cast<const __nv_bfloat16*>(residual);
-    p.C = static_cast<__nv_bfloat16*>(c);
-    p.ldr = ldr; p.ldc = ldc;
-    p.gelu = (flags & MPIPE_LINEAR_GELU) ? 1 : 0;
-    p.status_buf = status_buf;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(linear_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem) != cudaSuccess)
-            return MPIPE_ERR_CUDA;
-        attr_set = true;
-    }
-    const long long tiles = (long long)p.tiles_m * p.tiles_n;
-    const int grid = int(tiles < sm_count() ? tiles : sm_count());
-    profile_start(kProfileLinear, st);
-    linear_fwd_kernel<<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, p);
-    profile_stop(kProfileLinear, st);
-    return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
+    return mpipe::launch_linear(0, a, w, bias, residual, nullptr, c, M, N, K, lda, ldw, ldr, 0, ldc,
+                                (flags & MPIPE_LINEAR_GELU) ? 1 : 0, status_buf, stream);
+}
+
+int32_t mpipe_linear_dgrad(const void* dy, const void* w, const void* gelu_input, const void* residual, void* dx, int32_t M,
+                           int32_t N, int32_t K, int64_t lddy, int64_t ldw, int64_t ldu, int64_t ldr, int64_t lddx,
+                           int32_t* status_buf, void* stream) {
+    return mpipe::launch_linear(1, dy, w, nullptr, residual, gelu_input, dx, M, K, N, lddy, ldw, ldr, ldu, lddx, 0, status_buf,
+                                stream);
 }
 
 }  // extern "C"

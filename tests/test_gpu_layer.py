@@ -200,3 +200,23 @@ def test_layer_full_size_sampled_segments():
         lo, hi = int(cu[seg]), int(cu[seg + 1])
         ref, _ = OL.encoder_layer_fwd(x[lo:hi], ow, np.array([0, hi - lo], dtype=np.int32), H, w.softmax_scale, 1e-6)
         assert rel_l2(got[lo:hi], ref) <= LAYER_REL_L2, (seg, rel_l2(got[lo:hi], ref))
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 8, 8), (300, 72, 264), (257, 1024, 512), (1000, 1280, 1024), (129, 64, 3072)])
+@pytest.mark.parametrize("gelu_in,res", [(False, False), (True, False), (False, True)])
+def test_linear_dgrad_matches_oracle(M, N, K, gelu_in, res):
+    dy = W.normal_bf16(15, 0, (M, N))
+    w = W.scaled_normal_bf16(15, 1, (N, K), std=N ** -0.5)
+    u = W.normal_bf16(15, 2, (M, K)) if gelu_in else None
+    r = W.normal_bf16(15, 3, (M, K)) if res else None
+    dx = torch.full((M, K), 7.0, dtype=torch.bfloat16, device="cuda")
+    st = status_buf()
+    B.linear_dgrad(to_dev(dy), to_dev(w), dx, None if u is None else to_dev(u), None if r is None else to_dev(r), st)
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[0] == 0
+    ref = OL.linear_dgrad(OL.widen(dy), OL.widen(w))
+    if gelu_in:
+        ref = ref * OL.gelu_grad(OL.widen(u))
+    if res:
+        ref = ref + OL.widen(r)
+    _check_close(to_f64(dx), ref, atol=2e-3)

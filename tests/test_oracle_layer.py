@@ -150,3 +150,19 @@ def test_layer_with_rope_matches_manual_composition():
     o_ref, _ = oracle.attn_fwd(np.ascontiguousarray(L.rope(q, *tabs)), np.ascontiguousarray(L.rope(k, *tabs)),
                                np.ascontiguousarray(v), cu, 0.25)
     np.testing.assert_allclose(parts["o"], o_ref, atol=1e-14)
+
+
+def test_gelu_grad_and_linear_grads_against_finite_differences_and_autograd():
+    u = np.linspace(-5, 5, 101)
+    h = 1e-6
+    np.testing.assert_allclose(L.gelu_grad(u), (L.gelu(u + h) - L.gelu(u - h)) / (2 * h), atol=1e-9)
+    assert L.gelu_grad(np.array([0.0]))[0] == 0.5
+    rng = np.random.default_rng(8)
+    x, w, b = rng.standard_normal((5, 7)), rng.standard_normal((3, 7)), rng.standard_normal(3)
+    dy = rng.standard_normal((5, 3))
+    xt, wt, bt = (torch.tensor(a, requires_grad=True) for a in (x, w, b))
+    (F.linear(xt, wt, bt) * torch.from_numpy(dy)).sum().backward()
+    np.testing.assert_allclose(L.linear_dgrad(dy, w), xt.grad.numpy(), atol=1e-13)
+    dw, db = L.linear_wgrad(dy, x)
+    np.testing.assert_allclose(dw, wt.grad.numpy(), atol=1e-13)
+    np.testing.assert_allclose(db, bt.grad.numpy(), atol=1e-13)
