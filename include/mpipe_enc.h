@@ -269,6 +269,13 @@ int32_t mpipe_linear_fwd(const void* a, const void* w, const void* bias, const v
 int32_t mpipe_linear_dgrad(const void* dy, const void* w, const void* gelu_input, const void* residual, void* dx, int32_t M,
                            int32_t N, int32_t K, int64_t lddy, int64_t ldw, int64_t ldu, int64_t ldr, int64_t lddx,
                            int32_t* status_buf, void* stream);
+/* Weight gradient of a projection y = x W^T:  dw[N, K] += dy[n_tokens, N]^T x[n_tokens, K], accumulated in fp32 into the
+ * caller's gradient buffer (fp32 device [N, lddw], lddw a multiple of 4; the caller zeroes it at the start of a step
+ * and every microbatch adds to it).  dy, x: bf16 device, row strides multiples of 8, bases 16-byte aligned; N, K
+ * multiples of 8.  The token range is split over CTAs and partial tiles are added with TMA reductions, so the
+ * summation order (and the last bits) can differ from run to run. */
+int32_t mpipe_linear_wgrad(const void* dy, const void* x, float* dw, int32_t n_tokens, int32_t N, int32_t K, int64_t lddy,
+                           int64_t ldx, int64_t lddw, int32_t* status_buf, void* stream);
 int32_t mpipe_layernorm_fwd(const void* x, const void* gamma, const void* beta, void* y, int32_t n_tokens,
                             int32_t hidden, int64_t ldx, int64_t ldy, float eps, void* stream);
 int32_t mpipe_rope_apply(void* qk, int64_t tok_stride, int64_t k_offset, const float* cos_table, const float* sin_table,

@@ -32,6 +32,7 @@ ITEM_DTYPE = np.dtype([(n, np.int32) for n in ("seg", "tile", "row_start", "row_
 
 _i32, _i64, _vp, _f32, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float, ctypes.c_size_t
 _SIGNATURES = {
+    "mpipe_linear_wgrad": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _i64, _i64, _i64, _vp, _vp]),
     "mpipe_linear_dgrad": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _i64, _vp, _vp]),
     "mpipe_ipc_handle_bytes": (_i32, []),
     "mpipe_ipc_export": (_i32, [_vp, _vp]),
@@ -272,6 +273,16 @@ def linear_dgrad(dy, w, dx, gelu_input=None, residual=None, status_buf=None, str
                                    0 if gelu_input is None else _rows(gelu_input), 0 if residual is None else _rows(residual),
                                    _rows(dx), _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_linear_dgrad")
+
+
+def linear_wgrad(dy, x, dw, status_buf=None, stream=None) -> None:
+    """mpipe_linear_wgrad: dw[N,K] (fp32, accumulated in place) += dy[T,N]^T x[T,K]."""
+    T, N = dy.shape
+    K = x.shape[1]
+    assert x.shape[0] == T and tuple(dw.shape) == (N, K) and dw.dtype == torch.float32 and dw.stride(1) == 1
+    st = load().mpipe_linear_wgrad(_ptr(dy), _ptr(x), _ptr(dw), T, N, K, _rows(dy), _rows(x), dw.stride(0), _ptr(status_buf),
+                                   _stream(stream))
+    _check(st, "mpipe_linear_wgrad")
 
 
 def layernorm_fwd(x, gamma, beta, y, eps: float, stream=None) -> None:

@@ -2,6 +2,8 @@
 // (QKV, attention output, MLP) on the token matrix [T, hidden].  bf16 operands, fp32 accumulation in TMEM.
 // mpipe_linear_dgrad: dX[M, K] = epilogue(dY[M, N] * W[N, K]) -- the same kernel with the second operand read as
 // [contraction][output] (an MN-major B: four 64-column atoms per stage, loaded as four TMA boxes).
+// mpipe_linear_wgrad: dW[N, K] += dY[M, N]^T * X[M, K] in fp32 -- both operands MN-major (the token index is the
+// contraction), the token range split over CTAs, partial tiles added with TMA reduce-add.
 //
 // Persistent kernel, one CTA per SM, static round-robin over 128 x 256 output tiles (n fastest, so that the
 // CTAs of a wave share the few weight tiles in L2 and walk down the token rows together).
@@ -44,6 +46,7 @@ struct GemmParams {
     __nv_bfloat16* C;                // [M, ldc]
     int64_t ldr, ldc;
     int32_t gelu;
+    int32_t splits;                  // weight gradient: parts the contraction (token) range is cut into
     int32_t* status_buf;
 };
 
@@ -74,7 +77,9 @@ __device__ __forceinline__ float gelu_erf_grad(float u) {
 }
 
 // kBMode 0: W tile [256 output rows][64 k], K-major (forward).  kBMode 1: W tile [64 contraction rows][256 output
-// columns], MN-major: four [64][64] atoms 8 KB apart (input gradient).
+// columns], MN-major: four [64][64] atoms 8 KB apart (input gradient).  kBMode 2 (weight gradient): as 1, and the first
+// operand too is [64 contraction rows][128 output columns], MN-major, two atoms; work items are (tile, split) pairs and
+// the fp32 result is added to the output with TMA reductions instead of being stored as bf16.
 template <int kBMode>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
@@ -106,8 +111,12 @@ linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
-    const int n_tiles = p.tiles_m * p.tiles_n;
     const int nk = (p.K + kGemmBK - 1) / kGemmBK;
+    const int n_tiles = p.tiles_m * p.tiles_n * (kBMode == 2 ? p.splits : 1);   // work items
+    // work item -> output tile and range of contraction blocks
+    auto tile_of = [&](int t) { return kBMode == 2 ? t / p.splits : t; };
+    auto kb_lo_of = [&](int t) { return kBMode == 2 ? int((long long)(t % p.splits) * nk / p.splits) : 0; };
+    auto kb_hi_of = [&](int t) { return kBMode == 2 ? int((long long)(t % p.splits + 1) * nk / p.splits) : nk; };
 
     if (warp == 0) {
         if (lane == 0) {
@@ -116,14 +125,20 @@ linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             uint32_t it = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-                const int m0 = (t / p.tiles_n) * kGemmBM, n0 = (t % p.tiles_n) * kGemmBN;
-                for (int kb = 0; kb < nk; ++kb, ++it) {
+                const int m0 = (tile_of(t) / p.tiles_n) * kGemmBM, n0 = (tile_of(t) % p.tiles_n) * kGemmBN;
+                for (int kb = kb_lo_of(t); kb < kb_hi_of(t); ++kb, ++it) {
                     const int s = it % kGemmStages;
                     ok = mbar_wait<100>(&bars.empty[s], ((it / kGemmStages) & 1) ^ 1, &abort_flag);
                     if (!ok) break;
                     uint8_t* st = smem + s * kGemmStageBytes;
                     mbar_expect_tx(&bars.full[s], kGemmStageBytes);   // out-of-range rows / columns are zero-filled, still counted
-                    tma_load_3d(st, &map_a, &bars.full[s], kb * kGemmBK, 0, m0);
+                    if (kBMode == 2) {
+#pragma unroll
+                        for (int i = 0; i < kGemmBM / 64; ++i)
+                            tma_load_3d(st + i * (kGemmBK * 128), &map_a, &bars.full[s], m0 + 64 * i, 0, kb * kGemmBK);
+                    } else {
+                        tma_load_3d(st, &map_a, &bars.full[s], kb * kGemmBK, 0, m0);
+                    }
                     if (kBMode == 0) {
                         tma_load_3d(st + kGemmABytes, &map_w, &bars.full[s], kb * kGemmBK, 0, n0);
                     } else {
@@ -139,27 +154,29 @@ linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         const bool leader = elect_one();
         const uint32_t sbase = smem_u32(smem);
         constexpr uint32_t hi128 = umma_desc_hi(1024, kSwizzle128);
-        constexpr uint32_t idesc = umma_idesc_bf16(kGemmBM, kGemmBN, 0, kBMode);
+        constexpr uint32_t idesc = umma_idesc_bf16(kGemmBM, kGemmBN, kBMode == 2 ? 1 : 0, kBMode != 0 ? 1 : 0);
         uint32_t it = 0, tile_it = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_it) {
+            if (kb_lo_of(t) >= kb_hi_of(t)) { --tile_it; continue; }   // an empty split: no role touches it
             const uint32_t acc = tile_it & 1;
             ok = mbar_wait(&bars.acc_empty[acc], ((tile_it >> 1) & 1) ^ 1, &abort_flag);
             if (!ok) break;
             tc_fence_after();
-            for (int kb = 0; kb < nk; ++kb, ++it) {
+            for (int kb = kb_lo_of(t); kb < kb_hi_of(t); ++kb, ++it) {
                 const int s = it % kGemmStages;
                 ok = mbar_wait(&bars.full[s], (it / kGemmStages) & 1, &abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t a_lo = umma_desc_lo(sbase + s * kGemmStageBytes, 0);
+                const uint32_t a_lo = umma_desc_lo(sbase + s * kGemmStageBytes, kBMode == 2 ? kGemmBK * 128 : 0);
+                constexpr uint32_t a_step = kBMode == 2 ? 128 : 2;
                 const uint32_t b_lo = umma_desc_lo(sbase + s * kGemmStageBytes + kGemmABytes, kBMode == 0 ? 0 : kGemmBK * 128);
                 constexpr uint32_t b_step = kBMode == 0 ? 2 : 128;   // one K-step: 32 bytes along a row, or 16 rows of 128 bytes
                 if (leader) {
 #pragma unroll
                     for (int ks = 0; ks < kGemmBK / 16; ++ks)
-                        umma_ss(tmem + acc * kGemmBN, umma_desc(a_lo + ks * 2, hi128), umma_desc(b_lo + ks * b_step, hi128), idesc,
-                                (kb > 0 || ks > 0) ? 1u : 0u);
+                        umma_ss(tmem + acc * kGemmBN, umma_desc(a_lo + ks * a_step, hi128), umma_desc(b_lo + ks * b_step, hi128), idesc,
+                                (kb > kb_lo_of(t) || ks > 0) ? 1u : 0u);
                     umma_commit(&bars.empty[s]);
                 }
             }
@@ -177,10 +194,11 @@ linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         bool ok = true;
         for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile_it) {
             // no early exit: the warpgroup meets at named barriers, so after a time-out it keeps walking empty tiles
+            if (kb_lo_of(t) >= kb_hi_of(t)) { --tile_it; continue; }
             const uint32_t acc = tile_it & 1;
-            const int m0 = (t / p.tiles_n) * kGemmBM;
+            const int m0 = (tile_of(t) / p.tiles_n) * kGemmBM;
             const int m = m0 + r;
-            const int n_base = (t % p.tiles_n) * kGemmBN + wg * (kGemmBN / 2);
+            const int n_base = (tile_of(t) % p.tiles_n) * kGemmBN + wg * (kGemmBN / 2);
             const bool row_ok = m < p.M;
             const __nv_bfloat16* rrow = (p.residual != nullptr && row_ok) ? p.residual + int64_t(m) * p.ldr : nullptr;
             // the residual row is fetched one 32-column chunk ahead (each thread reads its own row: latency, not bandwidth)
@@ -269,6 +287,23 @@ linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                         for (int i = 0; i < 4; ++i) out[4 * g8 + i] = pack_bf16(f[2 * i], f[2 * i + 1]);
                     }
                 }
+                if (kBMode == 2) {   // fp32 partial tile: one [128 rows][32 fp32] box (128-byte swizzle), added to the output
+                    if (wt == 0) bulk_wait_group_read<0>();
+                    named_barrier_sync(1 + wg, 128);
+                    if (ok) {
+#pragma unroll
+                        for (int ch = 0; ch < 8; ++ch)
+                            *reinterpret_cast<uint4*>(boxes + r * 128 + ((ch ^ (r & 7)) << 4)) =
+                                make_uint4(v[4 * ch], v[4 * ch + 1], v[4 * ch + 2], v[4 * ch + 3]);
+                    }
+                    fence_async_smem();
+                    named_barrier_sync(1 + wg, 128);
+                    if (ok && wt == 0) {
+                        tma_reduce_add_3d(&map_c, boxes, n_base + c0, 0, m0);
+                        bulk_commit_group();
+                    }
+                    continue;
+                }
                 uint8_t* box = boxes + (box_it & 1) * kGemmOutBox;
                 if (wt == 0) bulk_wait_group_read<1>();   // the store issued two boxes ago has read this box
                 named_barrier_sync(1 + wg, 128);
@@ -333,6 +368,7 @@ static int32_t launch_linear(int b_mode, const void* a, const void* w, const voi
     p.C = static_cast<__nv_bfloat16*>(c);
     p.ldr = ldr; p.ldx = ldx; p.ldc = ldc;
     p.gelu = gelu;
+    p.splits = 1;
     p.status_buf = status_buf;
     const long long tiles = (long long)p.tiles_m * p.tiles_n;
     const int grid = int(tiles < sm_count() ? tiles : sm_count());
@@ -348,9 +384,56 @@ static int32_t launch_linear(int b_mode, const void* a, const void* w, const voi
     return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
 }
 
+// dW[n_rows, n_cols] (fp32) += dY[tokens, n_rows]^T X[tokens, n_cols]
+static int32_t launch_wgrad(const void* dy, const void* x, float* dw, int32_t tokens, int32_t n_rows, int32_t n_cols, int64_t lddy,
+                            int64_t ldx, int64_t lddw, int32_t* status_buf, void* stream) {
+    if (tokens < 0 || n_rows <= 0 || n_cols <= 0) return MPIPE_ERR_INVALID_ARG;
+    if (tokens == 0) return MPIPE_OK;
+    if (dy == nullptr || x == nullptr || dw == nullptr || lddy < n_rows || ldx < n_cols || lddw < n_cols) return MPIPE_ERR_INVALID_ARG;
+    if ((n_rows % 8) != 0 || (n_cols % 8) != 0 || (lddy % 8) != 0 || (ldx % 8) != 0 || (lddw % 4) != 0) return MPIPE_ERR_UNSUPPORTED;
+    if (!aligned16(dy) || !aligned16(x) || !aligned16(dw)) return MPIPE_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CUtensorMap map_a, map_w, map_c;
+    if (!make_tensor_map_thd(&map_a, dy, tokens, 1, n_rows, lddy, lddy, 64, kGemmBK, 128) ||
+        !make_tensor_map_thd(&map_w, x, tokens, 1, n_cols, ldx, ldx, 64, kGemmBK, 128) ||
+        !make_tensor_map_thd(&map_c, dw, n_rows, 1, n_cols, lddw, lddw, 32, kGemmBM, 128, 4))
+        return MPIPE_ERR_CUDA;
+    GemmParams p;
+    p.M = n_rows; p.N = n_cols; p.K = tokens;
+    p.tiles_m = cdiv(n_rows, kGemmBM);
+    p.tiles_n = cdiv(n_cols, kGemmBN);
+    p.bias = nullptr; p.residual = nullptr; p.aux = nullptr; p.C = nullptr;
+    p.ldr = p.ldx = p.ldc = 0;
+    p.gelu = 0;
+    p.status_buf = status_buf;
+    // split the token range so that (tiles x splits) fills whole waves of the SMs; more splits mean more reduction traffic
+    const int sms = sm_count(), tiles = p.tiles_m * p.tiles_n, nk = cdiv(tokens, kGemmBK);
+    int best = 1;
+    double best_score = -1.0;
+    for (int sp = 1; sp <= 32 && sp <= nk; ++sp) {
+        const long long items = (long long)tiles * sp;
+        const double eff = double(items) / double(((items + sms - 1) / sms) * sms);
+        const double score = eff - 0.004 * sp;
+        if (score > best_score) { best_score = score; best = sp; }
+    }
+    p.splits = best;
+    const long long items = (long long)tiles * p.splits;
+    const int grid = int(items < sms ? items : sms);
+    if (cudaFuncSetAttribute(linear_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem) != cudaSuccess) return MPIPE_ERR_CUDA;
+    profile_start(kProfileLinear, st);
+    linear_kernel<2><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, p);
+    profile_stop(kProfileLinear, st);
+    return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
+}
+
 }  // namespace mpipe
 
 extern "C" {
+
+int32_t mpipe_linear_wgrad(const void* dy, const void* x, float* dw, int32_t n_tokens, int32_t N, int32_t K, int64_t lddy,
+                           int64_t ldx, int64_t lddw, int32_t* status_buf, void* stream) {
+    return mpipe::launch_wgrad(dy, x, dw, n_tokens, N, K, lddy, ldx, lddw, status_buf, stream);
+}
 
 int32_t mpipe_linear_fwd(const void* a, const void* w, const void* bias, const void* residual, void* c, int32_t M,
                          int32_t N, int32_t K, int64_t lda, int64_t ldw, int64_t ldr, int64_t ldc, int32_t flags,

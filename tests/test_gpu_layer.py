@@ -220,3 +220,18 @@ def test_linear_dgrad_matches_oracle(M, N, K, gelu_in, res):
     if res:
         ref = ref + OL.widen(r)
     _check_close(to_f64(dx), ref, atol=2e-3)
+
+
+@pytest.mark.parametrize("T,N,K", [(1, 8, 8), (300, 72, 264), (5000, 1024, 512), (777, 136, 1024), (20000, 256, 256)])
+def test_linear_wgrad_matches_oracle_and_accumulates(T, N, K):
+    dy = W.normal_bf16(16, 0, (T, N))
+    x = W.normal_bf16(16, 1, (T, K))
+    dw = torch.full((N, K), 0.5, dtype=torch.float32, device="cuda")      # accumulates on top of what is there
+    st = status_buf()
+    B.linear_wgrad(to_dev(dy), to_dev(x), dw, st)
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[0] == 0
+    ref, _ = OL.linear_wgrad(OL.widen(dy), OL.widen(x))
+    got = dw.cpu().double().numpy() - 0.5
+    # fp32 accumulation of T exact bf16 products per element
+    assert np.abs(got - ref).max() <= 1e-5 * max(1.0, np.abs(ref).max()) + 4e-7 * T ** 0.5 * 16
