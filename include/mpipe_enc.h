@@ -280,6 +280,20 @@ int32_t mpipe_layernorm_fwd(const void* x, const void* gamma, const void* beta, 
                             int32_t hidden, int64_t ldx, int64_t ldy, float eps, void* stream);
 int32_t mpipe_rope_apply(void* qk, int64_t tok_stride, int64_t k_offset, const float* cos_table, const float* sin_table,
                          int32_t n_tokens, int32_t n_heads, int32_t head_dim, void* stream);
+/* Backward pieces of the layer (exist only for a trainable encoder, Lemma 1):
+ *   mpipe_rope_apply_bwd     the transpose of mpipe_rope_apply (rotation by the opposite angles), in place on dq, dk.
+ *   mpipe_layernorm_bwd      with xhat = (x - mean) rstd and g = dy * gamma:
+ *                              dx = rstd * (g - mean(g) - xhat * mean(g * xhat)) + dres      (dres may be NULL)
+ *                              dgamma[j] += sum_t dy[t,j] xhat[t,j],  dbeta[j] += sum_t dy[t,j]   (fp32, accumulated)
+ *                            x, dy, dres, dx: bf16 [n_tokens, hidden]; mean / rstd are recomputed from x.
+ *   mpipe_colsum_accumulate  out[j] += sum_t a[t, j] in fp32: the bias gradient of a projection from its dy.
+ * The fp32 accumulations use atomics: their last bits can differ from run to run. */
+int32_t mpipe_rope_apply_bwd(void* dqk, int64_t tok_stride, int64_t k_offset, const float* cos_table, const float* sin_table,
+                             int32_t n_tokens, int32_t n_heads, int32_t head_dim, void* stream);
+int32_t mpipe_layernorm_bwd(const void* x, const void* dy, const void* gamma, const void* dres, void* dx, float* dgamma,
+                            float* dbeta, int32_t n_tokens, int32_t hidden, int64_t ldx, int64_t lddy, int64_t ldr,
+                            int64_t lddx, float eps, void* stream);
+int32_t mpipe_colsum_accumulate(const void* a, float* out, int32_t n_tokens, int32_t n_cols, int64_t lda, void* stream);
 size_t mpipe_encoder_layer_workspace_bytes(int32_t n_tokens, int32_t hidden, int32_t ffn);
 int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weights_t* w, int32_t n_tokens,
                                 int32_t hidden, int32_t n_heads, int32_t ffn, const int32_t* cu_seqlens_dev,

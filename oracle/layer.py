@@ -42,6 +42,18 @@ def layernorm(x: np.ndarray, gamma: np.ndarray, beta: np.ndarray, eps: float) ->
     return (x - mean) / np.sqrt(var + eps) * gamma + beta
 
 
+def layernorm_bwd(x: np.ndarray, dy: np.ndarray, gamma: np.ndarray, eps: float):
+    """Gradients of y = xhat * gamma + beta, xhat = (x - mean) / sqrt(var + eps), per row:
+    dx = rstd (g - mean(g) - xhat mean(g xhat)) with g = dy gamma;  dgamma = sum_t dy xhat;  dbeta = sum_t dy."""
+    x, dy = np.asarray(x, dtype=np.float64), np.asarray(dy, dtype=np.float64)
+    mean = x.mean(axis=-1, keepdims=True)
+    rstd = 1.0 / np.sqrt(((x - mean) ** 2).mean(axis=-1, keepdims=True) + eps)
+    xhat = (x - mean) * rstd
+    g = dy * gamma
+    dx = rstd * (g - g.mean(axis=-1, keepdims=True) - xhat * (g * xhat).mean(axis=-1, keepdims=True))
+    return dx, (dy * xhat).sum(axis=0), dy.sum(axis=0)
+
+
 def linear(x: np.ndarray, w: np.ndarray, b=None) -> np.ndarray:
     """y = x w^T + b, w as [out, in]."""
     y = np.asarray(x, dtype=np.float64) @ np.asarray(w, dtype=np.float64).T

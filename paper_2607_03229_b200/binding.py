@@ -32,6 +32,9 @@ ITEM_DTYPE = np.dtype([(n, np.int32) for n in ("seg", "tile", "row_start", "row_
 
 _i32, _i64, _vp, _f32, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float, ctypes.c_size_t
 _SIGNATURES = {
+    "mpipe_rope_apply_bwd": (_i32, [_vp, _i64, _i64, _vp, _vp, _i32, _i32, _i32, _vp]),
+    "mpipe_layernorm_bwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i64, _i64, _i64, _i64, _f32, _vp]),
+    "mpipe_colsum_accumulate": (_i32, [_vp, _vp, _i32, _i32, _i64, _vp]),
     "mpipe_linear_wgrad": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _i64, _i64, _i64, _vp, _vp]),
     "mpipe_linear_dgrad": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i64, _i64, _i64, _i64, _i64, _vp, _vp]),
     "mpipe_ipc_handle_bytes": (_i32, []),
@@ -293,6 +296,31 @@ def layernorm_fwd(x, gamma, beta, y, eps: float, stream=None) -> None:
     st = load().mpipe_layernorm_fwd(_ptr(x), _ptr(gamma), _ptr(beta), _ptr(y), T, hidden, _rows(x), _rows(y), eps,
                                     _stream(stream))
     _check(st, "mpipe_layernorm_fwd")
+
+
+def rope_apply_bwd(dqkv, cos, sin, n_heads: int, head_dim: int, stream=None) -> None:
+    """mpipe_rope_apply_bwd in place on the dq and dk column blocks of a packed gradient dqkv [T, 3*hidden]."""
+    T = dqkv.shape[0]
+    hidden = n_heads * head_dim
+    assert dqkv.shape[1] == 3 * hidden and dqkv.dtype == torch.bfloat16 and dqkv.stride(1) == 1
+    st = load().mpipe_rope_apply_bwd(_ptr(dqkv), dqkv.stride(0), hidden, _ptr(cos), _ptr(sin), T, n_heads, head_dim, _stream(stream))
+    _check(st, "mpipe_rope_apply_bwd")
+
+
+def layernorm_bwd(x, dy, gamma, dx, dgamma, dbeta, eps: float, dres=None, stream=None) -> None:
+    """mpipe_layernorm_bwd; dgamma, dbeta: fp32 [hidden] CUDA tensors that are accumulated into."""
+    T, hidden = x.shape
+    assert dgamma.dtype == dbeta.dtype == torch.float32 and dgamma.numel() == dbeta.numel() == hidden
+    st = load().mpipe_layernorm_bwd(_ptr(x), _ptr(dy), _ptr(gamma), _ptr(dres), _ptr(dx), _ptr(dgamma), _ptr(dbeta), T, hidden,
+                                    _rows(x), _rows(dy), 0 if dres is None else _rows(dres), _rows(dx), eps, _stream(stream))
+    _check(st, "mpipe_layernorm_bwd")
+
+
+def colsum_accumulate(a, out, stream=None) -> None:
+    """mpipe_colsum_accumulate: out[j] (fp32) += sum over rows of a[:, j] (bf16)."""
+    T, N = a.shape
+    assert out.dtype == torch.float32 and out.numel() == N
+    _check(load().mpipe_colsum_accumulate(_ptr(a), _ptr(out), T, N, _rows(a), _stream(stream)), "mpipe_colsum_accumulate")
 
 
 class LayerWeights(ctypes.Structure):

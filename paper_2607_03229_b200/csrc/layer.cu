@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <algorithm>
+
 #include "common.h"
 
 namespace mpipe {
@@ -85,7 +87,7 @@ __global__ void __launch_bounds__(256) layernorm_kernel(const __nv_bfloat16* __r
 // One thread per (token, q|k, head, 8-pair chunk): 2 x 16 bytes in, 2 x 16 bytes out, 2 x 32 bytes of table.
 __global__ void __launch_bounds__(256) rope_kernel(__nv_bfloat16* __restrict__ qk, int64_t tok_stride, int64_t k_offset,
                                                    const float* __restrict__ cos_t, const float* __restrict__ sin_t, int32_t T,
-                                                   int32_t n_heads, int32_t head_dim) {
+                                                   int32_t n_heads, int32_t head_dim, float sin_sign) {
     const int half = head_dim >> 1, chunks = half >> 3;
     const int64_t idx = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
     const int64_t total = int64_t(T) * 2 * n_heads * chunks;
@@ -100,7 +102,9 @@ __global__ void __launch_bounds__(256) rope_kernel(__nv_bfloat16* __restrict__ q
     const float4* sp = reinterpret_cast<const float4*>(sin_t + t * half + c * 8);
     const float4 c0 = __ldg(cp), c1 = __ldg(cp + 1), s0 = __ldg(sp), s1 = __ldg(sp + 1);
     const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-    const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+    // sin_sign = -1 turns by the opposite angle: the transpose of the rotation, i.e. its backward
+    const float sn[8] = {sin_sign * s0.x, sin_sign * s0.y, sin_sign * s0.z, sin_sign * s0.w,
+                         sin_sign * s1.x, sin_sign * s1.y, sin_sign * s1.z, sin_sign * s1.w};
     const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
     uint32_t oa[4], ob[4];
 #pragma unroll
@@ -114,6 +118,148 @@ __global__ void __launch_bounds__(256) rope_kernel(__nv_bfloat16* __restrict__ q
     }
     *reinterpret_cast<uint4*>(x) = make_uint4(oa[0], oa[1], oa[2], oa[3]);
     *reinterpret_cast<uint4*>(x + half) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+}
+
+// LayerNorm backward.  With xhat = (x - mean) rstd and g = dy gamma:  dx = rstd (g - mean(g) - xhat mean(g xhat)) + dres,
+// dgamma += sum_t dy xhat, dbeta += sum_t dy (fp32 atomics, one per column and block).  One warp per row as in the forward;
+// a block walks rows blockIdx.x * 8 + warp, + gridDim.x * 8, ... and keeps its column sums in registers until the end.
+template <int kChunks>
+__global__ void __launch_bounds__(256) layernorm_bwd_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ dy,
+                                                            const __nv_bfloat16* __restrict__ gamma, const __nv_bfloat16* __restrict__ dres,
+                                                            __nv_bfloat16* __restrict__ dx, float* __restrict__ dgamma,
+                                                            float* __restrict__ dbeta, int32_t T, int32_t hidden, int64_t ldx,
+                                                            int64_t lddy, int64_t ldr, int64_t lddx, float eps) {
+    __shared__ float red[2][kChunks * 256];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_chunks = hidden >> 3;
+    float sg[kChunks][8], sb[kChunks][8];
+#pragma unroll
+    for (int i = 0; i < kChunks; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) sg[i][j] = sb[i][j] = 0.f;
+    const uint4* g4 = reinterpret_cast<const uint4*>(gamma);
+    for (int row = blockIdx.x * 8 + warp; row < T; row += gridDim.x * 8) {
+        const uint4* xr = reinterpret_cast<const uint4*>(x + int64_t(row) * ldx);
+        const uint4* dr = reinterpret_cast<const uint4*>(dy + int64_t(row) * lddy);
+        float xv[kChunks][8], gv[kChunks][8];
+        float sum = 0.f;
+#pragma unroll
+        for (int i = 0; i < kChunks; ++i) {
+            const int c = lane + 32 * i;
+            if (c < n_chunks) {
+                const uint4 q = xr[c];
+                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    xv[i][2 * j] = __uint_as_float(w[j] << 16);
+                    xv[i][2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+                    sum += xv[i][2 * j] + xv[i][2 * j + 1];
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        const float mean = sum / float(hidden);
+        float sq = 0.f;
+#pragma unroll
+        for (int i = 0; i < kChunks; ++i)
+            if (lane + 32 * i < n_chunks)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float d = xv[i][j] - mean;
+                    sq = fmaf(d, d, sq);
+                }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        const float rstd = rsqrtf(sq / float(hidden) + eps);
+        float s1 = 0.f, s2 = 0.f;   // sum g, sum g xhat
+#pragma unroll
+        for (int i = 0; i < kChunks; ++i) {
+            const int c = lane + 32 * i;
+            if (c < n_chunks) {
+                const uint4 q = dr[c], gq = __ldg(g4 + c);
+                const uint32_t w[4] = {q.x, q.y, q.z, q.w}, gw[4] = {gq.x, gq.y, gq.z, gq.w};
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float d = (j & 1) ? __uint_as_float(w[j >> 1] & 0xffff0000u) : __uint_as_float(w[j >> 1] << 16);
+                    const float gm = (j & 1) ? __uint_as_float(gw[j >> 1] & 0xffff0000u) : __uint_as_float(gw[j >> 1] << 16);
+                    const float xh = (xv[i][j] - mean) * rstd;
+                    xv[i][j] = xh;
+                    gv[i][j] = d * gm;
+                    s1 += gv[i][j];
+                    s2 = fmaf(gv[i][j], xh, s2);
+                    sg[i][j] = fmaf(d, xh, sg[i][j]);
+                    sb[i][j] += d;
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+            s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+        }
+        const float m1 = s1 / float(hidden), m2 = s2 / float(hidden);
+        uint4* outr = reinterpret_cast<uint4*>(dx + int64_t(row) * lddx);
+        const uint4* rr = dres != nullptr ? reinterpret_cast<const uint4*>(dres + int64_t(row) * ldr) : nullptr;
+#pragma unroll
+        for (int i = 0; i < kChunks; ++i) {
+            const int c = lane + 32 * i;
+            if (c < n_chunks) {
+                uint32_t rw[4] = {0u, 0u, 0u, 0u};
+                if (rr != nullptr) {
+                    const uint4 q = rr[c];
+                    rw[0] = q.x; rw[1] = q.y; rw[2] = q.z; rw[3] = q.w;
+                }
+                uint32_t o[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float lo = rstd * (gv[i][2 * j] - m1 - xv[i][2 * j] * m2) + __uint_as_float(rw[j] << 16);
+                    const float hi = rstd * (gv[i][2 * j + 1] - m1 - xv[i][2 * j + 1] * m2) + __uint_as_float(rw[j] & 0xffff0000u);
+                    const __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
+                    o[j] = *reinterpret_cast<const uint32_t*>(&pk);
+                }
+                outr[c] = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
+    }
+    // column sums: warps -> shared memory -> one atomic per column and block
+    for (int pass = 0; pass < 8; ++pass) {
+        if (warp == pass) {
+#pragma unroll
+            for (int i = 0; i < kChunks; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int col = (lane + 32 * i) * 8 + j;
+                    if (pass == 0) { red[0][col] = sg[i][j]; red[1][col] = sb[i][j]; }
+                    else { red[0][col] += sg[i][j]; red[1][col] += sb[i][j]; }
+                }
+        }
+        __syncthreads();
+    }
+    for (int col = threadIdx.x; col < hidden; col += 256) {
+        atomicAdd(dgamma + col, red[0][col]);
+        atomicAdd(dbeta + col, red[1][col]);
+    }
+}
+
+// out[n] += sum_t a[t, n] (fp32 atomics): the bias gradient of a projection.  blockIdx.x picks 256 chunks of 8 columns,
+// blockIdx.y a slice of the rows.
+__global__ void __launch_bounds__(256) colsum_kernel(const __nv_bfloat16* __restrict__ a, float* __restrict__ out, int32_t T, int32_t N,
+                                                     int64_t lda) {
+    const int chunk = blockIdx.x * 256 + threadIdx.x;
+    if (chunk * 8 >= N) return;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int row = blockIdx.y; row < T; row += gridDim.y) {
+        const uint4 q = *reinterpret_cast<const uint4*>(a + int64_t(row) * lda + chunk * 8);
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            acc[2 * j] += __uint_as_float(w[j] << 16);
+            acc[2 * j + 1] += __uint_as_float(w[j] & 0xffff0000u);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) atomicAdd(out + chunk * 8 + j, acc[j]);
 }
 
 static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
@@ -163,7 +309,63 @@ int32_t mpipe_rope_apply(void* qk, int64_t tok_stride, int64_t k_offset, const f
     const int64_t blocks = (total + 255) / 256;
     if (blocks > 0x7fffffffLL) return MPIPE_ERR_UNSUPPORTED;
     rope_kernel<<<int(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<__nv_bfloat16*>(qk), tok_stride, k_offset, cos_table,
-                                                                           sin_table, n_tokens, n_heads, head_dim);
+                                                                           sin_table, n_tokens, n_heads, head_dim, 1.0f);
+    return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
+}
+
+int32_t mpipe_rope_apply_bwd(void* dqk, int64_t tok_stride, int64_t k_offset, const float* cos_table, const float* sin_table,
+                             int32_t n_tokens, int32_t n_heads, int32_t head_dim, void* stream) {
+    using namespace mpipe;
+    if (n_tokens < 0 || n_heads <= 0 || head_dim <= 0) return MPIPE_ERR_INVALID_ARG;
+    if (n_tokens == 0) return MPIPE_OK;
+    if (dqk == nullptr || cos_table == nullptr || sin_table == nullptr) return MPIPE_ERR_INVALID_ARG;
+    if ((head_dim % 16) != 0 || (tok_stride % 8) != 0 || (k_offset % 8) != 0) return MPIPE_ERR_UNSUPPORTED;
+    if (!aligned16(dqk) || !aligned16(cos_table) || !aligned16(sin_table)) return MPIPE_ERR_UNSUPPORTED;
+    const int64_t total = int64_t(n_tokens) * 2 * n_heads * (head_dim / 16);
+    const int64_t blocks = (total + 255) / 256;
+    if (blocks > 0x7fffffffLL) return MPIPE_ERR_UNSUPPORTED;
+    rope_kernel<<<int(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<__nv_bfloat16*>(dqk), tok_stride, k_offset, cos_table,
+                                                                           sin_table, n_tokens, n_heads, head_dim, -1.0f);
+    return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
+}
+
+int32_t mpipe_layernorm_bwd(const void* x, const void* dy, const void* gamma, const void* dres, void* dx, float* dgamma, float* dbeta,
+                            int32_t n_tokens, int32_t hidden, int64_t ldx, int64_t lddy, int64_t ldr, int64_t lddx, float eps,
+                            void* stream) {
+    using namespace mpipe;
+    if (n_tokens < 0 || hidden <= 0 || !(eps >= 0.f)) return MPIPE_ERR_INVALID_ARG;
+    if (n_tokens == 0) return MPIPE_OK;
+    if (x == nullptr || dy == nullptr || gamma == nullptr || dx == nullptr || dgamma == nullptr || dbeta == nullptr) return MPIPE_ERR_INVALID_ARG;
+    if (ldx < hidden || lddy < hidden || lddx < hidden || (dres != nullptr && ldr < hidden)) return MPIPE_ERR_INVALID_ARG;
+    if ((hidden % 8) != 0 || hidden > kLnMaxChunks * 256 || (ldx % 8) != 0 || (lddy % 8) != 0 || (lddx % 8) != 0 ||
+        (dres != nullptr && (ldr % 8) != 0))
+        return MPIPE_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(dy) || !aligned16(gamma) || !aligned16(dres) || !aligned16(dx)) return MPIPE_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int grid = std::min(cdiv(n_tokens, 8), sm_count() * 4);
+    const int chunks = cdiv(hidden, 256);
+#define MPIPE_LNB_LAUNCH(C)                                                                                                    \
+    layernorm_bwd_kernel<C><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy),   \
+                                                  static_cast<const __nv_bfloat16*>(gamma), static_cast<const __nv_bfloat16*>(dres), \
+                                                  static_cast<__nv_bfloat16*>(dx), dgamma, dbeta, n_tokens, hidden, ldx, lddy, ldr, lddx, eps)
+    if (chunks <= 1) MPIPE_LNB_LAUNCH(1);
+    else if (chunks <= 2) MPIPE_LNB_LAUNCH(2);
+    else if (chunks <= 4) MPIPE_LNB_LAUNCH(4);
+    else if (chunks <= 5) MPIPE_LNB_LAUNCH(5);
+    else MPIPE_LNB_LAUNCH(kLnMaxChunks);
+#undef MPIPE_LNB_LAUNCH
+    return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
+}
+
+int32_t mpipe_colsum_accumulate(const void* a, float* out, int32_t n_tokens, int32_t n_cols, int64_t lda, void* stream) {
+    using namespace mpipe;
+    if (n_tokens < 0 || n_cols <= 0) return MPIPE_ERR_INVALID_ARG;
+    if (n_tokens == 0) return MPIPE_OK;
+    if (a == nullptr || out == nullptr || lda < n_cols) return MPIPE_ERR_INVALID_ARG;
+    if ((n_cols % 8) != 0 || (lda % 8) != 0 || !aligned16(a)) return MPIPE_ERR_UNSUPPORTED;
+    const int gx = cdiv(n_cols / 8, 256);
+    const int gy = std::max(1, std::min(n_tokens, (sm_count() * 8) / gx));
+    colsum_kernel<<<dim3(gx, gy), 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const __nv_bfloat16*>(a), out, n_tokens, n_cols, lda);
     return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
 }
 

@@ -235,3 +235,49 @@ def test_linear_wgrad_matches_oracle_and_accumulates(T, N, K):
     got = dw.cpu().double().numpy() - 0.5
     # fp32 accumulation of T exact bf16 products per element
     assert np.abs(got - ref).max() <= 1e-5 * max(1.0, np.abs(ref).max()) + 4e-7 * T ** 0.5 * 16
+
+
+@pytest.mark.parametrize("T,hidden", [(1, 8), (37, 256), (3000, 1024), (513, 1280), (9, 2048)])
+@pytest.mark.parametrize("with_res", [False, True])
+def test_layernorm_bwd_matches_oracle(T, hidden, with_res):
+    x = W.scaled_normal_bf16(17, 0, (T, hidden), std=2.0, mean=0.7)
+    dy = W.normal_bf16(17, 1, (T, hidden))
+    g = W.scaled_normal_bf16(17, 2, (hidden,), std=0.1, mean=1.0)
+    r = W.normal_bf16(17, 3, (T, hidden)) if with_res else None
+    dx = torch.empty((T, hidden), dtype=torch.bfloat16, device="cuda")
+    dg = torch.full((hidden,), 0.25, dtype=torch.float32, device="cuda")
+    db = torch.full((hidden,), -0.5, dtype=torch.float32, device="cuda")
+    B.layernorm_bwd(to_dev(x), to_dev(dy), to_dev(g), dx, dg, db, 1e-6, None if r is None else to_dev(r))
+    torch.cuda.synchronize()
+    dx_ref, dg_ref, db_ref = OL.layernorm_bwd(OL.widen(x), OL.widen(dy), OL.widen(g), 1e-6)
+    if with_res:
+        dx_ref = dx_ref + OL.widen(r)
+    _check_close(to_f64(dx), dx_ref, atol=2e-4)
+    tol = 1e-5 * max(1.0, np.abs(dg_ref).max()) + 2e-6 * T ** 0.5 * 8
+    assert np.abs(dg.cpu().double().numpy() - 0.25 - dg_ref).max() <= tol
+    assert np.abs(db.cpu().double().numpy() + 0.5 - db_ref).max() <= tol
+
+
+@pytest.mark.parametrize("T,N", [(1, 8), (777, 264), (20000, 3072)])
+def test_colsum_matches_oracle(T, N):
+    a = W.normal_bf16(18, 0, (T, N))
+    out = torch.full((N,), 2.0, dtype=torch.float32, device="cuda")
+    B.colsum_accumulate(to_dev(a), out)
+    torch.cuda.synchronize()
+    ref = OL.widen(a).sum(axis=0)
+    assert np.abs(out.cpu().double().numpy() - 2.0 - ref).max() <= 1e-5 * max(1.0, np.abs(ref).max()) + 1e-6 * T ** 0.5 * 8
+
+
+def test_rope_bwd_is_the_transpose_of_rope():
+    counts, H, D = [300, 77], 3, 80
+    T, hidden = sum(counts), H * D
+    g = W.normal_bf16(19, 0, (T, 3 * hidden))
+    cos, sin = W.rope2d_tables(counts, D)
+    dev = to_dev(g)
+    B.rope_apply_bwd(dev, torch.from_numpy(cos).cuda(), torch.from_numpy(sin).cuda(), H, D)
+    torch.cuda.synchronize()
+    ref = OL.widen(g).copy()
+    for i in range(2):   # the transpose of a rotation is the rotation by the opposite angle
+        blk = ref[:, i * hidden:(i + 1) * hidden].reshape(T, H, D)
+        ref[:, i * hidden:(i + 1) * hidden] = OL.rope(blk, cos.astype(np.float64), -sin.astype(np.float64)).reshape(T, hidden)
+    _check_close(to_f64(dev), ref, atol=1e-6)

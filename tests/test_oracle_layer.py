@@ -166,3 +166,16 @@ def test_gelu_grad_and_linear_grads_against_finite_differences_and_autograd():
     dw, db = L.linear_wgrad(dy, x)
     np.testing.assert_allclose(dw, wt.grad.numpy(), atol=1e-13)
     np.testing.assert_allclose(db, bt.grad.numpy(), atol=1e-13)
+
+
+def test_layernorm_bwd_matches_autograd():
+    rng = np.random.default_rng(9)
+    x, dy = rng.standard_normal((6, 24)) * 2 + 1, rng.standard_normal((6, 24))
+    g, b = 1 + 0.2 * rng.standard_normal(24), rng.standard_normal(24)
+    xt, gt, bt = (torch.tensor(a, requires_grad=True) for a in (x, g, b))
+    (F.layer_norm(xt, (24,), gt, bt, 1e-6) * torch.from_numpy(dy)).sum().backward()
+    dx, dg, db = L.layernorm_bwd(x, dy, g, 1e-6)
+    np.testing.assert_allclose(dx, xt.grad.numpy(), atol=1e-12)
+    np.testing.assert_allclose(dg, gt.grad.numpy(), atol=1e-12)
+    np.testing.assert_allclose(db, bt.grad.numpy(), atol=1e-12)
+    np.testing.assert_allclose(dx.sum(axis=1), 0, atol=1e-12)      # the normalised value does not see a shift of the row
