@@ -217,9 +217,9 @@ int32_t mpipe_validate_positions(const int32_t* positions, int32_t n, int32_t n_
 /*
  * The rest of the packed encoder layer -- what one Fwd(enc, r, m) event of the transpose schedule executes
  * besides attention (Section 4.2; the paper says only "ViT-style encoder", Section 2: the block below is the
- * pre-norm Transformer block of that family).  Forward only: it is the whole layer of a FROZEN encoder
- * (Lemma 1: no backward events exist then); for a TRAINED one it also writes the LSE that
- * mpipe_varlen_attn_bwd needs, the backward of the projections and norms is not part of this library yet.
+ * pre-norm Transformer block of that family).  The forward is the whole layer of a FROZEN encoder (Lemma 1: no
+ * backward events exist then); for a TRAINED one it also writes the LSE, and mpipe_encoder_layer_bwd below is its
+ * backward.
  *
  *   mpipe_linear_fwd     C[M, N] = act(A[M, K] W[N, K]^T + bias[N]) + residual[M, N]; all bf16, device, row-major
  *                        with row strides lda / ldw / ldr / ldc in elements (multiples of 8, bases 16-byte
@@ -294,6 +294,29 @@ int32_t mpipe_layernorm_bwd(const void* x, const void* dy, const void* gamma, co
                             float* dbeta, int32_t n_tokens, int32_t hidden, int64_t ldx, int64_t lddy, int64_t ldr,
                             int64_t lddx, float eps, void* stream);
 int32_t mpipe_colsum_accumulate(const void* a, float* out, int32_t n_tokens, int32_t n_cols, int64_t lda, void* stream);
+/*
+ * Bwd(enc, r, m) of the same layer -- exists only when the encoder is trainable (Lemma 1).  Given dy = dL/dy it writes
+ * dx = dL/dx (bf16 [n_tokens, hidden]) and ADDS the parameter gradients, in fp32, to the twelve buffers of `grads`
+ * (same shapes as the weights; the caller zeroes them at the start of a step, every microbatch accumulates).
+ * fwd_workspace is the workspace of the matching mpipe_encoder_layer_fwd call (TRAINED mode, same x, weights, plan and
+ * rope tables), untouched since: it holds the rotated q | k | v, the attention output, x1 and GELU(u); its LN slot is
+ * overwritten here.  lse is that call's LSE.  The two LayerNorm outputs and the MLP pre-activation u are recomputed
+ * (one extra projection) instead of being stored by the forward.  workspace: device, 256-byte aligned,
+ * >= mpipe_encoder_layer_bwd_workspace_bytes.  About twenty launches on `stream`, nothing allocated.  bwd_items_dev /
+ * n_bwd_items are the plan's backward list.  Sums over tokens use fp32 atomics and TMA reductions: parameter gradients
+ * are reproducible to rounding order only.
+ */
+typedef struct {
+    float *ln1_gamma, *ln1_beta, *w_qkv, *b_qkv, *w_o, *b_o, *ln2_gamma, *ln2_beta, *w_fc1, *b_fc1, *w_fc2, *b_fc2;
+} mpipe_layer_grads_t;
+size_t mpipe_encoder_layer_bwd_workspace_bytes(int32_t n_tokens, int32_t hidden, int32_t n_heads, int32_t ffn);
+int32_t mpipe_encoder_layer_bwd(const void* dy, const void* x, void* dx, const mpipe_layer_weights_t* w,
+                                const mpipe_layer_grads_t* grads, int32_t n_tokens, int32_t hidden, int32_t n_heads,
+                                int32_t ffn, const int32_t* cu_seqlens_dev, int32_t n_seg, int32_t max_seqlen,
+                                const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items, float softmax_scale,
+                                float ln_eps, const float* rope_cos, const float* rope_sin, const float* lse,
+                                void* fwd_workspace, void* workspace, size_t workspace_bytes, int32_t* status_buf,
+                                void* stream);
 size_t mpipe_encoder_layer_workspace_bytes(int32_t n_tokens, int32_t hidden, int32_t ffn);
 int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weights_t* w, int32_t n_tokens,
                                 int32_t hidden, int32_t n_heads, int32_t ffn, const int32_t* cu_seqlens_dev,

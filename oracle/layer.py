@@ -26,7 +26,7 @@ from dataclasses import dataclass
 
 import numpy as np
 
-from . import _f64, attn_fwd
+from . import _f64, attn_bwd, attn_fwd
 
 
 def widen(a) -> np.ndarray:
@@ -133,3 +133,38 @@ def encoder_layer_fwd(x, w: LayerWeights, cu_seqlens, n_heads: int, scale: float
     f = gelu(linear(m, w.w1, w.bb1))
     y = x1 + linear(f, w.w2, w.bb2)
     return y, {"a": a, "qkv": qkv, "o": o, "lse": lse, "x1": x1, "m": m, "f": f}
+
+
+def encoder_layer_bwd(x, w: LayerWeights, cu_seqlens, n_heads: int, scale: float, eps: float, dy, rope_tables=None):
+    """Gradient of the whole block by the chain rule, stage by stage in reverse (each stage's own gradient is one of the
+    functions above or oracle.attn_bwd).  Returns dx [T, hidden] and a dict of the twelve parameter gradients."""
+    x, dy = widen(x), np.asarray(widen(dy), dtype=np.float64)
+    T, hidden = x.shape
+    D = hidden // n_heads
+    _, p = encoder_layer_fwd(x, w, cu_seqlens, n_heads, scale, eps, rope_tables)
+    u = linear(p["m"], w.w1, w.bb1)
+    g = {}
+    # y = x1 + f W2^T + bb2
+    g["w_fc2"], g["b_fc2"] = linear_wgrad(dy, p["f"])
+    du = linear_dgrad(dy, w.w2) * gelu_grad(u)
+    g["w_fc1"], g["b_fc1"] = linear_wgrad(du, p["m"])
+    dm = linear_dgrad(du, w.w1)
+    dln, g["ln2_gamma"], g["ln2_beta"] = layernorm_bwd(p["x1"], dm, w.g2, eps)
+    dx1 = dy + dln
+    # x1 = x + o Wo^T + bo
+    o2 = p["o"].reshape(T, hidden)
+    g["w_o"], g["b_o"] = linear_wgrad(dx1, o2)
+    do = linear_dgrad(dx1, w.wo).reshape(T, n_heads, D)
+    qkv = p["qkv"]
+    q, k, v = (np.ascontiguousarray(qkv[:, i * hidden:(i + 1) * hidden].reshape(T, n_heads, D)) for i in range(3))
+    if rope_tables is not None:
+        q, k = rope(q, *rope_tables), rope(k, *rope_tables)
+    dq, dk, dv = attn_bwd(np.ascontiguousarray(do), q, k, v, cu_seqlens, scale)
+    if rope_tables is not None:   # the transpose of a rotation is the rotation by the opposite angle
+        c, s_ = rope_tables
+        dq, dk = rope(dq, c, -np.asarray(s_)), rope(dk, c, -np.asarray(s_))
+    dqkv = np.concatenate([t.reshape(T, hidden) for t in (dq, dk, dv)], axis=1)
+    g["w_qkv"], g["b_qkv"] = linear_wgrad(dqkv, p["a"])
+    da = linear_dgrad(dqkv, w.wqkv)
+    dln, g["ln1_gamma"], g["ln1_beta"] = layernorm_bwd(x, da, w.g1, eps)
+    return dx1 + dln, g

@@ -32,6 +32,9 @@ ITEM_DTYPE = np.dtype([(n, np.int32) for n in ("seg", "tile", "row_start", "row_
 
 _i32, _i64, _vp, _f32, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float, ctypes.c_size_t
 _SIGNATURES = {
+    "mpipe_encoder_layer_bwd_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32]),
+    "mpipe_encoder_layer_bwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _i32, _i32, _vp, _i32, _f32, _f32,
+                                       _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "mpipe_rope_apply_bwd": (_i32, [_vp, _i64, _i64, _vp, _vp, _i32, _i32, _i32, _vp]),
     "mpipe_layernorm_bwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i64, _i64, _i64, _i64, _f32, _vp]),
     "mpipe_colsum_accumulate": (_i32, [_vp, _vp, _i32, _i32, _i64, _vp]),
@@ -337,6 +340,39 @@ class LayerWeights(ctypes.Structure):
             setattr(w, name, t.data_ptr())
         w._keep = tensors
         return w
+
+
+class LayerGrads(ctypes.Structure):
+    """mpipe_layer_grads_t: twelve fp32 device pointers, same order and shapes as LayerWeights; accumulated into."""
+    _fields_ = LayerWeights._fields_
+
+    @classmethod
+    def from_tensors(cls, **tensors) -> "LayerGrads":
+        g = cls()
+        for name, _ in cls._fields_:
+            t = tensors[name]
+            assert t.dtype == torch.float32 and t.is_cuda and t.is_contiguous(), name
+            setattr(g, name, t.data_ptr())
+        g._keep = tensors
+        return g
+
+
+def encoder_layer_bwd_workspace_bytes(n_tokens: int, hidden: int, n_heads: int, ffn: int) -> int:
+    return load().mpipe_encoder_layer_bwd_workspace_bytes(n_tokens, hidden, n_heads, ffn)
+
+
+def encoder_layer_bwd(dy, x, dx, weights: LayerWeights, grads: LayerGrads, n_heads: int, ffn: int, plan: SegPlan,
+                      softmax_scale: float, ln_eps: float, lse, fwd_workspace, workspace, status_buf=None, stream=None,
+                      rope=None) -> None:
+    """mpipe_encoder_layer_bwd: dy, x, dx bf16 [T, hidden] contiguous; fwd_workspace untouched since the matching forward."""
+    T, hidden = x.shape
+    assert plan.mode == TRAINED and dy.is_contiguous() and x.is_contiguous() and dx.is_contiguous()
+    st = load().mpipe_encoder_layer_bwd(
+        _ptr(dy), _ptr(x), _ptr(dx), ctypes.addressof(weights), ctypes.addressof(grads), T, hidden, n_heads, ffn,
+        _ptr(plan.cu_seqlens_dev), plan.n_seg, plan.max_seqlen, _ptr(plan.bwd_items_dev), int(plan.bwd_items.size), softmax_scale,
+        ln_eps, _ptr(None if rope is None else rope[0]), _ptr(None if rope is None else rope[1]), _ptr(lse), _ptr(fwd_workspace),
+        _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status_buf), _stream(stream))
+    _check(st, "mpipe_encoder_layer_bwd")
 
 
 def encoder_layer_workspace_bytes(n_tokens: int, hidden: int, ffn: int) -> int:

@@ -420,4 +420,76 @@ int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weight
     return mpipe_linear_fwd(fc1, w->w_fc2, w->b_fc2, x1, y, n_tokens, hidden, ffn, ffn, ffn, hidden, hidden, 0, status_buf, stream);
 }
 
+size_t mpipe_encoder_layer_bwd_workspace_bytes(int32_t n_tokens, int32_t hidden, int32_t n_heads, int32_t ffn) {
+    using namespace mpipe;
+    if (n_tokens <= 0 || hidden <= 0 || n_heads <= 0 || ffn <= 0 || (hidden % n_heads) != 0) return 0;
+    const size_t t = size_t(n_tokens);
+    // pre-activation u, dL/du, dL/dqkv, dL/dx1, one [T, hidden] temporary, the attention backward's own workspace
+    return 2 * align256(t * ffn * 2) + align256(t * 3 * hidden * 2) + 2 * align256(t * hidden * 2) +
+           align256(mpipe_attn_workspace_bytes(n_tokens, n_heads, hidden / n_heads, MPIPE_ENC_TRAINED));
+}
+
+int32_t mpipe_encoder_layer_bwd(const void* dy, const void* x, void* dx, const mpipe_layer_weights_t* w, const mpipe_layer_grads_t* g,
+                                int32_t n_tokens, int32_t hidden, int32_t n_heads, int32_t ffn, const int32_t* cu_seqlens_dev,
+                                int32_t n_seg, int32_t max_seqlen, const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items,
+                                float softmax_scale, float ln_eps, const float* rope_cos, const float* rope_sin, const float* lse,
+                                void* fwd_workspace, void* workspace, size_t workspace_bytes, int32_t* status_buf, void* stream) {
+    using namespace mpipe;
+    if (n_tokens < 0 || hidden <= 0 || n_heads <= 0 || ffn <= 0 || w == nullptr || g == nullptr) return MPIPE_ERR_INVALID_ARG;
+    if (n_tokens == 0) return MPIPE_OK;
+    if (dy == nullptr || x == nullptr || dx == nullptr || lse == nullptr || fwd_workspace == nullptr || (hidden % n_heads) != 0)
+        return MPIPE_ERR_INVALID_ARG;
+    if ((rope_cos == nullptr) != (rope_sin == nullptr)) return MPIPE_ERR_INVALID_ARG;
+    if (workspace == nullptr || workspace_bytes < mpipe_encoder_layer_bwd_workspace_bytes(n_tokens, hidden, n_heads, ffn))
+        return MPIPE_ERR_WORKSPACE;
+    if (((reinterpret_cast<uintptr_t>(workspace) | reinterpret_cast<uintptr_t>(fwd_workspace)) & 255u) != 0) return MPIPE_ERR_UNSUPPORTED;
+    const int32_t head_dim = hidden / n_heads;
+    const size_t t = size_t(n_tokens);
+    const int64_t h = hidden, h3 = 3 * int64_t(hidden), f = ffn;
+    // what the forward left in its workspace: LN output (stale), packed q|k|v (q, k rotated), attention output, x1, GELU(u)
+    uint8_t* fw = static_cast<uint8_t*>(fwd_workspace);
+    uint8_t* norm = fw;               fw += align256(t * hidden * 2);
+    uint8_t* qkv = fw;                fw += align256(t * 3 * hidden * 2);
+    uint8_t* attn = fw;               fw += align256(t * hidden * 2);
+    uint8_t* x1 = fw;                 fw += align256(t * hidden * 2);
+    uint8_t* act = fw;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    uint8_t* ubuf = ws;               ws += align256(t * ffn * 2);
+    uint8_t* dubuf = ws;              ws += align256(t * ffn * 2);
+    uint8_t* dqkv = ws;               ws += align256(t * 3 * hidden * 2);
+    uint8_t* dx1 = ws;                ws += align256(t * hidden * 2);
+    uint8_t* tmp = ws;                ws += align256(t * hidden * 2);
+    uint8_t* attn_ws = ws;
+    const size_t attn_ws_bytes = mpipe_attn_workspace_bytes(n_tokens, n_heads, head_dim, MPIPE_ENC_TRAINED);
+    int32_t rc;
+#define MPIPE_TRY(call) do { if ((rc = (call)) != MPIPE_OK) return rc; } while (0)
+    // ---- MLP branch: y = x1 + GELU(m W1^T + b1) W2^T + b2, m = LN2(x1)
+    MPIPE_TRY(mpipe_layernorm_fwd(x1, w->ln2_gamma, w->ln2_beta, norm, n_tokens, hidden, h, h, ln_eps, stream));                 // m
+    MPIPE_TRY(mpipe_linear_wgrad(dy, act, g->w_fc2, n_tokens, hidden, ffn, h, f, f, status_buf, stream));                          // dW2 += dy^T GELU(u)
+    MPIPE_TRY(mpipe_colsum_accumulate(dy, g->b_fc2, n_tokens, hidden, h, stream));
+    MPIPE_TRY(mpipe_linear_fwd(norm, w->w_fc1, w->b_fc1, nullptr, ubuf, n_tokens, ffn, hidden, h, h, 0, f, 0, status_buf, stream)); // u (recomputed)
+    MPIPE_TRY(mpipe_linear_dgrad(dy, w->w_fc2, ubuf, nullptr, dubuf, n_tokens, hidden, ffn, h, f, f, 0, f, status_buf, stream));    // du = (dy W2) o GELU'(u)
+    MPIPE_TRY(mpipe_linear_wgrad(dubuf, norm, g->w_fc1, n_tokens, ffn, hidden, f, h, h, status_buf, stream));                     // dW1 += du^T m
+    MPIPE_TRY(mpipe_colsum_accumulate(dubuf, g->b_fc1, n_tokens, ffn, f, stream));
+    MPIPE_TRY(mpipe_linear_dgrad(dubuf, w->w_fc1, nullptr, nullptr, tmp, n_tokens, ffn, hidden, f, h, 0, 0, h, status_buf, stream)); // dm = du W1
+    MPIPE_TRY(mpipe_layernorm_bwd(x1, tmp, w->ln2_gamma, dy, dx1, g->ln2_gamma, g->ln2_beta, n_tokens, hidden, h, h, h, h, ln_eps, stream)); // dx1 = dy + LN2'(dm)
+    // ---- attention branch: x1 = x + o Wo^T + bo, o = attention(rope(a Wqkv^T + bqkv)), a = LN1(x)
+    MPIPE_TRY(mpipe_linear_wgrad(dx1, attn, g->w_o, n_tokens, hidden, hidden, h, h, h, status_buf, stream));                       // dWo += dx1^T o
+    MPIPE_TRY(mpipe_colsum_accumulate(dx1, g->b_o, n_tokens, hidden, h, stream));
+    MPIPE_TRY(mpipe_linear_dgrad(dx1, w->w_o, nullptr, nullptr, tmp, n_tokens, hidden, hidden, h, h, 0, 0, h, status_buf, stream)); // do = dx1 Wo
+    MPIPE_TRY(mpipe_varlen_attn_bwd(tmp, qkv, qkv + size_t(hidden) * 2, qkv + size_t(hidden) * 4, attn, lse, dqkv, dqkv + size_t(hidden) * 2,
+                                    dqkv + size_t(hidden) * 4, h3, head_dim, h, head_dim, h3, head_dim, cu_seqlens_dev, n_seg, n_tokens,
+                                    max_seqlen, bwd_items_dev, n_bwd_items, n_heads, head_dim, softmax_scale, MPIPE_ENC_TRAINED, attn_ws,
+                                    attn_ws_bytes, status_buf, stream));
+    if (rope_cos != nullptr)
+        MPIPE_TRY(mpipe_rope_apply_bwd(dqkv, h3, hidden, rope_cos, rope_sin, n_tokens, n_heads, head_dim, stream));
+    MPIPE_TRY(mpipe_layernorm_fwd(x, w->ln1_gamma, w->ln1_beta, norm, n_tokens, hidden, h, h, ln_eps, stream));                    // a (recomputed)
+    MPIPE_TRY(mpipe_linear_wgrad(dqkv, norm, g->w_qkv, n_tokens, 3 * hidden, hidden, h3, h, h, status_buf, stream));               // dWqkv += dqkv^T a
+    MPIPE_TRY(mpipe_colsum_accumulate(dqkv, g->b_qkv, n_tokens, 3 * hidden, h3, stream));
+    MPIPE_TRY(mpipe_linear_dgrad(dqkv, w->w_qkv, nullptr, nullptr, tmp, n_tokens, 3 * hidden, hidden, h3, h, 0, 0, h, status_buf, stream)); // da = dqkv Wqkv
+    MPIPE_TRY(mpipe_layernorm_bwd(x, tmp, w->ln1_gamma, dx1, dx, g->ln1_gamma, g->ln1_beta, n_tokens, hidden, h, h, h, h, ln_eps, stream)); // dx = dx1 + LN1'(da)
+#undef MPIPE_TRY
+    return MPIPE_OK;
+}
+
 }  // extern "C"

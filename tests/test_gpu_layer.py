@@ -281,3 +281,43 @@ def test_rope_bwd_is_the_transpose_of_rope():
         blk = ref[:, i * hidden:(i + 1) * hidden].reshape(T, H, D)
         ref[:, i * hidden:(i + 1) * hidden] = OL.rope(blk, cos.astype(np.float64), -sin.astype(np.float64)).reshape(T, hidden)
     _check_close(to_f64(dev), ref, atol=1e-6)
+
+
+GRAD_REL_L2 = 1.5e-2    # the backward chains ~10 bf16-rounded stages (recomputed activations included)
+
+
+@pytest.mark.parametrize("counts,H,D,ffn,rope", [([16, 49, 64, 100], 4, 64, 1024, False), ([300, 1, 129, 640], 4, 80, 1280, True),
+                                                  ([1024, 256, 777], 16, 64, 4096, False)])
+def test_layer_bwd_matches_oracle(counts, H, D, ffn, rope):
+    hidden, T = H * D, sum(counts)
+    pb = W.layer_params_bf16(23, hidden, ffn)
+    x, dy = W.normal_bf16(23, 0, (T, hidden)), W.normal_bf16(23, 1, (T, hidden))
+    plan = B.seg_plan(counts, B.TRAINED).to_device()
+    weights = B.LayerWeights.from_tensors(**{k: to_dev(v) for k, v in pb.items()})
+    grads_t = {k: torch.zeros(v.shape, dtype=torch.float32, device="cuda") for k, v in pb.items()}
+    grads = B.LayerGrads.from_tensors(**grads_t)
+    xd, dyd = to_dev(x), to_dev(dy)
+    y, dx = torch.empty_like(xd), torch.empty_like(xd)
+    lse = torch.empty((H, T), dtype=torch.float32, device="cuda")
+    ws_f = torch.empty(B.encoder_layer_workspace_bytes(T, hidden, ffn), dtype=torch.uint8, device="cuda")
+    ws_b = torch.empty(B.encoder_layer_bwd_workspace_bytes(T, hidden, H, ffn), dtype=torch.uint8, device="cuda")
+    st = status_buf()
+    scale = float(np.float32(1 / math.sqrt(D)))
+    tabs = W.rope2d_tables(counts, D) if rope else None
+    rope_dev = None if tabs is None else tuple(torch.from_numpy(t).cuda() for t in tabs)
+    B.encoder_layer_fwd(xd, y, weights, H, ffn, plan, scale, 1e-6, ws_f, lse, st, rope=rope_dev)
+    for _ in range(2):      # two microbatches: parameter gradients accumulate, dx is overwritten
+        B.encoder_layer_bwd(dyd, xd, dx, weights, grads, H, ffn, plan, scale, 1e-6, lse, ws_f, ws_b, st, rope=rope_dev)
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[0] == 0
+    ow = OL.LayerWeights(g1=OL.widen(pb["ln1_gamma"]), b1=OL.widen(pb["ln1_beta"]), wqkv=OL.widen(pb["w_qkv"]),
+                         bqkv=OL.widen(pb["b_qkv"]), wo=OL.widen(pb["w_o"]), bo=OL.widen(pb["b_o"]),
+                         g2=OL.widen(pb["ln2_gamma"]), b2=OL.widen(pb["ln2_beta"]), w1=OL.widen(pb["w_fc1"]),
+                         bb1=OL.widen(pb["b_fc1"]), w2=OL.widen(pb["w_fc2"]), bb2=OL.widen(pb["b_fc2"]))
+    cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    dx_ref, g_ref = OL.encoder_layer_bwd(x, ow, cu, H, scale, 1e-6, dy,
+                                         None if tabs is None else tuple(t.astype(np.float64) for t in tabs))
+    assert rel_l2(to_f64(dx), dx_ref) <= GRAD_REL_L2, rel_l2(to_f64(dx), dx_ref)
+    for name, ref in g_ref.items():
+        got = grads_t[name].cpu().double().numpy() / 2.0
+        assert rel_l2(got, ref.reshape(got.shape)) <= GRAD_REL_L2, (name, rel_l2(got, ref.reshape(got.shape)))

@@ -179,3 +179,56 @@ def test_layernorm_bwd_matches_autograd():
     np.testing.assert_allclose(dg, gt.grad.numpy(), atol=1e-12)
     np.testing.assert_allclose(db, bt.grad.numpy(), atol=1e-12)
     np.testing.assert_allclose(dx.sum(axis=1), 0, atol=1e-12)      # the normalised value does not see a shift of the row
+
+
+@pytest.mark.parametrize("with_rope", [False, True])
+def test_layer_bwd_matches_torch_autograd(with_rope):
+    rng = np.random.default_rng(10)
+    counts, H, D = [5, 1, 9], 2, 8
+    hidden, ffn, T = H * D, 3 * H * D, 15
+    w = _rand_weights(rng, hidden, ffn)
+    x, dy = rng.standard_normal((T, hidden)), rng.standard_normal((T, hidden))
+    cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    scale = float(np.float32(1 / math.sqrt(D)))
+    ang = rng.uniform(-2, 2, (T, D // 2))
+    tabs = (np.cos(ang), np.sin(ang)) if with_rope else None
+    dx, g = L.encoder_layer_bwd(x, w, cu, H, scale, 1e-6, dy, tabs)
+    # the same block from torch ops with autograd
+    t = lambda a: torch.tensor(np.asarray(a, dtype=np.float64), requires_grad=True)
+    names = {"ln1_gamma": "g1", "ln1_beta": "b1", "w_qkv": "wqkv", "b_qkv": "bqkv", "w_o": "wo", "b_o": "bo", "ln2_gamma": "g2",
+             "ln2_beta": "b2", "w_fc1": "w1", "b_fc1": "bb1", "w_fc2": "w2", "b_fc2": "bb2"}
+    P = {k_: t(getattr(w, v_)) for k_, v_ in names.items()}
+    X = t(x)
+    a = F.layer_norm(X, (hidden,), P["ln1_gamma"], P["ln1_beta"], 1e-6)
+    qkv = F.linear(a, P["w_qkv"], P["b_qkv"])
+    q, k, v = (qkv[:, i * hidden:(i + 1) * hidden].reshape(T, H, D) for i in range(3))
+    if with_rope:
+        c, s_ = torch.from_numpy(tabs[0])[:, None, :], torch.from_numpy(tabs[1])[:, None, :]
+        rot = lambda z: torch.cat([z[..., :D // 2] * c - z[..., D // 2:] * s_, z[..., D // 2:] * c + z[..., :D // 2] * s_], dim=-1)
+        q, k = rot(q), rot(k)
+    seg = torch.repeat_interleave(torch.arange(len(counts)), torch.tensor(counts))
+    sc = (q.permute(1, 0, 2) @ k.permute(1, 2, 0)) * scale
+    sc = sc.masked_fill(~(seg[:, None] == seg[None, :]), float("-inf"))
+    o = (torch.softmax(sc, dim=-1) @ v.permute(1, 0, 2)).permute(1, 0, 2).reshape(T, hidden)
+    x1 = X + F.linear(o, P["w_o"], P["b_o"])
+    m = F.layer_norm(x1, (hidden,), P["ln2_gamma"], P["ln2_beta"], 1e-6)
+    y = x1 + F.linear(F.gelu(F.linear(m, P["w_fc1"], P["b_fc1"])), P["w_fc2"], P["b_fc2"])
+    (y * torch.from_numpy(dy)).sum().backward()
+    np.testing.assert_allclose(dx, X.grad.numpy(), atol=1e-10)
+    for k_ in names:
+        np.testing.assert_allclose(g[k_], P[k_].grad.numpy(), atol=1e-10, err_msg=k_)
+
+
+def test_layer_bwd_finite_difference_on_the_input():
+    rng = np.random.default_rng(11)
+    H, D = 2, 8
+    hidden, ffn, T = H * D, 24, 6
+    w = _rand_weights(rng, hidden, ffn)
+    x, dy = rng.standard_normal((T, hidden)), rng.standard_normal((T, hidden))
+    cu = np.array([0, 2, 6], dtype=np.int32)
+    dx, _ = L.encoder_layer_bwd(x, w, cu, H, 0.25, 1e-6, dy)
+    loss = lambda z: float((L.encoder_layer_fwd(z, w, cu, H, 0.25, 1e-6)[0] * dy).sum())
+    h = 1e-6
+    for (i, j) in [(0, 0), (3, 5), (5, 15)]:
+        e = np.zeros_like(x); e[i, j] = h
+        assert abs((loss(x + e) - loss(x - e)) / (2 * h) - dx[i, j]) < 1e-6
