@@ -394,7 +394,8 @@ def ours_arm(args):
 
 
 # ----------------------------------------------------------------------------- encoder-layer line (--workload *_layer)
-LAYER_WORKLOADS = {"vit_l_layer": "vit_l", "qwen2vl_layer": "qwen2vl_frozen"}
+LAYER_WORKLOADS = {"vit_l_layer": "vit_l", "qwen2vl_layer": "qwen2vl_frozen", "vit_l_layer_trained": "vit_l",
+                   "qwen2vl_layer_trained": "qwen2vl"}
 
 
 def layer_flops(w, ffn):
@@ -437,14 +438,23 @@ def layer_arm(args):
     weights = B.LayerWeights.from_tensors(**params)
     x = rnd((T, hidden), 1.0)
     y = torch.empty_like(x)
-    plan = B.seg_plan(w.patch_counts, B.FROZEN).to_device(dev)
+    trained = _WORKLOAD_NAME.endswith("_trained")
+    plan = B.seg_plan(w.patch_counts, B.TRAINED if trained else B.FROZEN).to_device(dev)
     ws = torch.empty(B.encoder_layer_workspace_bytes(T, hidden, ffn), dtype=torch.uint8, device=dev)
     status = torch.zeros(4, dtype=torch.int32, device=dev)
+    lse = torch.empty((Hh, T), dtype=torch.float32, device=dev) if trained else None
+    if trained:
+        dy, dx = rnd((T, hidden), 1.0), torch.empty_like(x)
+        grads_t = {k_: torch.zeros(v_.shape, dtype=torch.float32, device=dev) for k_, v_ in params.items()}
+        grads = B.LayerGrads.from_tensors(**grads_t)
+        ws_b = torch.empty(B.encoder_layer_bwd_workspace_bytes(T, hidden, Hh, ffn), dtype=torch.uint8, device=dev)
     rope = None
     if base.startswith("qwen2vl"):   # the Qwen2-VL-like configuration carries a 2-D rotary encoding of q and k
         rope = tuple(torch.from_numpy(t).to(dev) for t in W.rope2d_tables(w.patch_counts, Dh))
-    step = lambda xin=x, yout=y, st=None: B.encoder_layer_fwd(xin, yout, weights, Hh, ffn, plan, w.softmax_scale, 1e-6, ws, None,
-                                                             status, st, rope)
+    def step(xin=x, yout=y, st=None):
+        B.encoder_layer_fwd(xin, yout, weights, Hh, ffn, plan, w.softmax_scale, 1e-6, ws, lse, status, st, rope)
+        if trained:
+            B.encoder_layer_bwd(dy, xin, dx, weights, grads, Hh, ffn, plan, w.softmax_scale, 1e-6, lse, ws, ws_b, status, st, rope)
     K, Wm = args.steps, max(args.warmup, 3)
     for _ in range(Wm):
         step()
@@ -477,13 +487,17 @@ def layer_arm(args):
         ("layernorm", lambda: B.layernorm_fwd(x, params["ln1_gamma"], params["ln1_beta"], norm, 1e-6)),
         ("linear_qkv", lambda: B.linear_fwd(norm, params["w_qkv"], qkv, params["b_qkv"], None, False, status)),
         ("rope", (lambda: B.rope_apply(qkv, rope[0], rope[1], Hh, Dh)) if rope is not None else None),
-        ("attn_fwd", lambda: B.varlen_attn_fwd(q3[:, 0], q3[:, 1], q3[:, 2], attn.view(T, Hh, Dh), None, plan, w.softmax_scale, status)),
+        ("attn_fwd", lambda: B.varlen_attn_fwd(q3[:, 0], q3[:, 1], q3[:, 2], attn.view(T, Hh, Dh), lse, plan, w.softmax_scale, status)),
         ("linear_out", lambda: B.linear_fwd(attn, params["w_o"], x1, params["b_o"], x, False, status)),
         ("linear_fc1", lambda: B.linear_fwd(norm, params["w_fc1"], fc1, params["b_fc1"], None, True, status)),
         ("linear_fc2", lambda: B.linear_fwd(fc1, params["w_fc2"], y, params["b_fc2"], x1, False, status)),
     ]
+    if trained:
+        stages.append(("layer_bwd (all of mpipe_encoder_layer_bwd)", lambda: B.encoder_layer_bwd(
+            dy, x, dx, weights, grads, Hh, ffn, plan, w.softmax_scale, 1e-6, lse, ws, ws_b, status, None, rope)))
     Kk = min(K, 20)
     kern_ms = {}
+    step()   # leaves a consistent forward workspace for the backward stage
     for name, fn in stages:
         if fn is None:
             continue
@@ -503,33 +517,48 @@ def layer_arm(args):
     hx = torch.empty(tuple(x.shape), dtype=torch.bfloat16).pin_memory()
     hx.copy_(x)
     hy = torch.empty(tuple(y.shape), dtype=torch.bfloat16).pin_memory()
+    hdy = torch.empty(tuple(y.shape), dtype=torch.bfloat16).pin_memory() if trained else None
+    hdx = torch.empty(tuple(y.shape), dtype=torch.bfloat16).pin_memory() if trained else None
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     f0.record()
     for _ in range(Ke):
         x.copy_(hx, non_blocking=True)
+        if trained:
+            dy.copy_(hdy, non_blocking=True)
         step()
         hy.copy_(y, non_blocking=True)
+        if trained:
+            hdx.copy_(dx, non_blocking=True)
     f1.record()
     torch.cuda.synchronize()
     ms_e2e = f0.elapsed_time(f1) / Ke
 
     gemm_flops, flops_step = layer_flops(w, ffn)
+    n_launch = 8 if rope is not None else 7
+    if trained:   # algorithmic backward work: input and weight gradient of every projection (2x the forward's) + attention
+        flops_step = 3.0 * gemm_flops + w.flops(True, True)    # backward (10 H D sum n^2); the recomputed fc1 is not counted
+        n_launch += 23 if rope is not None else 22
     (ms_step_mx, ms_e2e_mx), (flops_all, launches) = D.reduce_max_sum(
-        [ms_step, ms_e2e], [flops_step, float((8 if rope is not None else 7) * K)], device=dev)
+        [ms_step, ms_e2e], [flops_step, float(n_launch * K)], device=dev)
     if rank == 0:
         value = flops_all / (ms_step_mx * 1e-3) / 1e12
         lin_ms = sum(v for k_, v in kern_ms.items() if k_.startswith("linear"))
         lin_tf = gemm_flops / (lin_ms * 1e-3) / 1e12
         peak_tf = peaks["bf16_tflops_sustained"]
         line = {
-            "metric": "packed encoder layer forward (norms, QKV/out/MLP projections, varlen attention) TFLOP/s (1 B200)",
+            "metric": "packed encoder layer " + ("forward + backward" if trained else "forward") +
+                      " (norms, QKV/out/MLP projections, varlen attention) TFLOP/s (1 B200)",
             "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": ms_step_mx,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": _WORKLOAD_NAME + ": one pre-norm encoder layer over the packed microbatch of " +
-                       WORKLOAD_TEXT[base].split(":")[0] + f", hidden {hidden}, ffn {ffn}, frozen (forward only); one microbatch per GPU",
+                       WORKLOAD_TEXT[base].split(":")[0] + f", hidden {hidden}, ffn {ffn}, " + ("trained (forward + backward)" if trained else "frozen (forward only)") +
+                       "; one microbatch per GPU",
                        "tokens_rank0": T, "sum_n2_rank0": w.sum_n2, "heads": Hh, "head_dim": Dh,
-                       "l2": "inputs_exceed_l2", "step": "mpipe_encoder_layer_fwd: LN, QKV" + (", 2-D rope" if rope is not None else "") + ", attention, out-proj + residual, LN, fc1 + GELU, fc2 + residual"},
+                       "l2": "inputs_exceed_l2", "step": "mpipe_encoder_layer_fwd: LN, QKV" + (", 2-D rope" if rope is not None else "") +
+                               ", attention, out-proj + residual, LN, fc1 + GELU, fc2 + residual" +
+                               ("; mpipe_encoder_layer_bwd: input and weight gradients of the four projections, bias and norm "
+                                "gradients, attention backward, two recomputed norms and one recomputed projection" if trained else "")},
             "breakdown": {"kernel_ms": kern_ms, "linear_tflops": lin_tf,
                           "attn_fwd_tflops": w.flops(True, False) / (kern_ms["attn_fwd"] * 1e-3) / 1e12,
                           "layernorm_gbs": 4.0 * T * hidden / (kern_ms["layernorm"] * 1e-3) / 1e9,
@@ -538,11 +567,12 @@ def layer_arm(args):
             "roofline": {"kernel": "linear_fwd_kernel (4 launches per step)", "bound": "tensor", "achieved": lin_tf, "peak": peak_tf,
                          "unit": "TFLOP/s", "frac": lin_tf / peak_tf, "peak_kind": f"{peak_kind}, sustained bf16 GEMM", "traffic": None},
             "e2e": {"value": flops_all / (ms_e2e_mx * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e2e_mx, "steps": Ke,
-                    "h2d_bytes_per_step": int(hx.numel() * 2), "d2h_bytes_per_step": int(hy.numel() * 2)},
+                    "h2d_bytes_per_step": int(hx.numel() * 2) * (2 if trained else 1),
+                    "d2h_bytes_per_step": int(hy.numel() * 2) * (2 if trained else 1)},
             "gpu_launches": int(launches), "clocks": clocks,
         }
         if world == 1 and not args.profile_mode:
-            line["cpu_baseline"] = layer_cpu_baseline(w, hidden, ffn)
+            line["cpu_baseline"] = layer_cpu_baseline(w, hidden, ffn, trained)
         if args.profile_mode:
             line["profile_mode"] = True
         print(json.dumps(line))
@@ -550,7 +580,7 @@ def layer_arm(args):
     return 0
 
 
-def layer_cpu_baseline(w, hidden, ffn):
+def layer_cpu_baseline(w, hidden, ffn, trained=False):
     """The layer oracle on the first segments of the workload (a few thousand tokens), one pass on the host cores."""
     import oracle
     from oracle import layer as OL
@@ -567,9 +597,13 @@ def layer_cpu_baseline(w, hidden, ffn):
     cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
     oracle.build()
     t0 = time.perf_counter()
-    OL.encoder_layer_fwd(x, ow, cu, w.n_heads, w.softmax_scale, 1e-6)
+    if trained:   # the oracle's backward runs its own forward first
+        OL.encoder_layer_bwd(x, ow, cu, w.n_heads, w.softmax_scale, 1e-6, W.normal_bf16(w.seed, 1, (tok, hidden)))
+    else:
+        OL.encoder_layer_fwd(x, ow, cu, w.n_heads, w.softmax_scale, 1e-6)
     dt = time.perf_counter() - t0
-    flops = 2.0 * tok * hidden * (4 * hidden + 2 * ffn) + 4.0 * hidden * float(sum(n * n for n in counts))
+    sq = float(sum(n * n for n in counts))
+    flops = 2.0 * tok * hidden * (4 * hidden + 2 * ffn) * (3 if trained else 1) + (14.0 if trained else 4.0) * hidden * sq
     return {"value": flops / dt / 1e12, "unit": UNIT, "cores": oracle.n_threads(), "kind": "oracle", "seconds": dt,
             "sample": f"first {m} of {len(w.patch_counts)} segments ({tok} tokens, {flops:.3g} algorithmic FLOPs), one pass"}
 
