@@ -121,40 +121,49 @@ __global__ void __launch_bounds__(256) rope_kernel(__nv_bfloat16* __restrict__ q
 }
 
 // LayerNorm backward.  With xhat = (x - mean) rstd and g = dy gamma:  dx = rstd (g - mean(g) - xhat mean(g xhat)) + dres,
-// dgamma += sum_t dy xhat, dbeta += sum_t dy (fp32 atomics, one per column and block).  One warp per row as in the forward;
-// a block walks rows blockIdx.x * 8 + warp, + gridDim.x * 8, ... and keeps its column sums in registers until the end.
+// dgamma += sum_t dy xhat, dbeta += sum_t dy.  One warp per row as in the forward; a block of four warps walks rows
+// blockIdx.x * 4 + warp, + gridDim.x * 4, ...  Each warp keeps its own column sums in shared memory (plain
+// read-modify-write: a lane owns its columns, a warp handles one row at a time), so registers hold one row only and
+// several blocks fit an SM; at the end the four copies are added and each column costs one global atomic per block
+// (same-address atomics serialise in L2, so the grid is kept to a few blocks per SM).
 template <int kChunks>
-__global__ void __launch_bounds__(256) layernorm_bwd_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ dy,
+__global__ void __launch_bounds__(128) layernorm_bwd_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ dy,
                                                             const __nv_bfloat16* __restrict__ gamma, const __nv_bfloat16* __restrict__ dres,
                                                             __nv_bfloat16* __restrict__ dx, float* __restrict__ dgamma,
                                                             float* __restrict__ dbeta, int32_t T, int32_t hidden, int64_t ldx,
                                                             int64_t lddy, int64_t ldr, int64_t lddx, float eps) {
-    __shared__ float red[2][kChunks * 256];
+    extern __shared__ float red[];   // [4 warps][2][kChunks * 256]
+    constexpr int kCols = kChunks * 256;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_chunks = hidden >> 3;
-    float sg[kChunks][8], sb[kChunks][8];
-#pragma unroll
-    for (int i = 0; i < kChunks; ++i)
-#pragma unroll
-        for (int j = 0; j < 8; ++j) sg[i][j] = sb[i][j] = 0.f;
+    float* my_g = red + warp * 2 * kCols;
+    float* my_b = my_g + kCols;
+    for (int i = threadIdx.x; i < 4 * 2 * kCols; i += 128) red[i] = 0.f;
+    __syncthreads();
     const uint4* g4 = reinterpret_cast<const uint4*>(gamma);
-    for (int row = blockIdx.x * 8 + warp; row < T; row += gridDim.x * 8) {
+    for (int row = blockIdx.x * 4 + warp; row < T; row += gridDim.x * 4) {
         const uint4* xr = reinterpret_cast<const uint4*>(x + int64_t(row) * ldx);
         const uint4* dr = reinterpret_cast<const uint4*>(dy + int64_t(row) * lddy);
-        float xv[kChunks][8], gv[kChunks][8];
+        const uint4* rr = dres != nullptr ? reinterpret_cast<const uint4*>(dres + int64_t(row) * ldr) : nullptr;
+        uint4 xq[kChunks], dq[kChunks], rq[kChunks];
+#pragma unroll
+        for (int i = 0; i < kChunks; ++i) {   // every load of the row is issued before the first use
+            const int c = lane + 32 * i;
+            const bool in = c < n_chunks;
+            xq[i] = in ? xr[c] : make_uint4(0u, 0u, 0u, 0u);
+            dq[i] = in ? dr[c] : make_uint4(0u, 0u, 0u, 0u);
+            rq[i] = (in && rr != nullptr) ? rr[c] : make_uint4(0u, 0u, 0u, 0u);
+        }
+        float xv[kChunks][8];
         float sum = 0.f;
 #pragma unroll
         for (int i = 0; i < kChunks; ++i) {
-            const int c = lane + 32 * i;
-            if (c < n_chunks) {
-                const uint4 q = xr[c];
-                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+            const uint32_t w[4] = {xq[i].x, xq[i].y, xq[i].z, xq[i].w};
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    xv[i][2 * j] = __uint_as_float(w[j] << 16);
-                    xv[i][2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
-                    sum += xv[i][2 * j] + xv[i][2 * j + 1];
-                }
+            for (int j = 0; j < 4; ++j) {
+                xv[i][2 * j] = __uint_as_float(w[j] << 16);
+                xv[i][2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+                sum += xv[i][2 * j] + xv[i][2 * j + 1];   // chunks past the row hold zeros
             }
         }
 #pragma unroll
@@ -172,13 +181,19 @@ __global__ void __launch_bounds__(256) layernorm_bwd_kernel(const __nv_bfloat16*
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
         const float rstd = rsqrtf(sq / float(hidden) + eps);
+        float gv[kChunks][8];
         float s1 = 0.f, s2 = 0.f;   // sum g, sum g xhat
 #pragma unroll
         for (int i = 0; i < kChunks; ++i) {
             const int c = lane + 32 * i;
             if (c < n_chunks) {
-                const uint4 q = dr[c], gq = __ldg(g4 + c);
-                const uint32_t w[4] = {q.x, q.y, q.z, q.w}, gw[4] = {gq.x, gq.y, gq.z, gq.w};
+                const uint4 gq = __ldg(g4 + c);
+                const uint32_t w[4] = {dq[i].x, dq[i].y, dq[i].z, dq[i].w}, gw[4] = {gq.x, gq.y, gq.z, gq.w};
+                float4* pg = reinterpret_cast<float4*>(my_g + c * 8);
+                float4* pb = reinterpret_cast<float4*>(my_b + c * 8);
+                float4 ag[2] = {pg[0], pg[1]}, ab[2] = {pb[0], pb[1]};
+                float* fg = reinterpret_cast<float*>(ag);
+                float* fb = reinterpret_cast<float*>(ab);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const float d = (j & 1) ? __uint_as_float(w[j >> 1] & 0xffff0000u) : __uint_as_float(w[j >> 1] << 16);
@@ -188,9 +203,11 @@ __global__ void __launch_bounds__(256) layernorm_bwd_kernel(const __nv_bfloat16*
                     gv[i][j] = d * gm;
                     s1 += gv[i][j];
                     s2 = fmaf(gv[i][j], xh, s2);
-                    sg[i][j] = fmaf(d, xh, sg[i][j]);
-                    sb[i][j] += d;
+                    fg[j] = fmaf(d, xh, fg[j]);
+                    fb[j] += d;
                 }
+                pg[0] = ag[0]; pg[1] = ag[1];
+                pb[0] = ab[0]; pb[1] = ab[1];
             }
         }
 #pragma unroll
@@ -200,16 +217,11 @@ __global__ void __launch_bounds__(256) layernorm_bwd_kernel(const __nv_bfloat16*
         }
         const float m1 = s1 / float(hidden), m2 = s2 / float(hidden);
         uint4* outr = reinterpret_cast<uint4*>(dx + int64_t(row) * lddx);
-        const uint4* rr = dres != nullptr ? reinterpret_cast<const uint4*>(dres + int64_t(row) * ldr) : nullptr;
 #pragma unroll
         for (int i = 0; i < kChunks; ++i) {
             const int c = lane + 32 * i;
             if (c < n_chunks) {
-                uint32_t rw[4] = {0u, 0u, 0u, 0u};
-                if (rr != nullptr) {
-                    const uint4 q = rr[c];
-                    rw[0] = q.x; rw[1] = q.y; rw[2] = q.z; rw[3] = q.w;
-                }
+                const uint32_t rw[4] = {rq[i].x, rq[i].y, rq[i].z, rq[i].w};
                 uint32_t o[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -222,44 +234,59 @@ __global__ void __launch_bounds__(256) layernorm_bwd_kernel(const __nv_bfloat16*
             }
         }
     }
-    // column sums: warps -> shared memory -> one atomic per column and block
-    for (int pass = 0; pass < 8; ++pass) {
-        if (warp == pass) {
+    __syncthreads();
+    for (int col = threadIdx.x; col < hidden; col += 128) {
+        float sg = 0.f, sb = 0.f;
 #pragma unroll
-            for (int i = 0; i < kChunks; ++i)
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int col = (lane + 32 * i) * 8 + j;
-                    if (pass == 0) { red[0][col] = sg[i][j]; red[1][col] = sb[i][j]; }
-                    else { red[0][col] += sg[i][j]; red[1][col] += sb[i][j]; }
-                }
+        for (int w = 0; w < 4; ++w) {
+            sg += red[w * 2 * kCols + col];
+            sb += red[w * 2 * kCols + kCols + col];
         }
-        __syncthreads();
-    }
-    for (int col = threadIdx.x; col < hidden; col += 256) {
-        atomicAdd(dgamma + col, red[0][col]);
-        atomicAdd(dbeta + col, red[1][col]);
+        atomicAdd(dgamma + col, sg);
+        atomicAdd(dbeta + col, sb);
     }
 }
 
-// out[n] += sum_t a[t, n] (fp32 atomics): the bias gradient of a projection.  blockIdx.x picks 256 chunks of 8 columns,
-// blockIdx.y a slice of the rows.
+// out[n] += sum_t a[t, n] (fp32): the bias gradient of a projection.  A block is 32 chunk lanes (8 columns each) x 8 row
+// lanes over one group of 256 columns and one slice of the rows, four rows in flight per thread; the row lanes are added
+// in shared memory, so a column costs one global atomic per block (same-address atomics serialise in L2).
 __global__ void __launch_bounds__(256) colsum_kernel(const __nv_bfloat16* __restrict__ a, float* __restrict__ out, int32_t T, int32_t N,
-                                                     int64_t lda) {
-    const int chunk = blockIdx.x * 256 + threadIdx.x;
-    if (chunk * 8 >= N) return;
+                                                     int64_t lda, int32_t n_groups, int32_t n_slices) {
+    __shared__ float red[8][256];
+    const int cl = threadIdx.x & 31, rl = threadIdx.x >> 5;
+    const int group = blockIdx.x % n_groups, slice = blockIdx.x / n_groups;
+    const int chunk = group * 32 + cl;
+    const bool in = chunk * 8 < N;
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    for (int row = blockIdx.y; row < T; row += gridDim.y) {
-        const uint4 q = *reinterpret_cast<const uint4*>(a + int64_t(row) * lda + chunk * 8);
-        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+    const __nv_bfloat16* base = a + chunk * 8;
+    const int stride = n_slices * 8;
+    for (int row = slice * 8 + rl; row < T && in; row += 4 * stride) {
+        uint4 q[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            acc[2 * j] += __uint_as_float(w[j] << 16);
-            acc[2 * j + 1] += __uint_as_float(w[j] & 0xffff0000u);
+        for (int u = 0; u < 4; ++u) {
+            const int r = row + u * stride;
+            q[u] = r < T ? *reinterpret_cast<const uint4*>(base + int64_t(r) * lda) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                acc[2 * j] += __uint_as_float(w[j] << 16);
+                acc[2 * j + 1] += __uint_as_float(w[j] & 0xffff0000u);
+            }
         }
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) atomicAdd(out + chunk * 8 + j, acc[j]);
+    for (int j = 0; j < 8; ++j) red[rl][cl * 8 + j] = acc[j];
+    __syncthreads();
+    const int col = group * 256 + threadIdx.x;
+    if (col < N) {
+        float sacc = 0.f;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) sacc += red[r][threadIdx.x];
+        atomicAdd(out + col, sacc);
+    }
 }
 
 static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
@@ -342,12 +369,16 @@ int32_t mpipe_layernorm_bwd(const void* x, const void* dy, const void* gamma, co
         return MPIPE_ERR_UNSUPPORTED;
     if (!aligned16(x) || !aligned16(dy) || !aligned16(gamma) || !aligned16(dres) || !aligned16(dx)) return MPIPE_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int grid = std::min(cdiv(n_tokens, 8), sm_count() * 4);
+    const int grid = std::min(cdiv(n_tokens, 4), sm_count() * 6);
     const int chunks = cdiv(hidden, 256);
 #define MPIPE_LNB_LAUNCH(C)                                                                                                    \
-    layernorm_bwd_kernel<C><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy),   \
-                                                  static_cast<const __nv_bfloat16*>(gamma), static_cast<const __nv_bfloat16*>(dres), \
-                                                  static_cast<__nv_bfloat16*>(dx), dgamma, dbeta, n_tokens, hidden, ldx, lddy, ldr, lddx, eps)
+    do {                                                                                                                       \
+        cudaFuncSetAttribute(layernorm_bwd_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * 2 * (C) * 256 * 4);      \
+        layernorm_bwd_kernel<C><<<grid, 128, 4 * 2 * (C) * 256 * 4, st>>>(                                                      \
+            static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(dy), static_cast<const __nv_bfloat16*>(gamma), \
+            static_cast<const __nv_bfloat16*>(dres), static_cast<__nv_bfloat16*>(dx), dgamma, dbeta, n_tokens, hidden, ldx, lddy, \
+            ldr, lddx, eps);                                                                                                   \
+    } while (0)
     if (chunks <= 1) MPIPE_LNB_LAUNCH(1);
     else if (chunks <= 2) MPIPE_LNB_LAUNCH(2);
     else if (chunks <= 4) MPIPE_LNB_LAUNCH(4);
@@ -363,9 +394,10 @@ int32_t mpipe_colsum_accumulate(const void* a, float* out, int32_t n_tokens, int
     if (n_tokens == 0) return MPIPE_OK;
     if (a == nullptr || out == nullptr || lda < n_cols) return MPIPE_ERR_INVALID_ARG;
     if ((n_cols % 8) != 0 || (lda % 8) != 0 || !aligned16(a)) return MPIPE_ERR_UNSUPPORTED;
-    const int gx = cdiv(n_cols / 8, 256);
-    const int gy = std::max(1, std::min(n_tokens, (sm_count() * 8) / gx));
-    colsum_kernel<<<dim3(gx, gy), 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const __nv_bfloat16*>(a), out, n_tokens, n_cols, lda);
+    const int n_groups = cdiv(n_cols, 256);
+    const int n_slices = std::max(1, std::min(cdiv(n_tokens, 8), (sm_count() * 6) / n_groups));
+    colsum_kernel<<<n_groups * n_slices, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const __nv_bfloat16*>(a), out, n_tokens,
+                                                                                      n_cols, lda, n_groups, n_slices);
     return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
 }
 
