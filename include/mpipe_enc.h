@@ -295,7 +295,8 @@ int32_t mpipe_layernorm_bwd(const void* x, const void* dy, const void* gamma, co
                             int64_t lddx, float eps, void* stream);
 int32_t mpipe_colsum_accumulate(const void* a, float* out, int32_t n_tokens, int32_t n_cols, int64_t lda, void* stream);
 /*
- * Bwd(enc, r, m) of the same layer -- exists only when the encoder is trainable (Lemma 1).  Given dy = dL/dy it writes
+ * Bwd(enc, r, m) of the same layer -- exists only when the encoder is trainable (Lemma 1): with mode FROZEN the call
+ * returns MPIPE_OK at once and touches nothing.  TRAINED: given dy = dL/dy it writes
  * dx = dL/dx (bf16 [n_tokens, hidden]) and ADDS the parameter gradients, in fp32, to the twelve buffers of `grads`
  * (same shapes as the weights; the caller zeroes them at the start of a step, every microbatch accumulates).
  * fwd_workspace is the workspace of the matching mpipe_encoder_layer_fwd call (TRAINED mode, same x, weights, plan and
@@ -314,9 +315,9 @@ int32_t mpipe_encoder_layer_bwd(const void* dy, const void* x, void* dx, const m
                                 const mpipe_layer_grads_t* grads, int32_t n_tokens, int32_t hidden, int32_t n_heads,
                                 int32_t ffn, const int32_t* cu_seqlens_dev, int32_t n_seg, int32_t max_seqlen,
                                 const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items, float softmax_scale,
-                                float ln_eps, const float* rope_cos, const float* rope_sin, const float* lse,
-                                void* fwd_workspace, void* workspace, size_t workspace_bytes, int32_t* status_buf,
-                                void* stream);
+                                float ln_eps, const float* rope_cos, const float* rope_sin, int32_t mode,
+                                const float* lse, void* fwd_workspace, void* workspace, size_t workspace_bytes,
+                                int32_t* status_buf, void* stream);
 size_t mpipe_encoder_layer_workspace_bytes(int32_t n_tokens, int32_t hidden, int32_t ffn);
 int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weights_t* w, int32_t n_tokens,
                                 int32_t hidden, int32_t n_heads, int32_t ffn, const int32_t* cu_seqlens_dev,

@@ -34,7 +34,7 @@ _i32, _i64, _vp, _f32, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ct
 _SIGNATURES = {
     "mpipe_encoder_layer_bwd_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32]),
     "mpipe_encoder_layer_bwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _i32, _i32, _vp, _i32, _f32, _f32,
-                                       _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
+                                       _vp, _vp, _i32, _vp, _vp, _vp, _sz, _vp, _vp]),
     "mpipe_rope_apply_bwd": (_i32, [_vp, _i64, _i64, _vp, _vp, _i32, _i32, _i32, _vp]),
     "mpipe_layernorm_bwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i64, _i64, _i64, _i64, _f32, _vp]),
     "mpipe_colsum_accumulate": (_i32, [_vp, _vp, _i32, _i32, _i64, _vp]),
@@ -366,12 +366,13 @@ def encoder_layer_bwd(dy, x, dx, weights: LayerWeights, grads: LayerGrads, n_hea
                       rope=None) -> None:
     """mpipe_encoder_layer_bwd: dy, x, dx bf16 [T, hidden] contiguous; fwd_workspace untouched since the matching forward."""
     T, hidden = x.shape
-    assert plan.mode == TRAINED and dy.is_contiguous() and x.is_contiguous() and dx.is_contiguous()
+    assert dy.is_contiguous() and x.is_contiguous() and dx.is_contiguous()
     st = load().mpipe_encoder_layer_bwd(
         _ptr(dy), _ptr(x), _ptr(dx), ctypes.addressof(weights), ctypes.addressof(grads), T, hidden, n_heads, ffn,
         _ptr(plan.cu_seqlens_dev), plan.n_seg, plan.max_seqlen, _ptr(plan.bwd_items_dev), int(plan.bwd_items.size), softmax_scale,
-        ln_eps, _ptr(None if rope is None else rope[0]), _ptr(None if rope is None else rope[1]), _ptr(lse), _ptr(fwd_workspace),
-        _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status_buf), _stream(stream))
+        ln_eps, _ptr(None if rope is None else rope[0]), _ptr(None if rope is None else rope[1]), plan.mode, _ptr(lse),
+        _ptr(fwd_workspace), _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+        _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_encoder_layer_bwd")
 
 

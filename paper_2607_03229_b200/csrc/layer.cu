@@ -464,9 +464,12 @@ size_t mpipe_encoder_layer_bwd_workspace_bytes(int32_t n_tokens, int32_t hidden,
 int32_t mpipe_encoder_layer_bwd(const void* dy, const void* x, void* dx, const mpipe_layer_weights_t* w, const mpipe_layer_grads_t* g,
                                 int32_t n_tokens, int32_t hidden, int32_t n_heads, int32_t ffn, const int32_t* cu_seqlens_dev,
                                 int32_t n_seg, int32_t max_seqlen, const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items,
-                                float softmax_scale, float ln_eps, const float* rope_cos, const float* rope_sin, const float* lse,
-                                void* fwd_workspace, void* workspace, size_t workspace_bytes, int32_t* status_buf, void* stream) {
+                                float softmax_scale, float ln_eps, const float* rope_cos, const float* rope_sin, int32_t mode,
+                                const float* lse, void* fwd_workspace, void* workspace, size_t workspace_bytes, int32_t* status_buf,
+                                void* stream) {
     using namespace mpipe;
+    if (mode != MPIPE_ENC_FROZEN && mode != MPIPE_ENC_TRAINED) return MPIPE_ERR_INVALID_ARG;
+    if (mode == MPIPE_ENC_FROZEN) return MPIPE_OK;   // Lemma 1: a frozen encoder has no backward events
     if (n_tokens < 0 || hidden <= 0 || n_heads <= 0 || ffn <= 0 || w == nullptr || g == nullptr) return MPIPE_ERR_INVALID_ARG;
     if (n_tokens == 0) return MPIPE_OK;
     if (dy == nullptr || x == nullptr || dx == nullptr || lse == nullptr || fwd_workspace == nullptr || (hidden % n_heads) != 0)

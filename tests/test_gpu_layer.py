@@ -321,3 +321,17 @@ def test_layer_bwd_matches_oracle(counts, H, D, ffn, rope):
     for name, ref in g_ref.items():
         got = grads_t[name].cpu().double().numpy() / 2.0
         assert rel_l2(got, ref.reshape(got.shape)) <= GRAD_REL_L2, (name, rel_l2(got, ref.reshape(got.shape)))
+
+
+def test_layer_bwd_frozen_is_a_no_op():
+    T, hidden, ffn, H = 64, 256, 512, 4
+    pb = W.layer_params_bf16(5, hidden, ffn)
+    weights = B.LayerWeights.from_tensors(**{k: to_dev(v) for k, v in pb.items()})
+    grads_t = {k: torch.full(v.shape, 3.0, dtype=torch.float32, device="cuda") for k, v in pb.items()}
+    grads = B.LayerGrads.from_tensors(**grads_t)
+    x = to_dev(W.normal_bf16(5, 0, (T, hidden)))
+    dx = torch.full_like(x, 7.0)
+    plan = B.seg_plan([T], B.FROZEN).to_device()
+    B.encoder_layer_bwd(x, x, dx, weights, grads, H, ffn, plan, 0.125, 1e-6, None, None, None)   # nothing else is needed
+    torch.cuda.synchronize()
+    assert (dx == 7.0).all() and all((g == 3.0).all() for g in grads_t.values())
