@@ -36,7 +36,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one attn_bwd_kernel<64> launch on this workload, from the
 # ncu capture summarised in profiles/attn_bwd_kernel_vit_l.md.
-BWD_MAIN_DRAM_BYTES_PER_LAUNCH = 1.0320e9
+BWD_MAIN_DRAM_BYTES_PER_LAUNCH = 1.0274e9
 
 
 def load_peaks():
