@@ -335,3 +335,40 @@ def test_layer_bwd_frozen_is_a_no_op():
     B.encoder_layer_bwd(x, x, dx, weights, grads, H, ffn, plan, 0.125, 1e-6, None, None, None)   # nothing else is needed
     torch.cuda.synchronize()
     assert (dx == 7.0).all() and all((g == 3.0).all() for g in grads_t.values())
+
+
+def test_layer_bwd_full_size_sampled_segments():
+    """The bench's ViT-L microbatch through forward + backward; the input gradient of an image's rows depends on that image
+    alone (block-diagonal attention, row-wise everything else), so the oracle recomputes the two shortest images' dx."""
+    w = W.vit_l()
+    H, D = w.n_heads, w.head_dim
+    hidden, ffn, T = H * D, 4 * H * D, w.total_tokens
+    pb = W.layer_params_bf16(33, hidden, ffn)
+    x, dy = W.normal_bf16(33, 0, (T, hidden)), W.normal_bf16(33, 1, (T, hidden))
+    plan = B.seg_plan(w.patch_counts, B.TRAINED).to_device()
+    weights = B.LayerWeights.from_tensors(**{k: to_dev(v) for k, v in pb.items()})
+    grads_t = {k: torch.zeros(v.shape, dtype=torch.float32, device="cuda") for k, v in pb.items()}
+    grads = B.LayerGrads.from_tensors(**grads_t)
+    xd, dyd = to_dev(x), to_dev(dy)
+    y, dx = torch.empty_like(xd), torch.empty_like(xd)
+    lse = torch.empty((H, T), dtype=torch.float32, device="cuda")
+    ws_f = torch.empty(B.encoder_layer_workspace_bytes(T, hidden, ffn), dtype=torch.uint8, device="cuda")
+    ws_b = torch.empty(B.encoder_layer_bwd_workspace_bytes(T, hidden, H, ffn), dtype=torch.uint8, device="cuda")
+    st = status_buf()
+    B.encoder_layer_fwd(xd, y, weights, H, ffn, plan, w.softmax_scale, 1e-6, ws_f, lse, st)
+    B.encoder_layer_bwd(dyd, xd, dx, weights, grads, H, ffn, plan, w.softmax_scale, 1e-6, lse, ws_f, ws_b, st)
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[0] == 0
+    ow = OL.LayerWeights(g1=OL.widen(pb["ln1_gamma"]), b1=OL.widen(pb["ln1_beta"]), wqkv=OL.widen(pb["w_qkv"]),
+                         bqkv=OL.widen(pb["b_qkv"]), wo=OL.widen(pb["w_o"]), bo=OL.widen(pb["b_o"]),
+                         g2=OL.widen(pb["ln2_gamma"]), b2=OL.widen(pb["ln2_beta"]), w1=OL.widen(pb["w_fc1"]),
+                         bb1=OL.widen(pb["b_fc1"]), w2=OL.widen(pb["w_fc2"]), bb2=OL.widen(pb["b_fc2"]))
+    got = to_f64(dx)
+    cu = w.cu_seqlens
+    for seg in np.argsort(w.patch_counts)[:2]:
+        lo, hi = int(cu[seg]), int(cu[seg + 1])
+        ref, _ = OL.encoder_layer_bwd(x[lo:hi], ow, np.array([0, hi - lo], dtype=np.int32), H, w.softmax_scale, 1e-6, dy[lo:hi])
+        assert rel_l2(got[lo:hi], ref) <= GRAD_REL_L2, (seg, rel_l2(got[lo:hi], ref))
+    # the bias gradient of the last projection is the plain column sum of dy: an exact, full-size check of the accumulation
+    ref_b = OL.widen(dy).sum(axis=0)
+    assert np.abs(grads_t["b_fc2"].cpu().double().numpy() - ref_b).max() <= 1e-5 * np.abs(ref_b).max() + 1e-3
