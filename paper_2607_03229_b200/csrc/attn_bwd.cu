@@ -191,6 +191,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         const int g = int(gridDim.x), i = int(blockIdx.x);
         return round * g + ((round & 1) ? g - 1 - i : i);
     };
+    auto item_at = [&](int u) {
+        mpipe_work_item_t z = {0, 0, 0, 0, 0, 0};
+        return (u < n_units) ? p.items[u / p.n_heads] : z;
+    };
     // Every unit runs an even number of 64-query sub-tiles (a 128-query tile is two of them); a padding
     // sub-tile past the segment end contributes nothing because its probabilities are forced to zero.
     auto subtiles_of = [](const mpipe_work_item_t& it) { return 2 * ((it.kv_len + kBT - 1) / kBT); };
@@ -201,8 +205,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         if (lane == 0) {
             uint32_t unit_it = 0, sc = 0;
             bool ok = true;
+            mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
-                const mpipe_work_item_t it = p.items[u / p.n_heads];
+                const mpipe_work_item_t it = it_next;
+                it_next = item_at(unit_of(ur + 1));
                 const int head = u % p.n_heads;
                 const int n2 = subtiles_of(it);
                 const int kb = unit_it % Cfg::kKVBufs;            // K/V buffer of this unit
@@ -291,8 +297,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             };
             uint32_t unit_it = 0, sc = 0;   // sc: global sub-tile counter at the start of the unit (even)
             bool ok = true;
+            mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
-                const mpipe_work_item_t it = p.items[u / p.n_heads];
+                const mpipe_work_item_t it = it_next;
+                it_next = item_at(unit_of(ur + 1));
                 const int n2 = subtiles_of(it);
                 const int kb = unit_it % Cfg::kKVBufs;
                 const uint32_t kvb = sbase + kb * (2 * Cfg::kTile);
@@ -323,8 +331,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     }
                     if (!ok) break;
                 }
-                for (int s = b0; s < n2; s += kStep) {
-                    const int b = s & 1;
+                // One sub-tile of the issue order.  The TMEM stage b is a compile-time constant (the loop below is unrolled
+                // over the two stages), so stage offsets and barrier addresses fold into immediates.
+                auto sub_tile = [&](const int s, auto stage) -> bool {
+                    constexpr int b = decltype(stage)::value;
                     const uint32_t c = sc + s;
                     const uint32_t ph = (c >> 1) & 1;   // phase of the per-stage barriers
                     const bool cross = (s + 2 >= n2) && has_next;   // sub-tile s+2 is the next unit's
@@ -332,13 +342,13 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     const bool first = (s < 2);         // the stage's first sub-tile of the unit
                     MPIPE_TR(0, c * 8 + 0);
                     ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.p_full[b], ph, &abort_flag));
-                    if (!ok) break;
+                    if (!ok) return false;
                     if (first && b == 0) {          // the accumulators are free: the previous unit's epilogue has read them
                         ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag));
-                        if (!ok) break;
+                        if (!ok) return false;
                     } else if (first && kIssuers == 2) {   // ... and stage 0's overwriting dV MMA has been issued
                         ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.acc_v, unit_it & 1, &abort_flag));
-                        if (!ok) break;
+                        if (!ok) return false;
                     }
                     MPIPE_TR(0, c * 8 + 1);
                     tc_fence_after();
@@ -350,22 +360,22 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     if (more) {
                         if (cross && b == 0) {   // the next unit's K/V tiles (loaded while this unit ran)
                             ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.kv_full[kb ^ 1], ((unit_it + 1) / Cfg::kKVBufs) & 1, &abort_flag));
-                            if (!ok) break;
+                            if (!ok) return false;
                         }
                         ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[(c + 2) % NR], ((c + 2) / NR) & 1, &abort_flag));
-                        if (!ok) break;
+                        if (!ok) return false;
                         ok = wait_stat(c + 2);
-                        if (!ok) break;
+                        if (!ok) return false;
                         tc_fence_after();
                         issue_kk(Cfg::kColS + 64 * b, cross ? k_lo_n : k_lo, kt_lo, q_lo_of(c + 2));       // S^T(s+2)
                         if (leader) umma_commit(&bars.s_full[b]);
                     }
                     MPIPE_TR(0, c * 8 + 2);
                     ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.ds_full[b], ph, &abort_flag));
-                    if (!ok) break;
+                    if (!ok) return false;
                     if (first && b == 1 && kIssuers == 2) {
                         ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.acc_k, unit_it & 1, &abort_flag));
-                        if (!ok) break;
+                        if (!ok) return false;
                     }
                     MPIPE_TR(0, c * 8 + 3);
                     tc_fence_after();
@@ -385,11 +395,11 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     if (b == 1) {                                                             // dQ of the 128-query pair
                         if (kIssuers == 2) {   // the other half of dS^T (a single issuer has already waited for it)
                             ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.ds_full[0], ph, &abort_flag));
-                            if (!ok) break;
+                            if (!ok) return false;
                             if (leader) mbar_arrive(&bars.ds0_seen);   // lets stage 0's warpgroup complete the next phase
                         }
                         ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.dq_empty, ((c >> 1) & 1) ^ 1, &abort_flag));
-                        if (!ok) break;
+                        if (!ok) return false;
                         MPIPE_TR(0, c * 8 + 4);
                         tc_fence_after();
                         if (leader) {
@@ -404,6 +414,16 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                         }
                     }
                     MPIPE_TR(0, c * 8 + 5);
+                    return true;
+                };
+                if (kStep == 1) {
+                    for (int s = 0; s < n2 && ok; s += 2) {
+                        ok = sub_tile(s, std::integral_constant<int, 0>{});
+                        if (ok) ok = sub_tile(s + 1, std::integral_constant<int, 1>{});
+                    }
+                } else {
+                    for (int s = b0; s < n2 && ok; s += 2)
+                        ok = (b0 == 0) ? sub_tile(s, std::integral_constant<int, 0>{}) : sub_tile(s, std::integral_constant<int, 1>{});
                 }
                 if (!ok) break;
                 if (leader) umma_commit(&bars.dkv_full);
@@ -417,8 +437,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         setmaxnreg_dec<kRegsService>();
         uint32_t sc = 0;
         bool ok = true;
+        mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
         for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
-            const mpipe_work_item_t it = p.items[u / p.n_heads];
+            const mpipe_work_item_t it = it_next;
+            it_next = item_at(unit_of(ur + 1));
             const int head = u % p.n_heads;
             const int n2 = subtiles_of(it);
             const int q_end = it.kv_start + it.kv_len;
@@ -463,8 +485,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         uint8_t* ds_row = smem + Cfg::kSmemDS + g * (kBT * 128) + r * 128;
         uint32_t sc = 0;   // global sub-tile counter at the start of the unit (always even)
         bool ok = true;
+        mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
         for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
-            const mpipe_work_item_t it = p.items[u / p.n_heads];
+            const mpipe_work_item_t it = it_next;
+            it_next = item_at(unit_of(ur + 1));
             const int n2 = subtiles_of(it);
             const bool key_valid = r < it.row_len;
             const bool ragged_keys = it.row_len < kBT;
@@ -588,8 +612,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
         uint32_t pc = 0, unit_it = 0;   // pair counter
         bool ok = true;
+        mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
         for (int ur = 0, u = unit_of(0); u < n_units; ++ur, u = unit_of(ur), ++unit_it) {
-            const mpipe_work_item_t it = p.items[u / p.n_heads];
+            const mpipe_work_item_t it = it_next;
+            it_next = item_at(unit_of(ur + 1));
             const int head = u % p.n_heads;
             const int npairs = (it.kv_len + kBT - 1) / kBT;
             // No early exit inside this loop: the four warps meet at named barriers, so after a time-out

@@ -124,6 +124,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int g = int(gridDim.x), i = int(blockIdx.x);
         return round * g + ((round & 1) ? g - 1 - i : i);
     };
+    auto item_at = [&](int u) {
+        mpipe_work_item_t z = {0, 0, 0, 0, 0, 0};
+        return (u < n_units) ? p.items[u / p.n_heads] : z;
+    };
 
     if (warp == 0) {
         setmaxnreg_dec<kFwdRegsLight>();
@@ -131,8 +135,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (lane == 0) {
             uint32_t kv_it = 0, unit_it = 0;
             bool ok = true;
+            mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
-                const mpipe_work_item_t it = p.items[u / p.n_heads];
+                const mpipe_work_item_t it = it_next;
+                it_next = item_at(unit_of(ur + 1));
                 const int head = u % p.n_heads;
                 const bool two = it.row_len > kTileM;
                 const int nkv = (it.kv_len + kTileN - 1) / kTileN;
@@ -209,8 +215,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     }
                 }
             };
+            mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
-                const mpipe_work_item_t it = p.items[u / p.n_heads];
+                const mpipe_work_item_t it = it_next;
+                it_next = item_at(unit_of(ur + 1));
                 const bool two = it.row_len > kTileM;
                 const int nkv = (it.kv_len + kTileN - 1) / kTileN;
                 auto cols_of = [&](int j) {
@@ -289,8 +297,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const uint32_t t_o = tmem + lane_base + 256 + w * 128;
         uint32_t cnt = 0, ocnt = 0;
         bool ok = true;
+        mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
         for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
-            const mpipe_work_item_t it = p.items[u / p.n_heads];
+            const mpipe_work_item_t it = it_next;
+            it_next = item_at(unit_of(ur + 1));
             const int head = u % p.n_heads;
             const int rows_here = it.row_len - w * kTileM;  // valid rows of this tile
             if (rows_here <= 0) continue;
