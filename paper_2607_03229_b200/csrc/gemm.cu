@@ -114,9 +114,12 @@ linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     const int nk = (p.K + kGemmBK - 1) / kGemmBK;
     const int n_tiles = p.tiles_m * p.tiles_n * (kBMode == 2 ? p.splits : 1);   // work items
     // work item -> output tile and range of contraction blocks
-    auto tile_of = [&](int t) { return kBMode == 2 ? t / p.splits : t; };
-    auto kb_lo_of = [&](int t) { return kBMode == 2 ? int((long long)(t % p.splits) * nk / p.splits) : 0; };
-    auto kb_hi_of = [&](int t) { return kBMode == 2 ? int((long long)(t % p.splits + 1) * nk / p.splits) : nk; };
+    // (weight gradient: the split index is the slow one, so that the CTAs of a wave work on the same token range and
+    //  share its dY and X rows through L2)
+    const int n_out_tiles = p.tiles_m * p.tiles_n;
+    auto tile_of = [&](int t) { return kBMode == 2 ? t % n_out_tiles : t; };
+    auto kb_lo_of = [&](int t) { return kBMode == 2 ? int((long long)(t / n_out_tiles) * nk / p.splits) : 0; };
+    auto kb_hi_of = [&](int t) { return kBMode == 2 ? int((long long)(t / n_out_tiles + 1) * nk / p.splits) : nk; };
 
     if (warp == 0) {
         if (lane == 0) {
