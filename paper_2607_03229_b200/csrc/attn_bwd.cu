@@ -271,8 +271,11 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             constexpr uint32_t idesc_dq = umma_idesc_bf16(kBT, 64, 1, 1);      // MN-major A and B
             constexpr uint32_t idesc_dq_t = umma_idesc_bf16(kBT, 16, 1, 1);
             constexpr uint32_t kSubTailOff = Cfg::kSubMain >> 4;
-            auto q_lo_of = [&](uint32_t c) { return umma_desc_lo(sbase + Cfg::kSmemQ + (c % NR) * Cfg::kSub, 0); };
-            auto do_lo_of = [&](uint32_t c) { return umma_desc_lo(sbase + Cfg::kSmemDO + (c % NR) * Cfg::kSub, 0); };
+            // descriptor low words of the ring's Q / dO stages: base + stage * (stage bytes / 16); no carry out of the 14
+            // address bits as long as the stage lies in shared memory
+            const uint32_t q_lo0 = umma_desc_lo(sbase + Cfg::kSmemQ, 0), do_lo0 = umma_desc_lo(sbase + Cfg::kSmemDO, 0);
+            auto q_lo_of = [&](uint32_t c) { return q_lo0 + (c % NR) * uint32_t(Cfg::kSub >> 4); };
+            auto do_lo_of = [&](uint32_t c) { return do_lo0 + (c % NR) * uint32_t(Cfg::kSub >> 4); };
             // dst[128 keys x 64 q] = A[128 x D] * B[64 x D]^T, both K-major (main 64 columns + optional 16 tail)
             auto issue_kk = [&](uint32_t dcol, uint32_t a, uint32_t at, uint32_t bq) {
                 if (leader) {
