@@ -538,7 +538,7 @@ def layer_arm(args):
     n_launch = 8 if rope is not None else 7
     if trained:   # algorithmic backward work: input and weight gradient of every projection (2x the forward's) + attention
         flops_step = 3.0 * gemm_flops + w.flops(True, True)    # backward (10 H D sum n^2); the recomputed fc1 is not counted
-        n_launch += 23 if rope is not None else 22
+        n_launch += 23 if rope is not None else 22   # + the activation kernel of a trained forward, - the projection no longer recomputed
     (ms_step_mx, ms_e2e_mx), (flops_all, launches) = D.reduce_max_sum(
         [ms_step, ms_e2e], [flops_step, float(n_launch * K)], device=dev)
     if rank == 0:
@@ -558,7 +558,7 @@ def layer_arm(args):
                        "l2": "inputs_exceed_l2", "step": "mpipe_encoder_layer_fwd: LN, QKV" + (", 2-D rope" if rope is not None else "") +
                                ", attention, out-proj + residual, LN, fc1 + GELU, fc2 + residual" +
                                ("; mpipe_encoder_layer_bwd: input and weight gradients of the four projections, bias and norm "
-                                "gradients, attention backward, two recomputed norms and one recomputed projection" if trained else "")},
+                                "gradients, attention backward, two recomputed norms" if trained else "")},
             "breakdown": {"kernel_ms": kern_ms, "linear_tflops": lin_tf,
                           "attn_fwd_tflops": w.flops(True, False) / (kern_ms["attn_fwd"] * 1e-3) / 1e12,
                           "layernorm_gbs": 4.0 * T * hidden / (kern_ms["layernorm"] * 1e-3) / 1e9,

@@ -244,7 +244,11 @@ int32_t mpipe_validate_positions(const int32_t* positions, int32_t n, int32_t n_
  *        x, y: bf16 [n_tokens, hidden] contiguous, device; y may not alias x.  Weights: device bf16, nn.Linear
  *        layout [out, in], contiguous.  lse: fp32 [n_heads, n_tokens] when TRAINED, ignored when FROZEN.
  *        workspace: device, 256-byte aligned, >= mpipe_encoder_layer_workspace_bytes (MPIPE_ERR_WORKSPACE);
- *        caller-owned, contents undefined afterwards.  Seven launches (eight with rope) on `stream`, no allocation, no sync.
+ *        caller-owned; after a TRAINED call it holds what mpipe_encoder_layer_bwd reads (see there), otherwise its contents are
+ *        undefined afterwards.  The TRAINED forward rounds the MLP pre-activation to bf16 before the activation (it has to
+ *        keep it), the FROZEN one applies the activation to the fp32 accumulator: the two outputs agree to bf16 rounding,
+ *        not bit for bit.  Seven launches (eight with rope; one more when TRAINED: the activation is applied by a kernel of its own so that
+ *        the pre-activation can be kept for the backward) on `stream`, no allocation, no sync.
  *        head_dim = hidden / n_heads must be one the attention kernels support (64, 80).
  * Device-side findings (a bounded wait that ran out) are reported through status_buf as for the attention calls.
  */
@@ -300,9 +304,9 @@ int32_t mpipe_colsum_accumulate(const void* a, float* out, int32_t n_tokens, int
  * dx = dL/dx (bf16 [n_tokens, hidden]) and ADDS the parameter gradients, in fp32, to the twelve buffers of `grads`
  * (same shapes as the weights; the caller zeroes them at the start of a step, every microbatch accumulates).
  * fwd_workspace is the workspace of the matching mpipe_encoder_layer_fwd call (TRAINED mode, same x, weights, plan and
- * rope tables), untouched since: it holds the rotated q | k | v, the attention output, x1 and GELU(u); its LN slot is
- * overwritten here.  lse is that call's LSE.  The two LayerNorm outputs and the MLP pre-activation u are recomputed
- * (one extra projection) instead of being stored by the forward.  workspace: device, 256-byte aligned,
+ * rope tables), untouched since: it holds the rotated q | k | v, the attention output, x1, GELU(u) and (TRAINED forward
+ * only) the MLP pre-activation u; its LN slot is overwritten here.  lse is that call's LSE.  The two LayerNorm outputs
+ * are recomputed instead of being stored by the forward.  workspace: device, 256-byte aligned,
  * >= mpipe_encoder_layer_bwd_workspace_bytes.  About twenty launches on `stream`, nothing allocated.  bwd_items_dev /
  * n_bwd_items are the plan's backward list.  Sums over tokens use fp32 atomics and TMA reductions: parameter gradients
  * are reproducible to rounding order only.

@@ -10,6 +10,7 @@
 #include <algorithm>
 
 #include "common.h"
+#include "gelu.cuh"
 
 namespace mpipe {
 
@@ -289,6 +290,22 @@ __global__ void __launch_bounds__(256) colsum_kernel(const __nv_bfloat16* __rest
     }
 }
 
+// f = GELU(u), element-wise over a contiguous bf16 array (16 bytes per thread).  Used by a trained forward, which keeps
+// the pre-activation u for the backward and therefore cannot fuse the activation into the projection's epilogue.
+__global__ void __launch_bounds__(256) gelu_kernel(const uint4* __restrict__ u, uint4* __restrict__ f, int64_t n_chunks) {
+    const int64_t i = int64_t(blockIdx.x) * 256 + threadIdx.x;
+    if (i >= n_chunks) return;
+    const uint4 q = u[i];
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const __nv_bfloat162 pk = __floats2bfloat162_rn(gelu_erf(__uint_as_float(w[j] << 16)), gelu_erf(__uint_as_float(w[j] & 0xffff0000u)));
+        o[j] = *reinterpret_cast<const uint32_t*>(&pk);
+    }
+    f[i] = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 
 }  // namespace mpipe
@@ -405,9 +422,10 @@ size_t mpipe_encoder_layer_workspace_bytes(int32_t n_tokens, int32_t hidden, int
     using namespace mpipe;
     if (n_tokens <= 0 || hidden <= 0 || ffn <= 0) return 0;
     const size_t t = size_t(n_tokens);
-    // normalised rows (reused by both norms), packed QKV, attention output, x1, MLP hidden
+    // normalised rows (reused by both norms), packed QKV, attention output, x1, MLP hidden GELU(u), and u itself (kept by a
+    // trained forward for the backward; one size serves both modes)
     return align256(t * hidden * 2) + align256(t * 3 * hidden * 2) + align256(t * hidden * 2) + align256(t * hidden * 2) +
-           align256(t * ffn * 2);
+           2 * align256(t * ffn * 2);
 }
 
 int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weights_t* w, int32_t n_tokens, int32_t hidden,
@@ -429,7 +447,8 @@ int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weight
     uint8_t* qkv = ws;                ws += align256(t * 3 * hidden * 2);
     uint8_t* attn = ws;               ws += align256(t * hidden * 2);
     uint8_t* x1 = ws;                 ws += align256(t * hidden * 2);
-    uint8_t* fc1 = ws;
+    uint8_t* fc1 = ws;                ws += align256(t * ffn * 2);
+    uint8_t* ubuf = ws;
     int32_t rc;
     if ((rc = mpipe_layernorm_fwd(x, w->ln1_gamma, w->ln1_beta, norm, n_tokens, hidden, hidden, hidden, ln_eps, stream)) != MPIPE_OK) return rc;
     if ((rc = mpipe_linear_fwd(norm, w->w_qkv, w->b_qkv, nullptr, qkv, n_tokens, 3 * hidden, hidden, hidden, hidden, 0,
@@ -447,8 +466,17 @@ int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weight
     if ((rc = mpipe_linear_fwd(attn, w->w_o, w->b_o, x, x1, n_tokens, hidden, hidden, hidden, hidden, hidden, hidden, 0,
                                status_buf, stream)) != MPIPE_OK) return rc;
     if ((rc = mpipe_layernorm_fwd(x1, w->ln2_gamma, w->ln2_beta, norm, n_tokens, hidden, hidden, hidden, ln_eps, stream)) != MPIPE_OK) return rc;
-    if ((rc = mpipe_linear_fwd(norm, w->w_fc1, w->b_fc1, nullptr, fc1, n_tokens, ffn, hidden, hidden, hidden, 0, ffn,
-                               MPIPE_LINEAR_GELU, status_buf, stream)) != MPIPE_OK) return rc;
+    if (mode == MPIPE_ENC_TRAINED) {   // the backward needs the pre-activation: keep it, apply the activation separately
+        if ((rc = mpipe_linear_fwd(norm, w->w_fc1, w->b_fc1, nullptr, ubuf, n_tokens, ffn, hidden, hidden, hidden, 0, ffn, 0,
+                                   status_buf, stream)) != MPIPE_OK) return rc;
+        const int64_t n_chunks = int64_t(t) * ffn / 8;
+        gelu_kernel<<<int((n_chunks + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+            reinterpret_cast<const uint4*>(ubuf), reinterpret_cast<uint4*>(fc1), n_chunks);
+        if (cudaGetLastError() != cudaSuccess) return MPIPE_ERR_CUDA;
+    } else if ((rc = mpipe_linear_fwd(norm, w->w_fc1, w->b_fc1, nullptr, fc1, n_tokens, ffn, hidden, hidden, hidden, 0, ffn,
+                                      MPIPE_LINEAR_GELU, status_buf, stream)) != MPIPE_OK) {
+        return rc;
+    }
     return mpipe_linear_fwd(fc1, w->w_fc2, w->b_fc2, x1, y, n_tokens, hidden, ffn, ffn, ffn, hidden, hidden, 0, status_buf, stream);
 }
 
@@ -456,8 +484,8 @@ size_t mpipe_encoder_layer_bwd_workspace_bytes(int32_t n_tokens, int32_t hidden,
     using namespace mpipe;
     if (n_tokens <= 0 || hidden <= 0 || n_heads <= 0 || ffn <= 0 || (hidden % n_heads) != 0) return 0;
     const size_t t = size_t(n_tokens);
-    // pre-activation u, dL/du, dL/dqkv, dL/dx1, one [T, hidden] temporary, the attention backward's own workspace
-    return 2 * align256(t * ffn * 2) + align256(t * 3 * hidden * 2) + 2 * align256(t * hidden * 2) +
+    // dL/du, dL/dqkv, dL/dx1, one [T, hidden] temporary, the attention backward's own workspace
+    return align256(t * ffn * 2) + align256(t * 3 * hidden * 2) + 2 * align256(t * hidden * 2) +
            align256(mpipe_attn_workspace_bytes(n_tokens, n_heads, hidden / n_heads, MPIPE_ENC_TRAINED));
 }
 
@@ -481,15 +509,15 @@ int32_t mpipe_encoder_layer_bwd(const void* dy, const void* x, void* dx, const m
     const int32_t head_dim = hidden / n_heads;
     const size_t t = size_t(n_tokens);
     const int64_t h = hidden, h3 = 3 * int64_t(hidden), f = ffn;
-    // what the forward left in its workspace: LN output (stale), packed q|k|v (q, k rotated), attention output, x1, GELU(u)
+    // what the forward left in its workspace: LN output (stale), packed q|k|v (q, k rotated), attention output, x1, GELU(u), u
     uint8_t* fw = static_cast<uint8_t*>(fwd_workspace);
     uint8_t* norm = fw;               fw += align256(t * hidden * 2);
     uint8_t* qkv = fw;                fw += align256(t * 3 * hidden * 2);
     uint8_t* attn = fw;               fw += align256(t * hidden * 2);
     uint8_t* x1 = fw;                 fw += align256(t * hidden * 2);
-    uint8_t* act = fw;
+    uint8_t* act = fw;                fw += align256(t * ffn * 2);
+    uint8_t* ubuf = fw;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    uint8_t* ubuf = ws;               ws += align256(t * ffn * 2);
     uint8_t* dubuf = ws;              ws += align256(t * ffn * 2);
     uint8_t* dqkv = ws;               ws += align256(t * 3 * hidden * 2);
     uint8_t* dx1 = ws;                ws += align256(t * hidden * 2);
@@ -502,7 +530,6 @@ int32_t mpipe_encoder_layer_bwd(const void* dy, const void* x, void* dx, const m
     MPIPE_TRY(mpipe_layernorm_fwd(x1, w->ln2_gamma, w->ln2_beta, norm, n_tokens, hidden, h, h, ln_eps, stream));                 // m
     MPIPE_TRY(mpipe_linear_wgrad(dy, act, g->w_fc2, n_tokens, hidden, ffn, h, f, f, status_buf, stream));                          // dW2 += dy^T GELU(u)
     MPIPE_TRY(mpipe_colsum_accumulate(dy, g->b_fc2, n_tokens, hidden, h, stream));
-    MPIPE_TRY(mpipe_linear_fwd(norm, w->w_fc1, w->b_fc1, nullptr, ubuf, n_tokens, ffn, hidden, h, h, 0, f, 0, status_buf, stream)); // u (recomputed)
     MPIPE_TRY(mpipe_linear_dgrad(dy, w->w_fc2, ubuf, nullptr, dubuf, n_tokens, hidden, ffn, h, f, f, 0, f, status_buf, stream));    // du = (dy W2) o GELU'(u)
     MPIPE_TRY(mpipe_linear_wgrad(dubuf, norm, g->w_fc1, n_tokens, ffn, hidden, f, h, h, status_buf, stream));                     // dW1 += du^T m
     MPIPE_TRY(mpipe_colsum_accumulate(dubuf, g->b_fc1, n_tokens, ffn, f, stream));

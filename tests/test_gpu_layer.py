@@ -125,10 +125,12 @@ def test_layer_with_rope_matches_oracle():
     assert np.abs(lse - parts["lse"]).max() <= 2e-2
 
 
-def test_layer_frozen_equals_trained_output():
+def test_layer_frozen_agrees_with_trained_output():
+    # the trained forward keeps the MLP pre-activation (rounded to bf16) for the backward and applies the activation to
+    # that; the frozen one applies it to the fp32 accumulator: same result to bf16 rounding of one intermediate
     y_t, ref, _, _ = _run_layer([200, 56], 4, 64, 512, B.TRAINED)
     y_f, _, lse, _ = _run_layer([200, 56], 4, 64, 512, B.FROZEN)
-    assert lse is None and np.array_equal(y_t, y_f)
+    assert lse is None and rel_l2(y_f, y_t) <= 4e-3 and rel_l2(y_f, ref) <= LAYER_REL_L2   # one more bf16 rounding (2^-9) of one stage
 
 
 def test_layer_argument_checks():
