@@ -322,6 +322,28 @@ int32_t mpipe_encoder_layer_bwd(const void* dy, const void* x, void* dx, const m
                                 float ln_eps, const float* rope_cos, const float* rope_sin, int32_t mode,
                                 const float* lse, void* fwd_workspace, void* workspace, size_t workspace_bytes,
                                 int32_t* status_buf, void* stream);
+/*
+ * The whole encoder: n_layers blocks of the same shape applied in turn -- what one Fwd(enc, r, m) / Bwd(enc, r, m)
+ * event executes.  layers / grads: host arrays of n_layers structs.  lse: fp32 [n_layers, n_heads, n_tokens] when
+ * TRAINED.  mpipe_encoder_fwd's workspace (mpipe_encoder_workspace_bytes): FROZEN, one layer's workspace and two
+ * activation buffers, reused; TRAINED, every layer's workspace and input, kept for mpipe_encoder_bwd, which takes
+ * it as fwd_workspace (untouched) plus a workspace of its own (mpipe_encoder_bwd_workspace_bytes).  The rope tables
+ * and the plan are shared by all layers.  FROZEN: mpipe_encoder_bwd returns MPIPE_OK at once.
+ */
+size_t mpipe_encoder_workspace_bytes(int32_t n_layers, int32_t n_tokens, int32_t hidden, int32_t ffn, int32_t mode);
+size_t mpipe_encoder_bwd_workspace_bytes(int32_t n_tokens, int32_t hidden, int32_t n_heads, int32_t ffn);
+int32_t mpipe_encoder_fwd(const void* x, void* y, const mpipe_layer_weights_t* layers, int32_t n_layers, int32_t n_tokens,
+                          int32_t hidden, int32_t n_heads, int32_t ffn, const int32_t* cu_seqlens_dev, int32_t n_seg,
+                          int32_t max_seqlen, const mpipe_work_item_t* fwd_items_dev, int32_t n_fwd_items,
+                          float softmax_scale, float ln_eps, const float* rope_cos, const float* rope_sin, int32_t mode,
+                          float* lse, void* workspace, size_t workspace_bytes, int32_t* status_buf, void* stream);
+int32_t mpipe_encoder_bwd(const void* dy, const void* x, void* dx, const mpipe_layer_weights_t* layers,
+                          const mpipe_layer_grads_t* grads, int32_t n_layers, int32_t n_tokens, int32_t hidden,
+                          int32_t n_heads, int32_t ffn, const int32_t* cu_seqlens_dev, int32_t n_seg, int32_t max_seqlen,
+                          const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items, float softmax_scale, float ln_eps,
+                          const float* rope_cos, const float* rope_sin, int32_t mode, const float* lse,
+                          void* fwd_workspace, void* workspace, size_t workspace_bytes, int32_t* status_buf,
+                          void* stream);
 size_t mpipe_encoder_layer_workspace_bytes(int32_t n_tokens, int32_t hidden, int32_t ffn);
 int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weights_t* w, int32_t n_tokens,
                                 int32_t hidden, int32_t n_heads, int32_t ffn, const int32_t* cu_seqlens_dev,

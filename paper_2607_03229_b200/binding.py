@@ -32,6 +32,12 @@ ITEM_DTYPE = np.dtype([(n, np.int32) for n in ("seg", "tile", "row_start", "row_
 
 _i32, _i64, _vp, _f32, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float, ctypes.c_size_t
 _SIGNATURES = {
+    "mpipe_encoder_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32, _i32]),
+    "mpipe_encoder_bwd_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32]),
+    "mpipe_encoder_fwd": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32, _vp, _i32, _i32, _vp, _i32, _f32, _f32, _vp, _vp,
+                                 _i32, _vp, _vp, _sz, _vp, _vp]),
+    "mpipe_encoder_bwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32, _vp, _i32, _i32, _vp, _i32, _f32, _f32,
+                                 _vp, _vp, _i32, _vp, _vp, _vp, _sz, _vp, _vp]),
     "mpipe_encoder_layer_bwd_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32]),
     "mpipe_encoder_layer_bwd": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _i32, _i32, _vp, _i32, _f32, _f32,
                                        _vp, _vp, _i32, _vp, _vp, _vp, _sz, _vp, _vp]),
@@ -374,6 +380,49 @@ def encoder_layer_bwd(dy, x, dx, weights: LayerWeights, grads: LayerGrads, n_hea
         _ptr(fwd_workspace), _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
         _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_encoder_layer_bwd")
+
+
+def _struct_array(items):
+    arr = (type(items[0]) * len(items))()
+    for i, it in enumerate(items):
+        ctypes.memmove(ctypes.addressof(arr) + i * ctypes.sizeof(it), ctypes.addressof(it), ctypes.sizeof(it))
+    arr._keep = items
+    return arr
+
+
+def encoder_workspace_bytes(n_layers: int, n_tokens: int, hidden: int, ffn: int, mode: int) -> int:
+    return load().mpipe_encoder_workspace_bytes(n_layers, n_tokens, hidden, ffn, mode)
+
+
+def encoder_bwd_workspace_bytes(n_tokens: int, hidden: int, n_heads: int, ffn: int) -> int:
+    return load().mpipe_encoder_bwd_workspace_bytes(n_tokens, hidden, n_heads, ffn)
+
+
+def encoder_fwd(x, y, layers, n_heads: int, ffn: int, plan: SegPlan, softmax_scale: float, ln_eps: float, workspace, lse=None,
+                status_buf=None, stream=None, rope=None) -> None:
+    """mpipe_encoder_fwd: `layers` is a list of LayerWeights; lse fp32 [L, H, T] for a trained plan."""
+    T, hidden = x.shape
+    arr = _struct_array(layers)
+    st = load().mpipe_encoder_fwd(
+        _ptr(x), _ptr(y), ctypes.addressof(arr), len(layers), T, hidden, n_heads, ffn, _ptr(plan.cu_seqlens_dev), plan.n_seg,
+        plan.max_seqlen, _ptr(plan.fwd_items_dev), int(plan.fwd_items.size), softmax_scale, ln_eps,
+        _ptr(None if rope is None else rope[0]), _ptr(None if rope is None else rope[1]), plan.mode, _ptr(lse), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _ptr(status_buf), _stream(stream))
+    _check(st, "mpipe_encoder_fwd")
+
+
+def encoder_bwd(dy, x, dx, layers, grads, n_heads: int, ffn: int, plan: SegPlan, softmax_scale: float, ln_eps: float, lse,
+                fwd_workspace, workspace, status_buf=None, stream=None, rope=None) -> None:
+    """mpipe_encoder_bwd: `layers` / `grads` are lists of LayerWeights / LayerGrads."""
+    T, hidden = x.shape
+    la, ga = _struct_array(layers), _struct_array(grads)
+    st = load().mpipe_encoder_bwd(
+        _ptr(dy), _ptr(x), _ptr(dx), ctypes.addressof(la), ctypes.addressof(ga), len(layers), T, hidden, n_heads, ffn,
+        _ptr(plan.cu_seqlens_dev), plan.n_seg, plan.max_seqlen, _ptr(plan.bwd_items_dev), int(plan.bwd_items.size), softmax_scale,
+        ln_eps, _ptr(None if rope is None else rope[0]), _ptr(None if rope is None else rope[1]), plan.mode, _ptr(lse),
+        _ptr(fwd_workspace), _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+        _ptr(status_buf), _stream(stream))
+    _check(st, "mpipe_encoder_bwd")
 
 
 def encoder_layer_workspace_bytes(n_tokens: int, hidden: int, ffn: int) -> int:

@@ -554,4 +554,84 @@ int32_t mpipe_encoder_layer_bwd(const void* dy, const void* x, void* dx, const m
     return MPIPE_OK;
 }
 
+// ---- the whole encoder: n_layers identical blocks, one after the other (what Fwd(enc, r, m) / Bwd(enc, r, m) run)
+size_t mpipe_encoder_workspace_bytes(int32_t n_layers, int32_t n_tokens, int32_t hidden, int32_t ffn, int32_t mode) {
+    using namespace mpipe;
+    if (n_layers <= 0 || n_tokens <= 0 || hidden <= 0 || ffn <= 0) return 0;
+    const size_t per_layer = mpipe_encoder_layer_workspace_bytes(n_tokens, hidden, ffn);
+    const size_t act = align256(size_t(n_tokens) * hidden * 2);
+    // FROZEN: one layer workspace reused + two ping-pong activations.  TRAINED: every layer's workspace and input are kept.
+    return mode == MPIPE_ENC_TRAINED ? size_t(n_layers) * (per_layer + act) : per_layer + 2 * act;
+}
+
+int32_t mpipe_encoder_fwd(const void* x, void* y, const mpipe_layer_weights_t* layers, int32_t n_layers, int32_t n_tokens,
+                          int32_t hidden, int32_t n_heads, int32_t ffn, const int32_t* cu_seqlens_dev, int32_t n_seg,
+                          int32_t max_seqlen, const mpipe_work_item_t* fwd_items_dev, int32_t n_fwd_items, float softmax_scale,
+                          float ln_eps, const float* rope_cos, const float* rope_sin, int32_t mode, float* lse, void* workspace,
+                          size_t workspace_bytes, int32_t* status_buf, void* stream) {
+    using namespace mpipe;
+    if (n_layers <= 0 || layers == nullptr || n_tokens < 0) return MPIPE_ERR_INVALID_ARG;
+    if (mode != MPIPE_ENC_FROZEN && mode != MPIPE_ENC_TRAINED) return MPIPE_ERR_INVALID_ARG;
+    if (n_tokens == 0) return MPIPE_OK;
+    if (x == nullptr || y == nullptr || (mode == MPIPE_ENC_TRAINED && lse == nullptr)) return MPIPE_ERR_INVALID_ARG;
+    if (workspace == nullptr || workspace_bytes < mpipe_encoder_workspace_bytes(n_layers, n_tokens, hidden, ffn, mode)) return MPIPE_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MPIPE_ERR_UNSUPPORTED;
+    const size_t per_layer = mpipe_encoder_layer_workspace_bytes(n_tokens, hidden, ffn);
+    const size_t act = align256(size_t(n_tokens) * hidden * 2);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const void* in = x;
+    for (int l = 0; l < n_layers; ++l) {
+        // TRAINED: layer l's workspace at l * (per_layer + act), its OUTPUT (= layer l+1's input) right behind it
+        uint8_t* lws = mode == MPIPE_ENC_TRAINED ? ws + size_t(l) * (per_layer + act) : ws;
+        void* out = (l == n_layers - 1) ? y
+                    : (mode == MPIPE_ENC_TRAINED ? static_cast<void*>(lws + per_layer) : static_cast<void*>(ws + per_layer + size_t(l & 1) * act));
+        float* lse_l = mode == MPIPE_ENC_TRAINED ? lse + size_t(l) * n_heads * size_t(n_tokens) : nullptr;
+        const int32_t rc = mpipe_encoder_layer_fwd(in, out, layers + l, n_tokens, hidden, n_heads, ffn, cu_seqlens_dev, n_seg, max_seqlen,
+                                                   fwd_items_dev, n_fwd_items, softmax_scale, ln_eps, rope_cos, rope_sin, mode, lse_l, lws,
+                                                   per_layer, status_buf, stream);
+        if (rc != MPIPE_OK) return rc;
+        in = out;
+    }
+    return MPIPE_OK;
+}
+
+int32_t mpipe_encoder_bwd(const void* dy, const void* x, void* dx, const mpipe_layer_weights_t* layers, const mpipe_layer_grads_t* grads,
+                          int32_t n_layers, int32_t n_tokens, int32_t hidden, int32_t n_heads, int32_t ffn,
+                          const int32_t* cu_seqlens_dev, int32_t n_seg, int32_t max_seqlen, const mpipe_work_item_t* bwd_items_dev,
+                          int32_t n_bwd_items, float softmax_scale, float ln_eps, const float* rope_cos, const float* rope_sin,
+                          int32_t mode, const float* lse, void* fwd_workspace, void* workspace, size_t workspace_bytes,
+                          int32_t* status_buf, void* stream) {
+    using namespace mpipe;
+    if (mode != MPIPE_ENC_FROZEN && mode != MPIPE_ENC_TRAINED) return MPIPE_ERR_INVALID_ARG;
+    if (mode == MPIPE_ENC_FROZEN) return MPIPE_OK;
+    if (n_layers <= 0 || layers == nullptr || grads == nullptr || n_tokens < 0) return MPIPE_ERR_INVALID_ARG;
+    if (n_tokens == 0) return MPIPE_OK;
+    if (dy == nullptr || x == nullptr || dx == nullptr || lse == nullptr || fwd_workspace == nullptr) return MPIPE_ERR_INVALID_ARG;
+    const size_t per_bwd = mpipe_encoder_layer_bwd_workspace_bytes(n_tokens, hidden, n_heads, ffn);
+    const size_t act = align256(size_t(n_tokens) * hidden * 2);
+    if (workspace == nullptr || workspace_bytes < per_bwd + 2 * act) return MPIPE_ERR_WORKSPACE;
+    if (((reinterpret_cast<uintptr_t>(workspace) | reinterpret_cast<uintptr_t>(fwd_workspace)) & 255u) != 0) return MPIPE_ERR_UNSUPPORTED;
+    const size_t per_layer = mpipe_encoder_layer_workspace_bytes(n_tokens, hidden, ffn);
+    uint8_t* fws = static_cast<uint8_t*>(fwd_workspace);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const void* grad_in = dy;
+    for (int l = n_layers - 1; l >= 0; --l) {
+        uint8_t* lws = fws + size_t(l) * (per_layer + act);
+        const void* in = (l == 0) ? x : static_cast<const void*>(fws + size_t(l - 1) * (per_layer + act) + per_layer);   // layer l's input
+        void* grad_out = (l == 0) ? dx : static_cast<void*>(ws + per_bwd + size_t(l & 1) * act);
+        const int32_t rc = mpipe_encoder_layer_bwd(grad_in, in, grad_out, layers + l, grads + l, n_tokens, hidden, n_heads, ffn, cu_seqlens_dev,
+                                                   n_seg, max_seqlen, bwd_items_dev, n_bwd_items, softmax_scale, ln_eps, rope_cos, rope_sin,
+                                                   mode, lse + size_t(l) * n_heads * size_t(n_tokens), lws, ws, per_bwd, status_buf, stream);
+        if (rc != MPIPE_OK) return rc;
+        grad_in = grad_out;
+    }
+    return MPIPE_OK;
+}
+
+size_t mpipe_encoder_bwd_workspace_bytes(int32_t n_tokens, int32_t hidden, int32_t n_heads, int32_t ffn) {
+    using namespace mpipe;
+    const size_t per_bwd = mpipe_encoder_layer_bwd_workspace_bytes(n_tokens, hidden, n_heads, ffn);
+    return per_bwd == 0 ? 0 : per_bwd + 2 * align256(size_t(n_tokens) * hidden * 2);
+}
+
 }  // extern "C"

@@ -374,3 +374,48 @@ def test_layer_bwd_full_size_sampled_segments():
     # the bias gradient of the last projection is the plain column sum of dy: an exact, full-size check of the accumulation
     ref_b = OL.widen(dy).sum(axis=0)
     assert np.abs(grads_t["b_fc2"].cpu().double().numpy() - ref_b).max() <= 1e-5 * np.abs(ref_b).max() + 1e-3
+
+
+def test_encoder_stack_matches_oracle():
+    """Three layers through mpipe_encoder_fwd / mpipe_encoder_bwd against the oracle's layer applied three times."""
+    counts, H, D, ffn, L = [300, 1, 129], 4, 64, 512, 3
+    hidden, T = H * D, sum(counts)
+    pbs = [W.layer_params_bf16(40 + l, hidden, ffn) for l in range(L)]
+    x, dy = W.normal_bf16(40, 0, (T, hidden)), W.normal_bf16(40, 1, (T, hidden))
+    plan = B.seg_plan(counts, B.TRAINED).to_device()
+    layers = [B.LayerWeights.from_tensors(**{k: to_dev(v) for k, v in pb.items()}) for pb in pbs]
+    grads_t = [{k: torch.zeros(v.shape, dtype=torch.float32, device="cuda") for k, v in pb.items()} for pb in pbs]
+    grads = [B.LayerGrads.from_tensors(**g) for g in grads_t]
+    xd, dyd = to_dev(x), to_dev(dy)
+    y, dx = torch.empty_like(xd), torch.empty_like(xd)
+    lse = torch.empty((L, H, T), dtype=torch.float32, device="cuda")
+    ws_f = torch.empty(B.encoder_workspace_bytes(L, T, hidden, ffn, B.TRAINED), dtype=torch.uint8, device="cuda")
+    ws_b = torch.empty(B.encoder_bwd_workspace_bytes(T, hidden, H, ffn), dtype=torch.uint8, device="cuda")
+    st = status_buf()
+    scale = 0.125
+    B.encoder_fwd(xd, y, layers, H, ffn, plan, scale, 1e-6, ws_f, lse, st)
+    B.encoder_bwd(dyd, xd, dx, layers, grads, H, ffn, plan, scale, 1e-6, lse, ws_f, ws_b, st)
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[0] == 0
+    # frozen stack: same forward result to bf16 rounding, through the small reused workspace
+    plan_f = B.seg_plan(counts, B.FROZEN).to_device()
+    y_f = torch.empty_like(xd)
+    ws_small = torch.empty(B.encoder_workspace_bytes(L, T, hidden, ffn, B.FROZEN), dtype=torch.uint8, device="cuda")
+    B.encoder_fwd(xd, y_f, layers, H, ffn, plan_f, scale, 1e-6, ws_small, None, st)
+    torch.cuda.synchronize()
+    cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    ows = [OL.LayerWeights(g1=OL.widen(pb["ln1_gamma"]), b1=OL.widen(pb["ln1_beta"]), wqkv=OL.widen(pb["w_qkv"]),
+                           bqkv=OL.widen(pb["b_qkv"]), wo=OL.widen(pb["w_o"]), bo=OL.widen(pb["b_o"]),
+                           g2=OL.widen(pb["ln2_gamma"]), b2=OL.widen(pb["ln2_beta"]), w1=OL.widen(pb["w_fc1"]),
+                           bb1=OL.widen(pb["b_fc1"]), w2=OL.widen(pb["w_fc2"]), bb2=OL.widen(pb["b_fc2"])) for pb in pbs]
+    acts = [OL.widen(x)]
+    for ow in ows:
+        acts.append(OL.encoder_layer_fwd(acts[-1], ow, cu, H, scale, 1e-6)[0])
+    assert rel_l2(to_f64(y), acts[-1]) <= 2e-2 and rel_l2(to_f64(y_f), acts[-1]) <= 2e-2
+    g = OL.widen(dy)
+    for l in range(L - 1, -1, -1):
+        g, pg = OL.encoder_layer_bwd(acts[l], ows[l], cu, H, scale, 1e-6, g)
+        for name, ref in pg.items():
+            got = grads_t[l][name].cpu().double().numpy()
+            assert rel_l2(got, ref.reshape(got.shape)) <= 3e-2, (l, name, rel_l2(got, ref.reshape(got.shape)))
+    assert rel_l2(to_f64(dx), g) <= 3e-2
