@@ -74,6 +74,46 @@ def share_rows(t: "torch.Tensor", src_rank: int):
     return B.PeerRows(handle, rows, hidden, stride)
 
 
+LAYER_PARAM_SHAPES = (("ln1_gamma", lambda h, f: (h,)), ("ln1_beta", lambda h, f: (h,)), ("w_qkv", lambda h, f: (3 * h, h)),
+                      ("b_qkv", lambda h, f: (3 * h,)), ("w_o", lambda h, f: (h, h)), ("b_o", lambda h, f: (h,)),
+                      ("ln2_gamma", lambda h, f: (h,)), ("ln2_beta", lambda h, f: (h,)), ("w_fc1", lambda h, f: (f, h)),
+                      ("b_fc1", lambda h, f: (f,)), ("w_fc2", lambda h, f: (h, f)), ("b_fc2", lambda h, f: (h,)))
+
+
+def alloc_grad_bucket(n_layers: int, hidden: int, ffn: int, device="cuda"):
+    """One flat fp32 buffer for the gradients of the whole encoder and, per layer, a dict of views into it (the twelve
+    tensors mpipe_encoder_layer_bwd accumulates into).  One buffer = one all-reduce per step: a bucket sized for launch
+    latency rather than per-tensor collectives.  Every view starts on a 16-byte boundary."""
+    sizes, offs, total = [], [], 0
+    for _ in range(n_layers):
+        for name, shape in LAYER_PARAM_SHAPES:
+            shp = shape(hidden, ffn)
+            n = 1
+            for d in shp:
+                n *= d
+            offs.append(total)
+            sizes.append((name, shp, n))
+            total += (n + 3) // 4 * 4
+    flat = torch.zeros(total, dtype=torch.float32, device=device)
+    layers, i = [], 0
+    for _ in range(n_layers):
+        views = {}
+        for _name in LAYER_PARAM_SHAPES:
+            name, shp, n = sizes[i]
+            views[name] = flat[offs[i]:offs[i] + n].view(shp)
+            i += 1
+        layers.append(views)
+    return flat, layers
+
+
+def dp_reduce(flat_grads: "torch.Tensor", group=None) -> None:
+    """DpReduce(enc, ReplicaGroup) (Section 4.1): the trainable, transposed encoder is replicated on every rank of the
+    replica group and each rank saw only its own microbatches, so the accumulated fp32 gradients are summed over the
+    group -- one all-reduce of the bucket (NCCL on GPUs, NVLS inside the switch when available).  A no-op for one rank."""
+    if dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(flat_grads, op=dist.ReduceOp.SUM, group=group)
+
+
 def shutdown() -> None:
     if dist.is_initialized():
         dist.destroy_process_group()

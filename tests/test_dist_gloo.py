@@ -63,3 +63,38 @@ def test_seam_targets_route_every_microbatch_to_the_first_stage():
     ship, local = D.seam_targets(owner, first_stage_rank=1)
     assert sorted(local + [m for v in ship.values() for m in v]) == list(range(len(owner)))
     assert all(owner[m] == r for r, v in ship.items() for m in v) and all(owner[m] == 1 for m in local)
+
+
+def _reduce_worker(rank, world, port, out):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    import torch
+    from paper_2607_03229_b200 import dist as D
+    D.init("gloo")
+    flat, layers = D.alloc_grad_bucket(2, 16, 48, device="cpu")
+    # every view is a window of the bucket: writing through the views fills it
+    for l, views in enumerate(layers):
+        for i, (name, t) in enumerate(views.items()):
+            t.fill_(float((rank + 1) * (10 * l + i + 1)))
+    before = flat.clone()
+    D.dp_reduce(flat)                      # DpReduce(enc, ReplicaGroup): sum over the two replicas
+    ok = bool(torch.equal(flat, before * 3 / (rank + 1))) and all(t.data_ptr() % 16 == 0 for v in layers for t in v.values())
+    shapes = {k: tuple(v.shape) for k, v in layers[0].items()}
+    out.put((rank, ok, shapes["w_qkv"], shapes["w_fc2"], int(flat.numel())))
+    D.shutdown()
+
+
+def test_dp_reduce_sums_the_gradient_bucket_over_replicas():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_reduce_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, ok, s_qkv, s_fc2, n in res:
+        assert ok and s_qkv == (48, 16) and s_fc2 == (16, 48)
+        assert n >= 2 * (4 * 16 * 16 + 2 * 16 * 48)
