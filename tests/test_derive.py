@@ -217,3 +217,44 @@ def test_library_validity_normalize_stage_index_and_errors():
     bad[0] = [bad[0][1], bad[0][0], bad[0][2]]
     with pytest.raises(B.MpipeError):                           # a cycle is not an order graph
         B.order_makespan(d.events, np.concatenate([d.edges, bad[:1]]), np.ones(len(d.events)), 2)
+
+
+# ------------------------------------------------------------------------------------------ derive + makespan together
+def _makespan(sk, cut, L, tr, P, M, owner, cost_of):
+    d = B.derive([SK[s] for s in sk], cut, L, [int(t) for t in tr], P, M, owner)
+    ev, _ = _as_oracle(d)
+    T, start, bub = B.order_makespan(d.events, d.edges, [cost_of(e) for e in ev], P)
+    return T, bub, ev
+
+
+def test_transposed_encoder_is_free_when_it_costs_nothing_and_never_worse_than_a_pipelined_one():
+    P, M = 4, 8
+    unit = lambda e: 1.0 if (e.kind in ("Fwd", "Bwd") and e.region == 2) else 0.0
+    # a frozen encoder that costs nothing: the step is the backbone's 1F1B step, 2 (M + P - 1) with unit stage costs
+    T, bub, _ = _makespan(["transpose", "1f1b"], [4], 12, [False, True], P, M, None, unit)
+    assert T == 2 * (M + P - 1) and list(bub) == [T - 2 * M] * P
+    # the same model with the encoder as one more pipelined region (region 1 sharded over the same ranks, each rank's slab
+    # costing e / P per microbatch) against the transposed encoder (the whole e on the owner): the transposed step is never
+    # longer, and it is strictly shorter once the encoder is not negligible -- the warm-up bubble absorbs it
+    for e_cost in (0.5, 2.0):
+        enc_sharded = lambda e: (e_cost / P if e.region == 1 else 1.0) if e.kind == "Fwd" else (1.0 if e.kind == "Bwd" and e.region == 2 else 0.0)
+        enc_transposed = lambda e: (e_cost if e.region == 1 else 1.0) if e.kind == "Fwd" else (1.0 if e.kind == "Bwd" and e.region == 2 else 0.0)
+        T_pipe, _, _ = _makespan(["1f1b", "1f1b"], [4], 12, [False, True], P, M, None, enc_sharded)
+        owner = [(P - 1) - (m % P) for m in range(M)]     # later ranks have the longer warm-up slots
+        T_tr, bub_tr, ev = _makespan(["transpose", "1f1b"], [4], 12, [False, True], P, M, owner, enc_transposed)
+        assert T_tr <= T_pipe + 1e-12
+        # lower bounds that any order must respect: the busiest rank's work, and microbatch 1's own critical path
+        work = [sum(enc_transposed(e) for e in ev if e.rank == r) for r in range(P)]
+        assert T_tr >= max(work) - 1e-12 and T_tr >= e_cost + 2 * P - 1e-12
+        assert all(abs(b - (T_tr - w_)) < 1e-9 for b, w_ in zip(bub_tr, work))
+
+
+def test_trainable_encoder_adds_its_backward_to_the_cool_down():
+    P, M = 4, 6
+    cost = lambda e: {"Fwd": 1.0, "Bwd": 2.0}.get(e.kind, 0.0) if e.region == 2 else ({"Fwd": 0.25, "Bwd": 0.5}.get(e.kind, 0.0) if e.region == 1 else 0.0)
+    T_frozen, _, ev_f = _makespan(["transpose", "1f1b"], [4], 12, [False, True], P, M, None, cost)
+    T_trained, _, ev_t = _makespan(["transpose", "1f1b"], [4], 12, [True, True], P, M, None, cost)
+    assert T_trained >= T_frozen
+    assert sum(1 for e in ev_t if e.kind == "Bwd" and e.region == 1) == M and not any(e.kind == "Bwd" and e.region == 1 for e in ev_f)
+    # the last encoder backward can only start after the backbone's last backward on rank 0
+    assert T_trained >= T_frozen + 0.5 - 1e-12
