@@ -74,6 +74,60 @@ def test_many_units_per_cta(D):
     check_bwd(counts, 8, D, seed=19)
 
 
+def _random_mix(seed):
+    """Segment lengths drawn around the tile edges (64, 128, 256 rows) and from a wide range, some empty."""
+    edges = [1, 2, 15, 16, 17, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 256, 257, 383, 384, 385, 511, 512, 513]
+    n_seg = int(W.rand_int(seed, 1, 1, 3, 10)[0])
+    pick = W.rand_int(seed, 2, n_seg, 0, 3)
+    edge = W.rand_int(seed, 3, n_seg, 0, len(edges) - 1)
+    wide = W.rand_int(seed, 4, n_seg, 1, 700)
+    return [0 if pick[i] == 0 and i % 4 == 3 else (edges[int(edge[i])] if pick[i] < 2 else int(wide[i])) for i in range(n_seg)]
+
+
+@pytest.mark.parametrize("D", [64, 80])
+@pytest.mark.parametrize("seed", range(8))
+def test_random_length_mixes_forward_and_backward(seed, D):
+    """A seeded sweep over mixes of segment lengths at and around the tile edges, odd head counts included: the
+    forward output, the LSE it hands to the backward and all three gradients against the oracle."""
+    counts = _random_mix(1000 + seed)
+    if sum(counts) == 0:
+        counts = counts + [130]
+    H = 1 + (seed % 3)
+    T = int(sum(counts))
+    q, k, v, do = (W.normal_bf16(3000 + seed, s, (T, H, D)) for s in (1, 2, 3, 4))
+    scale = float(np.float32(1.0 / np.sqrt(D)))
+    o, lse, dq, dk, dv = gpu_fwd_bwd(q, k, v, do, counts, scale)
+    cu = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    O_ref, L_ref = oracle.attn_fwd(q, k, v, cu, scale)
+    assert max_abs(to_f64(o), O_ref) <= 1e-2 and rel_l2(to_f64(o), O_ref) <= 5e-3, counts
+    assert max_abs(to_f64(lse), L_ref) <= 1e-3, counts
+    ref = oracle.attn_bwd(do, q, k, v, cu, scale)
+    for name, g, r in zip(("dq", "dk", "dv"), (dq, dk, dv), ref):
+        if np.linalg.norm(r) == 0:
+            assert np.abs(to_f64(g)).max() <= 1e-2, (counts, name)
+        else:
+            assert rel_l2(to_f64(g), r) <= GRAD_REL_L2, (counts, name, rel_l2(to_f64(g), r))
+
+
+def test_repeated_backward_is_stable():
+    """The same inputs five times over: dK and dV (one issuing warp, fixed accumulation order at head dim 64) come
+    out bit-identical, dQ (fp32 reduce-add in the copy engine, order not fixed) within a bf16 rounding step."""
+    counts = [300, 129, 513, 64, 257]
+    T, H, D = sum(counts), 4, 64
+    q, k, v, do = (W.normal_bf16(77, s, (T, H, D)) for s in (1, 2, 3, 4))
+    scale = float(np.float32(1.0 / np.sqrt(D)))
+    first = None
+    for _ in range(5):
+        _, _, dq, dk, dv = gpu_fwd_bwd(q, k, v, do, counts, scale)
+        got = [x.clone() for x in (dq, dk, dv)]
+        if first is None:
+            first = got
+            continue
+        assert torch.equal(got[1], first[1]) and torch.equal(got[2], first[2])
+        a, b = to_f64(got[0]), to_f64(first[0])
+        assert np.abs(a - b).max() <= 2.0 ** -7 * max(1.0, np.abs(b).max())
+
+
 def test_frozen_backward_is_a_noop():
     w = W.tiny()
     q, k, v = w.qkv()
