@@ -109,10 +109,14 @@ size_t mpipe_attn_workspace_bytes(int32_t total_tokens, int32_t n_heads, int32_t
  *   o         device, bf16, same shape, strides tok_stride_o / head_stride_o              (output)
  *   lse       device, fp32 [n_heads, total_tokens] contiguous; written only when TRAINED (required
  *             then); ignored when FROZEN                                                  (output)
- *   cu_seqlens_dev   device int32[n_seg + 1]   (copy of the plan; validated on the host side only
- *                    through the items, which carry the same ranges)
+ *   cu_seqlens_dev   device int32[n_seg + 1]   (copy of the plan; the kernels take every range from the
+ *                    items, which carry the same boundaries, and do not read it)
  *   fwd_items_dev    device mpipe_work_item_t[n_fwd_items] from mpipe_seg_plan with
- *                    fwd_tile_rows = mpipe_fwd_tile_rows()
+ *                    fwd_tile_rows = mpipe_fwd_tile_rows().  The host cannot inspect device memory at
+ *                    launch time, so the kernel clamps every item to [0, total_tokens) rows before use:
+ *                    an item that does not fit (a plan made for another total_tokens, a corrupted
+ *                    buffer) sets status_buf[0] = MPIPE_ERR_INDEX, status_buf[1] = the unit index, and
+ *                    whatever part of it lies outside the tensors is neither read nor written.
  *   total_tokens == 0 or n_fwd_items == 0: returns MPIPE_OK without launching.
  * Rows past a segment's end inside a tile are computed but never stored.  fp32 accumulation,
  * bf16 probabilities; results are deterministic run to run.
@@ -134,7 +138,12 @@ int32_t mpipe_varlen_attn_fwd(const void* q, const void* k, const void* v, void*
  *   dq, dk, dv device bf16, strides tok_stride_grad / head_stride_grad                    (outputs)
  *   bwd_items_dev  from mpipe_seg_plan with bwd_tile_rows = mpipe_bwd_tile_rows()
  *   workspace      device, >= mpipe_attn_workspace_bytes(...), 256-byte aligned; contents are scratch
- * dQ is accumulated with fp32 atomics across key tiles: its low bits may differ run to run.
+ *                  (fp32 dQ accumulator + Delta).  The alignment is a requirement of the TMA tensor map
+ *                  through which the accumulator is updated.
+ *   Items are clamped to [0, total_tokens) on the device exactly as in the forward (MPIPE_ERR_INDEX).
+ * dQ is summed over key tiles in fp32 by the copy engine (TMA reduce-add from shared memory); the order
+ * of those additions is not fixed, so the low bits of dQ may differ from run to run.  dK and dV are
+ * reproducible at head_dim 64.
  */
 int32_t mpipe_varlen_attn_bwd(const void* dout, const void* q, const void* k, const void* v, const void* o,
                               const float* lse, void* dq, void* dk, void* dv, int64_t tok_stride_qkv,
@@ -165,7 +174,13 @@ int32_t mpipe_varlen_attn_bwd(const void* dout, const void* q, const void* k, co
  *   - The call itself allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
  *     The first call on each device looks up the array's device address once, with that device
  *     current; make that first call before starting any stream capture.  A failed look-up returns
- *     MPIPE_ERR_CUDA.
+ *     MPIPE_ERR_CUDA.  With lazy module loading the CUDA runtime materialises the library's device
+ *     code, this array included, when the first kernel of the library is used, and that first look-up
+ *     may synchronise the device: do one warm-up call at start-up if neither is acceptable later.
+ *     The per-device address cache is plain host memory: first calls on one device from several host
+ *     threads at once are harmless (they store the same value) but are not ordered.
+ *   - Argument errors are reported exactly as by mpipe_varlen_attn_bwd (the same checks run first);
+ *     only then is the size compared with the limit.
  *   - All calls on a device share the one array, which keeps whatever the previous call left in
  *     it.  Nothing needs to be cleared by the caller: each call's first kernel zeroes the
  *     accumulator and rewrites Delta for its own problem.  Because the array is shared, two calls
@@ -444,8 +459,9 @@ int32_t mpipe_order_makespan(const mpipe_event_t* events, int32_t n_events, cons
  * duration, Section 4.3, and this is how a benchmark reads that duration for one kernel): while set,
  * the launch of kernel `which` (0 = attention forward, 1 = attention backward main kernel, 2 = merge
  * / merge_bwd, 3 = mpipe_linear_fwd, 4 = mpipe_layernorm_fwd) records the two cudaEvent_t handles on the call's stream directly before and after
- * it.  NULL handles switch it off.  Process-wide, not thread-safe: set it from the thread that makes
- * the calls.  Returns MPIPE_ERR_INVALID_ARG for an unknown `which`.
+ * it.  NULL handles switch it off.  The setting is per host thread (thread-local): it affects only the
+ * launches the setting thread makes afterwards, so the library keeps no state shared between callers.
+ * Returns MPIPE_ERR_INVALID_ARG for an unknown `which`.
  */
 int32_t mpipe_set_profile_events(int32_t which, void* start_event, void* stop_event);
 

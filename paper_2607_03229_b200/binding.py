@@ -216,11 +216,21 @@ def _thd_strides(t: torch.Tensor):
     return t.stride(0), t.stride(1)
 
 
+def _check_plan(plan: SegPlan, T: int, items_dev, n_items: int, what: str) -> None:
+    """The plan must have been made for these tensors and uploaded: the kernels index the tensors with the
+    rows its items name."""
+    assert plan.total_tokens == T, f"{what}: plan was made for {plan.total_tokens} tokens, tensors hold {T}"
+    if T > 0 and n_items > 0:
+        assert items_dev is not None and plan.cu_seqlens_dev is not None, f"{what}: plan.to_device() first"
+        assert items_dev.numel() == 6 * n_items and items_dev.dtype == torch.int32
+
+
 def varlen_attn_fwd(q, k, v, o, lse, plan: SegPlan, softmax_scale: float, status_buf=None, stream=None) -> None:
     """mpipe_varlen_attn_fwd.  q,k,v,o: bf16 CUDA tensors [T,H,D]; lse: fp32 [H,T] or None (frozen)."""
     T, H, D = q.shape
     assert k.shape == q.shape and v.shape == q.shape and o.shape == q.shape
     assert q.dtype == k.dtype == v.dtype == o.dtype == torch.bfloat16
+    _check_plan(plan, T, plan.fwd_items_dev, int(plan.fwd_items.size), "varlen_attn_fwd")
     ts, hs = _thd_strides(q)
     assert _thd_strides(k) == (ts, hs) and _thd_strides(v) == (ts, hs), "q, k, v must share strides"
     tso, hso = _thd_strides(o)
@@ -233,25 +243,33 @@ def varlen_attn_fwd(q, k, v, o, lse, plan: SegPlan, softmax_scale: float, status
     _check(st, "mpipe_varlen_attn_fwd")
 
 
-def varlen_attn_bwd(dout, q, k, v, o, lse, dq, dk, dv, plan: SegPlan, softmax_scale: float, workspace,
-                    status_buf=None, stream=None) -> None:
-    """mpipe_varlen_attn_bwd.  A frozen plan returns at once (nothing is launched)."""
+def _bwd_args(what, dout, q, k, v, o, lse, dq, dk, dv, plan: SegPlan, softmax_scale: float):
+    """Shape / dtype / stride checks and argument marshalling shared by the two backward entry points."""
     T, H, D = q.shape
     ts, hs = _thd_strides(q)
     tso, hso = _thd_strides(o)
     if plan.mode == TRAINED:
-        assert _thd_strides(k) == (ts, hs) and _thd_strides(v) == (ts, hs)
+        for name, t in (("k", k), ("v", v), ("o", o), ("dout", dout), ("dq", dq), ("dk", dk), ("dv", dv)):
+            assert tuple(t.shape) == (T, H, D) and t.dtype == torch.bfloat16, f"{what}: {name} must be bf16 {(T, H, D)}"
+        assert lse.dtype == torch.float32 and lse.is_contiguous() and tuple(lse.shape) == (H, T)
+        _check_plan(plan, T, plan.bwd_items_dev, int(plan.bwd_items.size), what)
+        assert _thd_strides(k) == (ts, hs) and _thd_strides(v) == (ts, hs), "q, k, v must share strides"
         assert _thd_strides(dout) == (tso, hso), "dout must share o's strides"
         tsg, hsg = _thd_strides(dq)
-        assert _thd_strides(dk) == (tsg, hsg) and _thd_strides(dv) == (tsg, hsg)
+        assert _thd_strides(dk) == (tsg, hsg) and _thd_strides(dv) == (tsg, hsg), "dq, dk, dv must share strides"
     else:
         tsg, hsg = ts, hs
+    return (_ptr(dout), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(dq), _ptr(dk), _ptr(dv), ts, hs, tso, hso,
+            tsg, hsg, _ptr(plan.cu_seqlens_dev), plan.n_seg, plan.total_tokens, plan.max_seqlen,
+            _ptr(plan.bwd_items_dev), int(plan.bwd_items.size), H, D, softmax_scale, plan.mode)
+
+
+def varlen_attn_bwd(dout, q, k, v, o, lse, dq, dk, dv, plan: SegPlan, softmax_scale: float, workspace,
+                    status_buf=None, stream=None) -> None:
+    """mpipe_varlen_attn_bwd.  A frozen plan returns at once (nothing is launched)."""
+    args = _bwd_args("varlen_attn_bwd", dout, q, k, v, o, lse, dq, dk, dv, plan, softmax_scale)
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
-    st = load().mpipe_varlen_attn_bwd(
-        _ptr(dout), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(dq), _ptr(dk), _ptr(dv), ts, hs, tso, hso,
-        tsg, hsg, _ptr(plan.cu_seqlens_dev), plan.n_seg, plan.total_tokens, plan.max_seqlen,
-        _ptr(plan.bwd_items_dev), int(plan.bwd_items.size), H, D, softmax_scale, plan.mode, _ptr(workspace),
-        ws_bytes, _ptr(status_buf), _stream(stream))
+    st = load().mpipe_varlen_attn_bwd(*args, _ptr(workspace), ws_bytes, _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_varlen_attn_bwd")
 
 
@@ -464,15 +482,8 @@ def varlen_attn_bwd_static(dout, q, k, v, o, lse, dq, dk, dv, plan: SegPlan, sof
     """mpipe_varlen_attn_bwd_static: the backward with the library's built-in 32 MiB scratch, for callers
     that may not allocate device memory.  Same tensors as varlen_attn_bwd, no workspace argument; problems
     whose scratch would not fit are refused with ERR_WORKSPACE.  Calls sharing a device must not overlap."""
-    T, H, D = q.shape
-    ts, hs = _thd_strides(q)
-    tso, hso = _thd_strides(o)
-    tsg, hsg = _thd_strides(dq) if plan.mode == TRAINED else (ts, hs)
-    st = load().mpipe_varlen_attn_bwd_static(
-        _ptr(dout), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(dq), _ptr(dk), _ptr(dv), ts, hs, tso, hso,
-        tsg, hsg, _ptr(plan.cu_seqlens_dev), plan.n_seg, plan.total_tokens, plan.max_seqlen,
-        _ptr(plan.bwd_items_dev), int(plan.bwd_items.size), H, D, softmax_scale, plan.mode, _ptr(status_buf),
-        _stream(stream))
+    args = _bwd_args("varlen_attn_bwd_static", dout, q, k, v, o, lse, dq, dk, dv, plan, softmax_scale)
+    st = load().mpipe_varlen_attn_bwd_static(*args, _ptr(status_buf), _stream(stream))
     _check(st, "mpipe_varlen_attn_bwd_static")
 
 

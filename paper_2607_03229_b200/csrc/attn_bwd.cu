@@ -15,8 +15,9 @@
 //   dV  += P^T dO           tcgen05, A operand read from TMEM, dO as MN-major B
 //   dK  += dS^T Q           tcgen05, A operand read from TMEM, Q as MN-major B
 //   dQ_i = dS K             tcgen05, dS^T in shared memory read as an MN-major A, K as MN-major B
-// dQ_i is read back from TMEM by a reducer warpgroup and added to the global fp32 accumulator with
-// vector atomics; dK (x softmax_scale) and dV leave TMEM once per unit.
+// dQ_i is read back from TMEM by a reducer warpgroup, staged in shared memory and added to the global fp32
+// accumulator by the copy engine (cp.reduce.async.bulk.tensor, fp32 add): the order of those additions is not
+// fixed, so the low bits of dQ can differ from run to run.  dK (x softmax_scale) and dV leave TMEM once per unit.
 //
 // Warp roles (512 threads): 0 TMA producer, 1 / 3 tcgen05 issuers of TMEM stage 0 / 1, 2 TMEM allocation and
 // LSE/Delta staging, 4-7 / 8-11 softmax of stage 0 / 1, 12-15 dQ reducer and epilogue.
@@ -29,35 +30,7 @@
 
 namespace mpipe {
 
-// Development aid, compiled in only with -DMPIPE_TRACE: CTA 0 records clock64() at a few pipeline
-// points per role into a global table that mpipe_dbg_read_trace() copies out.
-#ifdef MPIPE_TRACE
-__device__ long long g_trace[4][4096];
-__device__ int g_dbg_flags;   // knock-out switches for experiments: 1 no atomics, 2 no dS smem store, 4 no LSE/Delta smem loads, 8 no ex2
-#define MPIPE_DBG(bit) ((dbg_flags & (bit)) != 0)
-#define MPIPE_TR(role, idx)                                                                  \
-    do {                                                                                     \
-        if (blockIdx.x == 0 && (idx) < 4096) g_trace[role][(idx)] = clock64();               \
-    } while (0)
-__device__ int g_where[16];
-#define MW(call) ((blockIdx.x == (g_dbg_flags >> 16) && (threadIdx.x & 31) == 0 ? (void)(g_where[threadIdx.x >> 5] = __LINE__) : (void)0), call)
-#else
-#define MW(call) call
-#define MPIPE_DBG(bit) false
-#define MPIPE_TR(role, idx) \
-    do {                    \
-    } while (0)
-#endif
-
-#ifndef MPIPE_STREAM
-#define MPIPE_STREAM 1
-#endif
-#ifndef MPIPE_SLEEP_AUX
-#define MPIPE_SLEEP_AUX 100
-#endif
-#ifndef MPIPE_SLEEP_MMA
-#define MPIPE_SLEEP_MMA 0
-#endif
+constexpr int kSleepAux = 100;   // ns between polls of the roles with slack (producer, staging, reducer)
 constexpr int kBwdThreads = 512;
 // Register re-balancing (setmaxnreg): an increase can only draw on registers that other warps of the
 // same CTA have released, so what the 4 service and 4 reducer warps give back must cover what the 8
@@ -142,9 +115,6 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
     const int lane = tid & 31;
-#ifdef MPIPE_TRACE
-    const int dbg_flags = g_dbg_flags;
-#endif
 
     if (tid == 0) {
         abort_flag = 0;
@@ -191,9 +161,14 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         const int g = int(gridDim.x), i = int(blockIdx.x);
         return round * g + ((round & 1) ? g - 1 - i : i);
     };
+    // Items are clamped to the tensors before use (see sanitize_item): a corrupt plan cannot make a store, a
+    // reduction or an LSE / Delta read leave them.
     auto item_at = [&](int u) {
         mpipe_work_item_t z = {0, 0, 0, 0, 0, 0};
-        return (u < n_units) ? p.items[u / p.n_heads] : z;
+        if (u >= n_units) return z;
+        z = p.items[u / p.n_heads];
+        if (sanitize_item(z, kBT, p.total_tokens) && tid == 12 * 32) report_status(p.status_buf, MPIPE_ERR_INDEX, u);
+        return z;
     };
     // Every unit runs an even number of 64-query sub-tiles (a 128-query tile is two of them); a padding
     // sub-tile past the segment end contributes nothing because its probabilities are forced to zero.
@@ -213,7 +188,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 const int n2 = subtiles_of(it);
                 const int kb = unit_it % Cfg::kKVBufs;            // K/V buffer of this unit
                 uint8_t* kv = smem + kb * (2 * Cfg::kTile);
-                ok = MW(mbar_wait<MPIPE_SLEEP_AUX>(&bars.kv_empty[kb], ((unit_it / Cfg::kKVBufs) & 1) ^ 1, &abort_flag));
+                ok = mbar_wait<kSleepAux>(&bars.kv_empty[kb], ((unit_it / Cfg::kKVBufs) & 1) ^ 1, &abort_flag);
                 if (!ok) break;
                 mbar_expect_tx(&bars.kv_full[kb], 2 * Cfg::kTile);
                 tma_load_3d(kv + Cfg::kSmemK, &maps.k, &bars.kv_full[kb], 0, head, it.row_start);
@@ -225,7 +200,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 for (int s = 0; s < n2; ++s, ++sc) {
                     const int rs = sc % NR;
                     const int row = it.kv_start + s * kQS;
-                    ok = MW(mbar_wait<MPIPE_SLEEP_AUX>(&bars.qdo_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag));
+                    ok = mbar_wait<kSleepAux>(&bars.qdo_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
                     if (!ok) break;
                     mbar_expect_tx(&bars.qdo_full[rs], 2 * Cfg::kSub);
                     uint8_t* qd = smem + Cfg::kSmemQ + rs * Cfg::kSub;
@@ -263,7 +238,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             // of their own for them (S^T complete implies staged).  Folded: qdo_full completes only when the staging
             // warp has arrived too, so there is nothing more to wait for here.
             auto wait_stat = [&](uint32_t c) {
-                return Cfg::kStatFolded ? true : MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.stat_full[c % NS], (c / NS) & 1, &abort_flag));
+                return Cfg::kStatFolded ? true : mbar_wait(&bars.stat_full[c % NS], (c / NS) & 1, &abort_flag);
             };
             constexpr uint32_t idesc_s = umma_idesc_bf16(kBT, kQS, 0, 0);      // K-major x K-major, N = 64 queries
             constexpr uint32_t idesc_ts = umma_idesc_bf16(kBT, 64, 0, 1);      // A in TMEM, MN-major B, N = 64
@@ -313,16 +288,16 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 // With two K/V buffers the stream of sub-tiles runs on across the unit boundary: the S^T / dP^T MMAs
                 // of the next unit's first two sub-tiles are issued inside this unit's last two iterations, from
                 // the other (prefetched) buffer, so the softmax warps never see the pipeline drain between units.
-                constexpr bool kStream = (Cfg::kKVBufs == 2) && MPIPE_STREAM;
+                constexpr bool kStream = (Cfg::kKVBufs == 2);
                 const bool has_next = kStream && unit_of(ur + 1) < n_units;
                 const uint32_t kvb_n = sbase + (kb ^ 1) * (2 * Cfg::kTile);
                 const uint32_t k_lo_n = umma_desc_lo(kvb_n + Cfg::kSmemK, 0), v_lo_n = umma_desc_lo(kvb_n + Cfg::kSmemV, 0);
-                ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.kv_full[kb], (unit_it / Cfg::kKVBufs) & 1, &abort_flag));
+                ok = mbar_wait(&bars.kv_full[kb], (unit_it / Cfg::kKVBufs) & 1, &abort_flag);
                 if (!ok) break;
                 if (!kStream || unit_it == 0) {
                     for (int s = b0; s < 2; s += kStep) {   // prologue: S^T and dP^T of the first sub-tile of each stage served
                         const uint32_t c = sc + s;
-                        ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[c % NR], (c / NR) & 1, &abort_flag));
+                        ok = mbar_wait(&bars.qdo_full[c % NR], (c / NR) & 1, &abort_flag);
                         if (!ok) break;
                         ok = wait_stat(c);
                         if (!ok) break;
@@ -343,17 +318,15 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     const bool cross = (s + 2 >= n2) && has_next;   // sub-tile s+2 is the next unit's
                     const bool more = (s + 2 < n2) || cross;
                     const bool first = (s < 2);         // the stage's first sub-tile of the unit
-                    MPIPE_TR(0, c * 8 + 0);
-                    ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.p_full[b], ph, &abort_flag));
+                    ok = mbar_wait(&bars.p_full[b], ph, &abort_flag);
                     if (!ok) return false;
                     if (first && b == 0) {          // the accumulators are free: the previous unit's epilogue has read them
-                        ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag));
+                        ok = mbar_wait(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag);
                         if (!ok) return false;
                     } else if (first && kIssuers == 2) {   // ... and stage 0's overwriting dV MMA has been issued
-                        ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.acc_v, unit_it & 1, &abort_flag));
+                        ok = mbar_wait(&bars.acc_v, unit_it & 1, &abort_flag);
                         if (!ok) return false;
                     }
-                    MPIPE_TR(0, c * 8 + 1);
                     tc_fence_after();
                     issue_ts(Cfg::kColDV, Cfg::kColS + 64 * b, do_lo_of(c), !(first && b == 0));         // dV += P^T dO
                     if (first && b == 0 && kIssuers == 2) {
@@ -362,10 +335,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     }
                     if (more) {
                         if (cross && b == 0) {   // the next unit's K/V tiles (loaded while this unit ran)
-                            ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.kv_full[kb ^ 1], ((unit_it + 1) / Cfg::kKVBufs) & 1, &abort_flag));
+                            ok = mbar_wait(&bars.kv_full[kb ^ 1], ((unit_it + 1) / Cfg::kKVBufs) & 1, &abort_flag);
                             if (!ok) return false;
                         }
-                        ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.qdo_full[(c + 2) % NR], ((c + 2) / NR) & 1, &abort_flag));
+                        ok = mbar_wait(&bars.qdo_full[(c + 2) % NR], ((c + 2) / NR) & 1, &abort_flag);
                         if (!ok) return false;
                         ok = wait_stat(c + 2);
                         if (!ok) return false;
@@ -373,14 +346,12 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                         issue_kk(Cfg::kColS + 64 * b, cross ? k_lo_n : k_lo, kt_lo, q_lo_of(c + 2));       // S^T(s+2)
                         if (leader) umma_commit(&bars.s_full[b]);
                     }
-                    MPIPE_TR(0, c * 8 + 2);
-                    ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.ds_full[b], ph, &abort_flag));
+                    ok = mbar_wait(&bars.ds_full[b], ph, &abort_flag);
                     if (!ok) return false;
                     if (first && b == 1 && kIssuers == 2) {
-                        ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.acc_k, unit_it & 1, &abort_flag));
+                        ok = mbar_wait(&bars.acc_k, unit_it & 1, &abort_flag);
                         if (!ok) return false;
                     }
-                    MPIPE_TR(0, c * 8 + 3);
                     tc_fence_after();
                     issue_ts(Cfg::kColDK, Cfg::kColDP + 64 * b, q_lo_of(c), !(first && b == 0));          // dK += dS^T Q
                     if (first && b == 0 && kIssuers == 2) {
@@ -397,13 +368,12 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     }
                     if (b == 1) {                                                             // dQ of the 128-query pair
                         if (kIssuers == 2) {   // the other half of dS^T (a single issuer has already waited for it)
-                            ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.ds_full[0], ph, &abort_flag));
+                            ok = mbar_wait(&bars.ds_full[0], ph, &abort_flag);
                             if (!ok) return false;
                             if (leader) mbar_arrive(&bars.ds0_seen);   // lets stage 0's warpgroup complete the next phase
                         }
-                        ok = MW(mbar_wait<MPIPE_SLEEP_MMA>(&bars.dq_empty, ((c >> 1) & 1) ^ 1, &abort_flag));
+                        ok = mbar_wait(&bars.dq_empty, ((c >> 1) & 1) ^ 1, &abort_flag);
                         if (!ok) return false;
-                        MPIPE_TR(0, c * 8 + 4);
                         tc_fence_after();
                         if (leader) {
 #pragma unroll
@@ -416,7 +386,6 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                             umma_commit(&bars.dq_full[ph]);
                         }
                     }
-                    MPIPE_TR(0, c * 8 + 5);
                     return true;
                 };
                 if (kStep == 1) {
@@ -465,8 +434,8 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 }
                 // the stage is free when the MMAs that read the Q / dO sub-tile of four sub-tiles ago have completed
                 // (that commit follows the arrival of its dS^T, i.e. the softmax warps' last read of the stage)
-                ok = MW(mbar_wait<MPIPE_SLEEP_AUX>(Cfg::kStatFolded ? &bars.qdo_empty[rs] : &bars.stat_empty[rs],
-                                                   ((sc / NS) & 1) ^ 1, &abort_flag));
+                ok = mbar_wait<kSleepAux>(Cfg::kStatFolded ? &bars.qdo_empty[rs] : &bars.stat_empty[rs],
+                                                   ((sc / NS) & 1) ^ 1, &abort_flag);
                 if (!ok) break;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) dst[((e < 2) ? 0 : kQS) + lane + 32 * (e & 1)] = val[e];
@@ -502,11 +471,9 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 const float* stat = reinterpret_cast<const float*>(smem + Cfg::kSmemStat + rs * (2 * kQS * 4));
                 const float4* lse4 = reinterpret_cast<const float4*>(stat);
                 const float4* dl4 = reinterpret_cast<const float4*>(stat + kQS);
-                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 0);
                 // (the LSE / Delta stage was complete before this S^T was issued)
-                ok = MW(mbar_wait(&bars.s_full[g], ph, &abort_flag));
+                ok = mbar_wait(&bars.s_full[g], ph, &abort_flag);
                 if (!ok) break;
-                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 1);
                 tc_fence_after();
                 // P^T = exp2(S^T * scale*log2e - LSE*log2e): both 32-column halves are requested before the
                 // one wait; multiply-add on packed fp32 pairs
@@ -522,7 +489,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                         uint32_t pk[16];
 #pragma unroll
                         for (int c4 = 0; c4 < 8; ++c4) {
-                            const float4 l4 = MPIPE_DBG(4) ? make_float4(1.f, 1.f, 1.f, 1.f) : lse4[h * 8 + c4];
+                            const float4 l4 = lse4[h * 8 + c4];
                             const int e = h * 32 + 4 * c4;
                             const float2 x01 = fma2(make_float2(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), sc2,
                                                     make_float2(l4.x, l4.y));
@@ -538,22 +505,19 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                         tmem_st16(t_s + h * 16, pk);
                     }
                 }
-                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 6);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars.p_full[g]);
-                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 2);
 
-                ok = MW(mbar_wait(&bars.dp_full[g], ph, &abort_flag));
+                ok = mbar_wait(&bars.dp_full[g], ph, &abort_flag);
                 if (!ok) break;
                 // dS^T buffer (pair & 1) is free once dQ of pair - 2 has completed. With one issuing warp that is implied
                 // by s_full above (S^T(c) was issued, in order, after that dQ); with two it is waited for.
                 if (kIssuers == 2 && (c >> 1) >= 2) {
-                    ok = MW(mbar_wait(&bars.dq_full[ph], ((c >> 2) + 1) & 1, &abort_flag));
+                    ok = mbar_wait(&bars.dq_full[ph], ((c >> 2) + 1) & 1, &abort_flag);
                     if (!ok) break;
                 }
-                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 3);
                 tc_fence_after();
                 // dS^T = P^T o (dP^T - Delta); key rows past the segment are zeroed on the packed words
                 {
@@ -561,11 +525,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     tmem_ld32(t_dp, *reinterpret_cast<uint32_t(*)[32]>(&dr[0]));
                     tmem_ld32(t_dp + 32, *reinterpret_cast<uint32_t(*)[32]>(&dr[32]));
                     tmem_wait_ld();
-                    if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 7);
                     uint32_t pk[32];
 #pragma unroll
                     for (int c4 = 0; c4 < 16; ++c4) {
-                        const float4 d4 = MPIPE_DBG(4) ? make_float4(1.f, 1.f, 1.f, 1.f) : dl4[c4];
+                        const float4 d4 = dl4[c4];
                         const int e = 4 * c4;
                         const float2 t01 = add2(make_float2(__uint_as_float(dr[e]), __uint_as_float(dr[e + 1])),
                                                 make_float2(d4.x, d4.y));
@@ -580,13 +543,12 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) pk[i] = key_valid ? pk[i] : 0u;
                     }
-                    if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 5);
                     tmem_st16(t_dp, *reinterpret_cast<uint32_t(*)[16]>(&pk[0]));
                     tmem_st16(t_dp + 16, *reinterpret_cast<uint32_t(*)[16]>(&pk[16]));
                     // the same 64 values as 8 x 16 bytes of row r of the [key][q] tile (128-byte swizzle)
 #pragma unroll
                     for (int chunk = 0; chunk < 8; ++chunk) {
-                        if (!MPIPE_DBG(2)) *reinterpret_cast<uint4*>(ds_row + ph * Cfg::kDSBytes + ((chunk ^ (r & 7)) << 4)) =
+                        *reinterpret_cast<uint4*>(ds_row + ph * Cfg::kDSBytes + ((chunk ^ (r & 7)) << 4)) =
                             make_uint4(pk[4 * chunk], pk[4 * chunk + 1], pk[4 * chunk + 2], pk[4 * chunk + 3]);
                     }
                 }
@@ -597,11 +559,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 // With two issuing warps ds_full[0] has two consumers; the second (stage 1's issuer, before dQ) can lag, and
                 // a parity wait cannot tell phase n from n + 2: do not complete a phase before it has seen the last one.
                 if (kIssuers == 2 && g == 0 && (c >> 1) >= 1) {
-                    ok = MW(mbar_wait(&bars.ds0_seen, ((c >> 1) - 1) & 1, &abort_flag));
+                    ok = mbar_wait(&bars.ds0_seen, ((c >> 1) - 1) & 1, &abort_flag);
                     if (!ok) break;
                 }
                 if (lane == 0) mbar_arrive(&bars.ds_full[g]);
-                if (lane == 0 && (warp & 3) == 0) MPIPE_TR(1 + g, (c >> 1) * 8 + 4);
             }
             sc += n2;
         }
@@ -624,9 +585,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             // No early exit inside this loop: the four warps meet at named barriers, so after a time-out
             // they keep walking the (now empty) iterations together instead of leaving one another behind.
             for (int i = 0; i < npairs; ++i, ++pc) {
-                if (lane == 0 && warp == 12) MPIPE_TR(3, pc * 8 + 0);
-                if (ok) ok = MW(mbar_wait<MPIPE_SLEEP_AUX>(&bars.dq_full[pc & 1], (pc >> 1) & 1, &abort_flag));
-                if (lane == 0 && warp == 12) MPIPE_TR(3, pc * 8 + 1);
+                if (ok) ok = mbar_wait<kSleepAux>(&bars.dq_full[pc & 1], (pc >> 1) & 1, &abort_flag);
                 tc_fence_after();
                 uint8_t* stage = smem + Cfg::kSmemStage;
                 const int q0 = it.kv_start + i * kBT;
@@ -665,7 +624,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 }
                 fence_async_smem();
                 named_barrier_sync(1, 128);
-                if (ok && rt == 0 && !MPIPE_DBG(1)) {
+                if (ok && rt == 0 && it.seg >= 0) {
                     tma_reduce_add_3d(&maps.dq_acc, stage, 0, head, q0);
                     if (Cfg::kTail) tma_reduce_add_3d(&maps.dq_acc_tail, stage + Cfg::kStageMain, 64, head, q0);
                     bulk_commit_group();
@@ -681,16 +640,15 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 }
                 fence_async_smem();
                 named_barrier_sync(1, 128);
-                if (ok && rt == 0 && !MPIPE_DBG(1)) {
+                if (ok && rt == 0 && it.seg >= 0) {
                     tma_reduce_add_3d(&maps.dq_acc, stage, 32, head, q0);
                     bulk_commit_group();
                 }
-                if (lane == 0 && warp == 12) MPIPE_TR(3, pc * 8 + 2);
             }
-            if (ok) ok = MW(mbar_wait<MPIPE_SLEEP_AUX>(&bars.dkv_full, unit_it & 1, &abort_flag));
+            if (ok) ok = mbar_wait<kSleepAux>(&bars.dkv_full, unit_it & 1, &abort_flag);
             if (!ok) continue;   // keep walking the units so that the named barriers above stay matched
             tc_fence_after();
-            const bool store = r < it.row_len;
+            const bool store = r < it.row_len && it.seg >= 0;
             const int64_t tok = int64_t(it.row_start) + r;
             __nv_bfloat16* dv_row = p.dv + tok * p.tok_stride_g + int64_t(head) * p.head_stride_g;
             __nv_bfloat16* dk_row = p.dk + tok * p.tok_stride_g + int64_t(head) * p.head_stride_g;
@@ -816,9 +774,7 @@ static int32_t launch_bwd(const void* dout, const void* q, const void* k, const 
             !make_tensor_map_thd(&m.dq_acc_tail, dq_acc, total_tokens, n_heads, D, int64_t(n_heads) * D, D, 16, kBT, 64, 4))
             return MPIPE_ERR_CUDA;
     }
-    if (cudaFuncSetAttribute(attn_bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemAlloc) !=
-        cudaSuccess)
-        return MPIPE_ERR_CUDA;
+    if (!ensure_dynamic_smem<attn_bwd_kernel<D>>(Cfg::kSmemAlloc)) return MPIPE_ERR_CUDA;
     const int64_t rows = int64_t(total_tokens) * n_heads;
     const int64_t prepass_blocks = (rows + (D == 64 ? 32 : 16) - 1) / (D == 64 ? 32 : 16);
     const int64_t prepass_cap = int64_t(sm_count()) * 64;
@@ -843,17 +799,6 @@ static size_t round256(size_t x) { return (x + 255) & ~size_t(255); }
 
 extern "C" {
 
-#ifdef MPIPE_TRACE
-int32_t mpipe_dbg_set_flags(int32_t flags) {
-    return cudaMemcpyToSymbol(mpipe::g_dbg_flags, &flags, sizeof(int)) == cudaSuccess ? 0 : 1;
-}
-int32_t mpipe_dbg_read_where(int* host_out) {
-    return cudaMemcpyFromSymbol(host_out, mpipe::g_where, sizeof(int) * 16) == cudaSuccess ? 0 : 1;
-}
-int32_t mpipe_dbg_read_trace(long long* host_out) {
-    return cudaMemcpyFromSymbol(host_out, mpipe::g_trace, sizeof(long long) * 4 * 4096) == cudaSuccess ? 0 : 1;
-}
-#endif
 
 int32_t mpipe_bwd_tile_rows(void) { return mpipe::kBT; }
 
@@ -863,15 +808,17 @@ size_t mpipe_attn_workspace_bytes(int32_t total_tokens, int32_t n_heads, int32_t
            mpipe::round256(size_t(total_tokens) * n_heads * 4);
 }
 
-int32_t mpipe_varlen_attn_bwd(const void* dout, const void* q, const void* k, const void* v, const void* o,
-                              const float* lse, void* dq, void* dk, void* dv, int64_t tok_stride_qkv,
-                              int64_t head_stride_qkv, int64_t tok_stride_o, int64_t head_stride_o,
-                              int64_t tok_stride_grad, int64_t head_stride_grad, const int32_t* cu_seqlens_dev,
-                              int32_t n_seg, int32_t total_tokens, int32_t max_seqlen,
-                              const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items, int32_t n_heads,
-                              int32_t head_dim, float softmax_scale, int32_t mode, void* workspace,
-                              size_t workspace_bytes, int32_t* status_buf, void* stream) {
+namespace {
+// Argument checks shared by the two backward entry points.  Returns MPIPE_OK when the call may go on;
+// *nothing_to_do is set when it is complete without a launch (frozen encoder, no tokens, no items).
+int32_t bwd_check_args(const void* dout, const void* q, const void* k, const void* v, const void* o, const float* lse,
+                       const void* dq, const void* dk, const void* dv, int64_t tok_stride_qkv, int64_t head_stride_qkv,
+                       int64_t tok_stride_o, int64_t head_stride_o, int64_t tok_stride_grad, int64_t head_stride_grad,
+                       const int32_t* cu_seqlens_dev, int32_t n_seg, int32_t total_tokens, int32_t max_seqlen,
+                       const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items, int32_t n_heads, int32_t head_dim,
+                       float softmax_scale, int32_t mode, bool* nothing_to_do) {
     using namespace mpipe;
+    *nothing_to_do = true;
     if (mode != MPIPE_ENC_FROZEN && mode != MPIPE_ENC_TRAINED) return MPIPE_ERR_INVALID_ARG;
     if (mode == MPIPE_ENC_FROZEN) return MPIPE_OK;  // Lemma 1: a frozen encoder has no backward event
     if (n_seg < 0 || total_tokens < 0 || max_seqlen < 0 || n_bwd_items < 0 || n_heads <= 0) return MPIPE_ERR_INVALID_ARG;
@@ -891,6 +838,26 @@ int32_t mpipe_varlen_attn_bwd(const void* dout, const void* q, const void* k, co
         return MPIPE_ERR_INVALID_ARG;
     if (!(softmax_scale > 0.f) || !(softmax_scale < 1e30f)) return MPIPE_ERR_INVALID_ARG;
     if (int64_t(n_bwd_items) * n_heads >= (int64_t(1) << 31)) return MPIPE_ERR_INVALID_ARG;
+    *nothing_to_do = false;
+    return MPIPE_OK;
+}
+}  // namespace
+
+int32_t mpipe_varlen_attn_bwd(const void* dout, const void* q, const void* k, const void* v, const void* o,
+                              const float* lse, void* dq, void* dk, void* dv, int64_t tok_stride_qkv,
+                              int64_t head_stride_qkv, int64_t tok_stride_o, int64_t head_stride_o,
+                              int64_t tok_stride_grad, int64_t head_stride_grad, const int32_t* cu_seqlens_dev,
+                              int32_t n_seg, int32_t total_tokens, int32_t max_seqlen,
+                              const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items, int32_t n_heads,
+                              int32_t head_dim, float softmax_scale, int32_t mode, void* workspace,
+                              size_t workspace_bytes, int32_t* status_buf, void* stream) {
+    using namespace mpipe;
+    bool nothing_to_do = false;
+    const int32_t chk = bwd_check_args(dout, q, k, v, o, lse, dq, dk, dv, tok_stride_qkv, head_stride_qkv, tok_stride_o,
+                                       head_stride_o, tok_stride_grad, head_stride_grad, cu_seqlens_dev, n_seg,
+                                       total_tokens, max_seqlen, bwd_items_dev, n_bwd_items, n_heads, head_dim,
+                                       softmax_scale, mode, &nothing_to_do);
+    if (chk != MPIPE_OK || nothing_to_do) return chk;
     const size_t need = mpipe_attn_workspace_bytes(total_tokens, n_heads, head_dim, mode);
     if (workspace == nullptr || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
         return MPIPE_ERR_WORKSPACE;
@@ -932,7 +899,9 @@ constexpr size_t kStaticScratchBytes = size_t(32) << 20;
 static __device__ __align__(256) unsigned char g_bwd_static_scratch[kStaticScratchBytes];
 
 // Device address of the array, looked up once per device.  On the host the array's name is only a
-// stand-in symbol, not a device address, so kernels must be given the looked-up pointer.
+// stand-in symbol, not a device address, so kernels must be given the looked-up pointer.  The cache is
+// plain host memory without a lock: two host threads that make their first call on a device at the same
+// time both look the address up and store the same value.
 void* g_bwd_static_scratch_ptr[64] = {nullptr};
 
 int32_t static_scratch_for_current_device(void** out) {
@@ -962,9 +931,13 @@ int32_t mpipe_varlen_attn_bwd_static(const void* dout, const void* q, const void
                                      int32_t max_seqlen, const mpipe_work_item_t* bwd_items_dev, int32_t n_bwd_items,
                                      int32_t n_heads, int32_t head_dim, float softmax_scale, int32_t mode,
                                      int32_t* status_buf, void* stream) {
-    if (mode != MPIPE_ENC_FROZEN && mode != MPIPE_ENC_TRAINED) return MPIPE_ERR_INVALID_ARG;
-    if (mode == MPIPE_ENC_FROZEN) return MPIPE_OK;
-    if (total_tokens < 0 || n_heads <= 0 || head_dim <= 0) return MPIPE_ERR_INVALID_ARG;
+    // The same checks, in the same order, as mpipe_varlen_attn_bwd: a bad argument gets the same status from both.
+    bool nothing_to_do = false;
+    const int32_t chk = bwd_check_args(dout, q, k, v, o, lse, dq, dk, dv, tok_stride_qkv, head_stride_qkv, tok_stride_o,
+                                       head_stride_o, tok_stride_grad, head_stride_grad, cu_seqlens_dev, n_seg,
+                                       total_tokens, max_seqlen, bwd_items_dev, n_bwd_items, n_heads, head_dim,
+                                       softmax_scale, mode, &nothing_to_do);
+    if (chk != MPIPE_OK || nothing_to_do) return chk;
     // The problem must fit the built-in scratch; larger ones have to use mpipe_varlen_attn_bwd.
     if (mpipe_attn_workspace_bytes(total_tokens, n_heads, head_dim, mode) > kStaticScratchBytes)
         return MPIPE_ERR_WORKSPACE;

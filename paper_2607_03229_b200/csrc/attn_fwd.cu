@@ -28,10 +28,7 @@ constexpr int kFwdThreads = 384;
 constexpr int kTileM = 128;        // query rows per tile (= TMEM lanes)
 constexpr int kTileN = 128;        // keys per K/V tile
 constexpr float kRescaleThreshold = 8.0f;  // in log2 units
-#ifndef MPIPE_FWD_POLY_MASK
-#define MPIPE_FWD_POLY_MASK 0x52
-#endif
-constexpr unsigned kPolyMask = MPIPE_FWD_POLY_MASK;   // bit i: column pair i (mod 8) uses the polynomial exp2
+constexpr unsigned kPolyMask = 0x52;   // bit i: column pair i (mod 8) uses the polynomial exp2 (3 of 8)
 // setmaxnreg: the 4 light warps release what the 8 softmax warps take (an increase blocks until the CTA's
 // own pool has the registers).
 constexpr int kFwdRegsLaunch = 168, kFwdRegsLight = 56, kFwdRegsSoftmax = 224;
@@ -124,9 +121,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int g = int(gridDim.x), i = int(blockIdx.x);
         return round * g + ((round & 1) ? g - 1 - i : i);
     };
+    // Items are clamped to the tensors before use (see sanitize_item): a corrupt plan cannot make a store leave them.
     auto item_at = [&](int u) {
         mpipe_work_item_t z = {0, 0, 0, 0, 0, 0};
-        return (u < n_units) ? p.items[u / p.n_heads] : z;
+        if (u >= n_units) return z;
+        z = p.items[u / p.n_heads];
+        if (sanitize_item(z, 2 * kTileM, p.total_tokens) && tid == 4 * 32) report_status(p.status_buf, MPIPE_ERR_INDEX, u);
+        return z;
     };
 
     if (warp == 0) {
@@ -388,7 +389,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             ++ocnt;
             tc_fence_after();
             const float inv_l = 1.0f / l;
-            const bool store = r < rows_here;
+            const bool store = r < rows_here && it.seg >= 0;
             const int64_t tok = int64_t(it.row_start) + w * kTileM + r;
             __nv_bfloat16* orow = p.o + tok * p.tok_stride_o + int64_t(head) * p.head_stride_o;
 #pragma unroll
@@ -439,9 +440,7 @@ static int32_t launch_fwd(const void* q, const void* k, const void* v, int64_t t
             !make_tensor_map_thd(&mkt, k, total_tokens, n_heads, D, tok_stride, head_stride, 16, kTileN, 32))
             return MPIPE_ERR_CUDA;
     }
-    if (cudaFuncSetAttribute(attn_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemAlloc) !=
-        cudaSuccess)
-        return MPIPE_ERR_CUDA;
+    if (!ensure_dynamic_smem<attn_fwd_kernel<D>>(Cfg::kSmemAlloc)) return MPIPE_ERR_CUDA;
     const int n_units = prm.n_items * prm.n_heads;
     const int grid = n_units < sm_count() ? n_units : sm_count();
     profile_start(kProfileFwd, stream);

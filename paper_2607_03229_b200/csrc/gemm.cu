@@ -356,10 +356,10 @@ static int32_t launch_linear(int b_mode, const void* a, const void* w, const voi
     const int grid = int(tiles < sm_count() ? tiles : sm_count());
     profile_start(kProfileLinear, st);
     if (b_mode == 0) {
-        if (cudaFuncSetAttribute(linear_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem) != cudaSuccess) return MPIPE_ERR_CUDA;
+        if (!ensure_dynamic_smem<linear_kernel<0>>(kGemmSmem)) return MPIPE_ERR_CUDA;
         linear_kernel<0><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, p);
     } else {
-        if (cudaFuncSetAttribute(linear_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem) != cudaSuccess) return MPIPE_ERR_CUDA;
+        if (!ensure_dynamic_smem<linear_kernel<1>>(kGemmSmem)) return MPIPE_ERR_CUDA;
         linear_kernel<1><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, p);
     }
     profile_stop(kProfileLinear, st);
@@ -401,7 +401,7 @@ static int32_t launch_wgrad(const void* dy, const void* x, float* dw, int32_t to
     p.splits = best;
     const long long items = (long long)tiles * p.splits;
     const int grid = int(items < sms ? items : sms);
-    if (cudaFuncSetAttribute(linear_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem) != cudaSuccess) return MPIPE_ERR_CUDA;
+    if (!ensure_dynamic_smem<linear_kernel<2>>(kGemmSmem)) return MPIPE_ERR_CUDA;
     profile_start(kProfileLinear, st);
     linear_kernel<2><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, p);
     profile_stop(kProfileLinear, st);

@@ -6,7 +6,7 @@
 
 namespace mpipe {
 
-ProfileEvents g_profile[kProfileSlots];
+thread_local ProfileEvents g_profile[kProfileSlots];
 
 int sm_count() {
     static int cached[64] = {0};

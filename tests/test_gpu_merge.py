@@ -103,3 +103,56 @@ def test_merge_bwd_gathers_rows_and_frozen_is_a_noop():
     B.merge_tokens_bwd(to_dev(d_emb), d_enc, pos_d, B.TRAINED)
     torch.cuda.synchronize()
     assert np.array_equal(to_bits(d_enc), oracle.merge_tokens_bwd(d_emb, w.positions))
+
+
+@pytest.mark.parametrize("hidden,n_llm,n_enc", [(8, 5, 5), (24, 100, 37), (4096, 300, 111), (1280, 2049, 1000)])
+def test_merge_bwd_ragged_shapes(hidden, n_llm, n_enc):
+    d_emb = W.normal_bf16(15, 2, (n_llm, hidden))
+    pos = np.argsort(W.rand_u64(15, 3, n_llm), kind="stable")[:n_enc].astype(np.int32)
+    pad = 3
+    buf = torch.full((n_enc + 2 * pad, hidden), 7.0, dtype=torch.bfloat16, device="cuda")
+    st = status_buf()
+    B.merge_tokens_bwd(to_dev(d_emb), buf[pad:pad + n_enc], torch.from_numpy(pos).cuda(), B.TRAINED, st)
+    torch.cuda.synchronize()
+    assert int(st[0]) == 0
+    assert torch.all(buf[:pad] == 7.0) and torch.all(buf[pad + n_enc:] == 7.0), "canary rows overwritten"
+    assert np.array_equal(to_bits(buf[pad:pad + n_enc]), oracle.merge_tokens_bwd(d_emb, pos))
+
+
+def test_merge_bwd_strided_rows():
+    """Gradient rows read from, and written into, column blocks of wider buffers."""
+    d_emb_full = to_dev(W.normal_bf16(16, 2, (80, 768)))
+    d_enc_full = torch.full((50, 512), 7.0, dtype=torch.bfloat16, device="cuda")
+    d_emb, d_enc = d_emb_full[:, 256:512], d_enc_full[:, 128:384]
+    pos = np.argsort(W.rand_u64(16, 3, 80), kind="stable")[:50].astype(np.int32)
+    B.merge_tokens_bwd(d_emb, d_enc, torch.from_numpy(pos).cuda(), B.TRAINED)
+    torch.cuda.synchronize()
+    assert np.array_equal(to_bits(d_enc), oracle.merge_tokens_bwd(to_bits(d_emb), pos))
+    assert torch.all(d_enc_full[:, :128] == 7.0) and torch.all(d_enc_full[:, 384:] == 7.0)
+
+
+def test_merge_bwd_out_of_range_position_is_skipped_and_flagged():
+    d_emb = W.normal_bf16(17, 2, (10, 64))
+    pos = np.array([2, 10, 7, -1], dtype=np.int32)
+    d_enc = torch.full((4, 64), 7.0, dtype=torch.bfloat16, device="cuda")
+    st = status_buf()
+    B.merge_tokens_bwd(to_dev(d_emb), d_enc, torch.from_numpy(pos).cuda(), B.TRAINED, st)
+    torch.cuda.synchronize()
+    st = st.cpu().numpy()
+    assert st[0] == B.ERR_INDEX and st[1] in (1, 3)
+    got = to_bits(d_enc)
+    assert np.array_equal(got[0], d_emb[2]) and np.array_equal(got[2], d_emb[7])
+    assert torch.all(d_enc[1] == 7.0) and torch.all(d_enc[3] == 7.0)      # rows with no valid source stay untouched
+
+
+@pytest.mark.parametrize("fraction", [0.25, 0.75])
+def test_merge_bwd_modality_mix_full_size(fraction):
+    """The reverse seam at benchmark size: gradient rows of 8 x 8192 LLM tokens at hidden 4096 gathered back."""
+    w = W.modality_mix(fraction)
+    d_emb = w.llm_embeds()          # any bf16 matrix of the right shape stands for dL/d(embeddings)
+    d_enc = torch.empty((w.total_tokens, 4096), dtype=torch.bfloat16, device="cuda")
+    st = status_buf()
+    B.merge_tokens_bwd(to_dev(d_emb), d_enc, torch.from_numpy(w.positions).cuda(), B.TRAINED, st)
+    torch.cuda.synchronize()
+    assert int(st[0]) == 0
+    assert np.array_equal(to_bits(d_enc), oracle.merge_tokens_bwd(d_emb, w.positions))
