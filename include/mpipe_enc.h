@@ -260,10 +260,10 @@ int32_t mpipe_validate_positions(const int32_t* positions, int32_t n, int32_t n_
  *        layout [out, in], contiguous.  lse: fp32 [n_heads, n_tokens] when TRAINED, ignored when FROZEN.
  *        workspace: device, 256-byte aligned, >= mpipe_encoder_layer_workspace_bytes (MPIPE_ERR_WORKSPACE);
  *        caller-owned; after a TRAINED call it holds what mpipe_encoder_layer_bwd reads (see there), otherwise its contents are
- *        undefined afterwards.  The TRAINED forward rounds the MLP pre-activation to bf16 before the activation (it has to
- *        keep it), the FROZEN one applies the activation to the fp32 accumulator: the two outputs agree to bf16 rounding,
- *        not bit for bit.  Seven launches (eight with rope; one more when TRAINED: the activation is applied by a kernel of its own so that
- *        the pre-activation can be kept for the backward) on `stream`, no allocation, no sync.
+ *        undefined afterwards.  In both modes the activation is applied to the fp32 accumulator of the fc1 projection;
+ *        the TRAINED forward stores the pre-activation (bf16) from the same accumulator in the same launch, so y is
+ *        bit-identical in the two modes (Corollary 1: freezing changes nothing in the forward).  Seven launches (eight
+ *        with rope) on `stream`, no allocation, no sync.
  *        head_dim = hidden / n_heads must be one the attention kernels support (64, 80).
  * Device-side findings (a bounded wait that ran out) are reported through status_buf as for the attention calls.
  */

@@ -4,24 +4,35 @@
 // Three launches on the caller's stream:
 //   1. prepass   Delta[h,t] = sum_d dO[t,h,d] O[t,h,d]  and the fp32 dQ accumulator is cleared
 //   2. main      one persistent CTA per SM walks (key tile x head) units; a unit keeps one 128-key
-//                K/V tile resident and loops over the 128-row query tiles of the same segment
+//                K/V tile resident and steps through the 128-row query tiles of the same segment
 //   3. convert   dQ = softmax_scale * accumulator -> bf16
 //
-// Main kernel, per query tile i (everything transposed so that the key index is the TMEM lane):
-//   S^T  = K Q^T            tcgen05, operands in shared memory               -> TMEM
-//   dP^T = V dO^T           tcgen05                                           -> TMEM
-//   P^T  = exp2(S^T * scale*log2e - LSE*log2e)       softmax warps, written over S^T as bf16
+// Main kernel, per step = one [128 keys x 128 queries] block (everything transposed so that the key index is the
+// TMEM lane):
+//   S^T  = K Q^T            tcgen05, N = 128, operands in shared memory          -> TMEM (128 columns)
+//   dP^T = V dO^T           tcgen05, N = 128                                      -> TMEM (128 columns)
+//   P^T  = exp2(scale*log2e * (S^T - LSE/scale))     softmax warps, written over S^T as bf16
 //   dS^T = P^T o (dP^T - Delta)                      softmax warps, over dP^T as bf16 + to shared memory
-//   dV  += P^T dO           tcgen05, A operand read from TMEM, dO as MN-major B
+// The row terms -LSE_q / scale and -Delta_q are ADDED BY THE TENSOR CORE: each of the two score products runs one
+// more 16-element K-step whose key-side operand is a column of ones and whose query-side operand holds the term
+// split into three bf16 parts (24 bits, i.e. all of the fp32 value).  The softmax warps then need no per-query
+// value at all -- fetching 128 of them per thread and step from shared memory, whose port the operand reads of the
+// MMAs keep busy, was the largest single cost of a step (about a sixth of it).
+//   dV  += P^T dO           tcgen05, A operand read from TMEM, dO as MN-major B, N = head_dim
 //   dK  += dS^T Q           tcgen05, A operand read from TMEM, Q as MN-major B
 //   dQ_i = dS K             tcgen05, dS^T in shared memory read as an MN-major A, K as MN-major B
 // dQ_i is read back from TMEM by a reducer warpgroup, staged in shared memory and added to the global fp32
 // accumulator by the copy engine (cp.reduce.async.bulk.tensor, fp32 add): the order of those additions is not
 // fixed, so the low bits of dQ can differ from run to run.  dK (x softmax_scale) and dV leave TMEM once per unit.
 //
-// Warp roles (512 threads): 0 TMA producer, 1 / 3 tcgen05 issuers of TMEM stage 0 / 1, 2 TMEM allocation and
-// LSE/Delta staging, 4-7 / 8-11 softmax of stage 0 / 1, 12-15 dQ reducer and epilogue.
-// Every wait is bounded (see sm100_ptx.cuh); expiry sets status_buf and drains the CTA.
+// The block is as large as the TMEM budget allows (S^T 128 + dP^T 128 + dV, dK, dQ head_dim columns each) because
+// the kernel is bound by the NUMBER of tcgen05.mma instructions its one issuing thread gets through and by the
+// barrier hops between that thread and the softmax warps, not by the tensor pipe: a 128 x 128 step takes 32 MMAs
+// (34 at head_dim 80) and four hops; two 64-query half steps took 40 (68) and eight.
+//
+// Warp roles (512 threads): 0 TMA producer, 1 tcgen05 issuer, 2 TMEM allocation and LSE/Delta staging, 4-11 softmax
+// (thread = key row; warps 4-7 take query columns 0-63 of the block, warps 8-11 columns 64-127), 12-15 dQ reducer
+// and epilogue.  Every wait is bounded (see sm100_ptx.cuh); expiry sets status_buf and drains the CTA.
 #include <cuda.h>
 #include <math_constants.h>
 #include "common.h"
@@ -39,40 +50,47 @@ constexpr int kRegsLaunch = 128, kRegsService = 72, kRegsReducer = 96, kRegsSoft
 static_assert(4 * (kRegsLaunch - kRegsService) + 4 * (kRegsLaunch - kRegsReducer) >= 8 * (kRegsSoftmax - kRegsLaunch),
               "setmaxnreg pool arithmetic");
 constexpr int kBT = 128;  // keys per unit = TMEM lanes
-constexpr int kQS = 64;   // query rows per sub-tile (one pipeline stage of S^T / dP^T)
+constexpr int kBQ = 128;  // query rows per step
+constexpr int kQH = 64;   // query columns of a step handled by one softmax warpgroup
 
+// Shared-memory layout of a [128 rows x head_dim] bf16 tile.  head_dim 64: one TMA box, rows of 128 bytes, 128-byte
+// swizzle.  head_dim 80: three boxes of 32 elements (rows of 64 bytes, 64-byte swizzle) 8 KB apart, the last one half
+// beyond the tensor and zero-filled by TMA; with a single swizzle mode over the whole row a tile serves as a K-major
+// operand (five 16-element K-steps) and, as an MN-major operand, as ONE N = 80 operand (two and a half 32-element
+// atoms) -- a 64 + 16 split needs two MMA instructions for every product over the head dimension.
 template <int D>
 struct BwdCfg {
-    static constexpr int kTail = D - 64;
-    static constexpr int kTileMain = kBT * 128;                 // K, V: [128 rows][64 bf16], 128-byte swizzle
-    static constexpr int kTileTail = kTail ? kBT * 32 : 0;      //       [128 rows][16 bf16], 32-byte swizzle
-    static constexpr int kTile = kTileMain + kTileTail;
-    static constexpr int kSubMain = kQS * 128;                  // Q, dO sub-tiles: [64 rows][64 bf16]
-    static constexpr int kSubTail = kTail ? kQS * 32 : 0;
-    static constexpr int kSub = kSubMain + kSubTail;
-    static constexpr int kRing = 4;                             // Q/dO sub-tile stages
-    // Issuing warps: two (one per TMEM stage) decouple the warpgroups and gain ~10 % at D = 80; at D = 64 a single
-    // in-order issuer measured ~3 % faster (and keeps dK/dV bit-reproducible), so that is what D = 64 uses.
-    static constexpr int kIssuers = (D == 64) ? 1 : 2;
-    static constexpr int kKVBufs = (D == 64) ? 2 : 1;           // D = 64: the next unit's K/V tiles load during the current unit
-    // LSE / Delta stages.  One issuing warp: they travel with the Q / dO stages (same ring, same full / empty barriers:
-    // the issuer has no waits to spare).  Two issuing warps: a ring of 8 with barriers of its own, staged far ahead.
-    static constexpr bool kStatFolded = (kIssuers == 1);
-    static constexpr int kStatRing = kStatFolded ? kRing : 8;
-    // dQ staging for the TMA reduction: one [128 q][32 fp32] box (used twice per pair) + the 16-column tail box
-    static constexpr int kStageMain = kBT * 128;
-    static constexpr int kStageBytes = kStageMain + (kTail ? kBT * 64 : 0);
-    static constexpr int kSmemK = 0;                            // buffer i at kSmemK + i * 2 * kTile (K then V)
+    static constexpr int kBoxElems = (D == 64) ? 64 : 32;
+    static constexpr int kBoxes = (D == 64) ? 1 : 3;
+    static constexpr int kRowBytes = kBoxElems * 2;
+    static constexpr int kBoxBytes = 128 * kRowBytes;             // 16 KB / 8 KB
+    static constexpr int kTile = kBoxes * kBoxBytes;              // K, V, Q, dO tiles: 16 KB / 24 KB
+    static constexpr uint32_t kSwz = (D == 64) ? kSwizzle128 : kSwizzle64;
+    static constexpr uint32_t kSBO = 8 * kRowBytes;               // 8 rows of one box
+    static constexpr int kKSteps = D / 16;                        // K-steps of a product over the head dimension
+    static constexpr int kKVBufs = (D == 64) ? 2 : 1;             // 2: the next unit's K/V tiles load during the current unit
+    static constexpr int kRing = 2;                               // Q / dO / row-term stages
+    // One more 16-element K-step carries the per-query row terms into the two score products (see the staging warp):
+    // [128 rows][32 bytes] operands, 32-byte swizzle.
+    static constexpr int kExtra = 128 * 32;
+    // dQ staging for the TMA reduction: 16 fp32 columns at a time through three rotating [128 q][16 fp32] boxes
+    // (rows of 64 bytes, 64-byte swizzle), so that the copy engine reads two boxes while the third is being filled
+    static constexpr int kStageBox = kBQ * 64;
+    static constexpr int kStageBoxes = 3;
+    static constexpr int kStageBytes = kStageBoxes * kStageBox;
+    static constexpr int kSmemK = 0;                              // buffer i at i * 2 * kTile (K then V)
     static constexpr int kSmemV = kTile;
     static constexpr int kSmemQ = kKVBufs * 2 * kTile;
-    static constexpr int kSmemDO = kSmemQ + kRing * kSub;
-    static constexpr int kDSBytes = 2 * kBT * 128;              // dS^T of a pair as [key][q]: two 64-query atoms of 16 KB
-    static constexpr int kSmemDS = kSmemDO + kRing * kSub;      // two of them: pair j writes buffer j & 1 while dQ(j-1) reads the other
-    static constexpr int kSmemStage = kSmemDS + 2 * kDSBytes;
-    static constexpr int kSmemStat = kSmemStage + kStageBytes;  // kStatRing x (LSE[64], Delta[64]) fp32
-    static constexpr int kSmemTotal = kSmemStat + kStatRing * 2 * kQS * 4;
+    static constexpr int kSmemDO = kSmemQ + kRing * kTile;
+    static constexpr int kDSBytes = 2 * kBT * 128;                // dS^T of a step as [key][q]: two 64-query atoms of 16 KB
+    static constexpr int kSmemDS = kSmemDO + kRing * kTile;
+    static constexpr int kSmemStage = kSmemDS + kDSBytes;
+    static constexpr int kSmemOnes = kSmemStage + kStageBytes;    // the key-side operand of the extra K-step (constant)
+    static constexpr int kSmemQX = kSmemOnes + kExtra;            // kRing x query-side operand for S^T (-LSE / softmax_scale)
+    static constexpr int kSmemDOX = kSmemQX + kRing * kExtra;     // kRing x query-side operand for dP^T (-Delta)
+    static constexpr int kSmemTotal = kSmemDOX + kRing * kExtra;
     static constexpr int kSmemAlloc = kSmemTotal + 1024;
-    // TMEM columns: S^T stage b at 64*b, dP^T stage b at 128 + 64*b (P^T / dS^T overlay their first 32 columns)
+    // TMEM columns; P^T / dS^T (bf16) overlay the first 32 columns of each warpgroup's 64-column half of S^T / dP^T
     static constexpr int kColS = 0, kColDP = 128, kColDV = 256, kColDK = 256 + D, kColDQ = 256 + 2 * D;
     static_assert(kSmemAlloc <= 227 * 1024, "shared memory budget");
     static_assert(kColDQ + D <= 512, "TMEM budget");
@@ -90,13 +108,13 @@ struct BwdParams {
 };
 
 struct BwdBarriers {
-    uint64_t kv_full[2], kv_empty[2], dkv_full, dkv_empty, acc_v, acc_k;
-    uint64_t qdo_full[4], qdo_empty[4], stat_full[8], stat_empty[8];
-    uint64_t s_full[2], p_full[2], dp_full[2], ds_full[2], dq_full[2], dq_empty, ds0_seen;
+    uint64_t kv_full[2], kv_empty[2], dkv_full, dkv_empty;
+    uint64_t qdo_full[4], qdo_empty[4];
+    uint64_t s_full, p_full, dp_full, ds_full, dq_full, dq_empty;
 };
 
 struct BwdMaps {
-    CUtensorMap q, k, v, dout, q_tail, k_tail, v_tail, dout_tail, dq_acc, dq_acc_tail;
+    CUtensorMap q, k, v, dout, dq_acc;
 };
 
 template <int D>
@@ -104,8 +122,6 @@ __global__ void __maxnreg__(kRegsLaunch)
 attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
     using Cfg = BwdCfg<D>;
     constexpr int NR = Cfg::kRing;
-    constexpr int NS = Cfg::kStatRing;
-    constexpr int kIssuers = Cfg::kIssuers;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ BwdBarriers bars;
@@ -120,35 +136,33 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         abort_flag = 0;
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars.kv_full[i], 1);
-            mbar_init(&bars.kv_empty[i], kIssuers);   // one commit from each issuing warp
+            mbar_init(&bars.kv_empty[i], 1);
         }
-        mbar_init(&bars.acc_v, 1);
-        mbar_init(&bars.acc_k, 1);
-        mbar_init(&bars.dkv_full, kIssuers);
+        mbar_init(&bars.dkv_full, 1);
         mbar_init(&bars.dkv_empty, 4);
         for (int s = 0; s < 4; ++s) {
-            mbar_init(&bars.qdo_full[s], Cfg::kStatFolded ? 2 : 1);   // the producer's expect_tx arrival (+ the staging warp)
+            mbar_init(&bars.qdo_full[s], 2);    // the producer's expect_tx arrival + the staging warp
             mbar_init(&bars.qdo_empty[s], 1);
         }
-        for (int s = 0; s < 8; ++s) {
-            mbar_init(&bars.stat_full[s], 1);
-            mbar_init(&bars.stat_empty[s], 1);   // released by the issuing warp once the sub-tile's dS^T has arrived
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(&bars.s_full[b], 1);
-            mbar_init(&bars.p_full[b], 4);
-            mbar_init(&bars.dp_full[b], 1);
-            mbar_init(&bars.ds_full[b], 4);
-        }
-        mbar_init(&bars.ds0_seen, 1);
-        mbar_init(&bars.dq_full[0], 1);
-        mbar_init(&bars.dq_full[1], 1);
-        mbar_init(&bars.dq_empty, 4);
+        mbar_init(&bars.s_full, 1);
+        mbar_init(&bars.p_full, 8);             // one arrival per softmax warp
+        mbar_init(&bars.dp_full, 1);
+        mbar_init(&bars.ds_full, 8);
+        mbar_init(&bars.dq_full, 1);
+        mbar_init(&bars.dq_empty, 4);           // one arrival per reducer warp
         fence_mbar_init();
     }
     if (warp == 2) {
         tmem_alloc(&tmem_base_slot, 512);
         tmem_relinquish();
+    }
+    if (tid >= 128 && tid < 256) {
+        // Key-side operand of the extra K-step: every row is (1, 1, 1, 0 x 5 | 1, 1, 1, 0 x 5).  The query-side rows carry
+        // their three parts in the first 16-byte half only and zeros in the second, so the dot product is the sum of
+        // the three parts whichever way the 32-byte swizzle orders a row's two halves.
+        uint4* row = reinterpret_cast<uint4*>(smem + Cfg::kSmemOnes + (tid - 128) * 32);
+        row[0] = row[1] = make_uint4(0x3F803F80u, 0x00003F80u, 0u, 0u);
+        fence_async_smem();
     }
     tc_fence_before();
     __syncthreads();
@@ -163,16 +177,17 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
     };
     // Items are clamped to the tensors before use (see sanitize_item): a corrupt plan cannot make a store, a
     // reduction or an LSE / Delta read leave them.
-    auto item_at = [&](int u) {
+    auto item_at = [&](int u) {   // the raw item, loaded one unit ahead of its use
         mpipe_work_item_t z = {0, 0, 0, 0, 0, 0};
-        if (u >= n_units) return z;
-        z = p.items[u / p.n_heads];
+        return (u < n_units) ? p.items[u / p.n_heads] : z;
+    };
+    auto checked = [&](mpipe_work_item_t z, int u) {   // clamped at the point of use, so that the load stays off the critical path
         if (sanitize_item(z, kBT, p.total_tokens) && tid == 12 * 32) report_status(p.status_buf, MPIPE_ERR_INDEX, u);
         return z;
     };
-    // Every unit runs an even number of 64-query sub-tiles (a 128-query tile is two of them); a padding
-    // sub-tile past the segment end contributes nothing because its probabilities are forced to zero.
-    auto subtiles_of = [](const mpipe_work_item_t& it) { return 2 * ((it.kv_len + kBT - 1) / kBT); };
+    // Steps of a unit: the 128-query tiles of the segment; rows of the last one past the segment end contribute
+    // nothing because their probabilities are forced to zero.
+    auto steps_of = [](const mpipe_work_item_t& it) { return (it.kv_len + kBQ - 1) / kBQ; };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -180,303 +195,244 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         if (lane == 0) {
             uint32_t unit_it = 0, sc = 0;
             bool ok = true;
+            auto load_tile = [&](uint8_t* dst, const CUtensorMap* map, uint64_t* bar, int head, int row) {
+#pragma unroll
+                for (int bx = 0; bx < Cfg::kBoxes; ++bx)
+                    tma_load_3d(dst + bx * Cfg::kBoxBytes, map, bar, bx * Cfg::kBoxElems, head, row);
+            };
             mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
-                const mpipe_work_item_t it = it_next;
+                const mpipe_work_item_t it = checked(it_next, u);
                 it_next = item_at(unit_of(ur + 1));
                 const int head = u % p.n_heads;
-                const int n2 = subtiles_of(it);
+                const int nq = steps_of(it);
                 const int kb = unit_it % Cfg::kKVBufs;            // K/V buffer of this unit
                 uint8_t* kv = smem + kb * (2 * Cfg::kTile);
                 ok = mbar_wait<kSleepAux>(&bars.kv_empty[kb], ((unit_it / Cfg::kKVBufs) & 1) ^ 1, &abort_flag);
                 if (!ok) break;
                 mbar_expect_tx(&bars.kv_full[kb], 2 * Cfg::kTile);
-                tma_load_3d(kv + Cfg::kSmemK, &maps.k, &bars.kv_full[kb], 0, head, it.row_start);
-                tma_load_3d(kv + Cfg::kSmemV, &maps.v, &bars.kv_full[kb], 0, head, it.row_start);
-                if (Cfg::kTail) {
-                    tma_load_3d(kv + Cfg::kSmemK + Cfg::kTileMain, &maps.k_tail, &bars.kv_full[kb], 64, head, it.row_start);
-                    tma_load_3d(kv + Cfg::kSmemV + Cfg::kTileMain, &maps.v_tail, &bars.kv_full[kb], 64, head, it.row_start);
-                }
-                for (int s = 0; s < n2; ++s, ++sc) {
+                load_tile(kv + Cfg::kSmemK, &maps.k, &bars.kv_full[kb], head, it.row_start);
+                load_tile(kv + Cfg::kSmemV, &maps.v, &bars.kv_full[kb], head, it.row_start);
+                for (int j = 0; j < nq; ++j, ++sc) {
                     const int rs = sc % NR;
-                    const int row = it.kv_start + s * kQS;
+                    const int row = it.kv_start + j * kBQ;
                     ok = mbar_wait<kSleepAux>(&bars.qdo_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
                     if (!ok) break;
-                    mbar_expect_tx(&bars.qdo_full[rs], 2 * Cfg::kSub);
-                    uint8_t* qd = smem + Cfg::kSmemQ + rs * Cfg::kSub;
-                    uint8_t* dd = smem + Cfg::kSmemDO + rs * Cfg::kSub;
-                    tma_load_3d(qd, &maps.q, &bars.qdo_full[rs], 0, head, row);
-                    tma_load_3d(dd, &maps.dout, &bars.qdo_full[rs], 0, head, row);
-                    if (Cfg::kTail) {
-                        tma_load_3d(qd + Cfg::kSubMain, &maps.q_tail, &bars.qdo_full[rs], 64, head, row);
-                        tma_load_3d(dd + Cfg::kSubMain, &maps.dout_tail, &bars.qdo_full[rs], 64, head, row);
-                    }
+                    mbar_expect_tx(&bars.qdo_full[rs], 2 * Cfg::kTile);
+                    load_tile(smem + Cfg::kSmemQ + rs * Cfg::kTile, &maps.q, &bars.qdo_full[rs], head, row);
+                    load_tile(smem + Cfg::kSmemDO + rs * Cfg::kTile, &maps.dout, &bars.qdo_full[rs], head, row);
                 }
             }
         }
         __syncwarp();
-    } else if (warp == 1 || (warp == 3 && kIssuers == 2)) {
-        // ------------------------------------------------------------------ tcgen05 issuers
-        // One issuing warp per TMEM stage (warp 1: even sub-tiles, warp 3: odd sub-tiles), so that neither
-        // warpgroup's MMAs wait behind the other's slowest step; a barrier hop costs ~200 cycles (~340 when it
-        // starts from a tcgen05.commit), and a single in-order issuer made every one of them serial.
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ tcgen05 issuer
         // The whole warp walks the loop (uniform control flow); one elected lane issues and commits.
         // Descriptors are precomputed halves: a K-step only adds a constant to the low word.
-        // Cross-warp ordering on the tensor pipe is needed in two places only: the first (overwriting) dV / dK
-        // MMA of a unit comes from stage 0 and must precede stage 1's first accumulation (acc_v / acc_k), and
-        // the pair's dQ MMA (issued by stage 1) needs both stages' dS^T in shared memory (ds_full[0]).
+        // Issue order per step j:  dV(j), S^T(j+1) | dK(j), dQ(j), dP^T(j+1).  S^T(j+1) goes out as soon as the P^T that
+        // overlays S^T(j) has been consumed, so that the softmax warps find it ready when they return from dS^T(j).
         setmaxnreg_dec<kRegsService>();
         {
-            const int b0 = (kIssuers == 2) ? (warp >> 1) : 0;   // first TMEM stage served by this warp
-            constexpr int kStep = (kIssuers == 2) ? 2 : 1;      // two issuers: every other sub-tile; one: all, in order
             const bool leader = elect_one();
             const uint32_t sbase = smem_u32(smem);
-            constexpr uint32_t hi128 = umma_desc_hi(1024, kSwizzle128);
-            constexpr uint32_t hi32 = umma_desc_hi(256, kSwizzle32);
+            constexpr uint32_t hi_t = umma_desc_hi(Cfg::kSBO, Cfg::kSwz);      // Q / K / V / dO tiles
+            constexpr uint32_t hi128 = umma_desc_hi(1024, kSwizzle128);        // the dS^T tile
+            constexpr uint32_t idesc_s = umma_idesc_bf16(kBT, kBQ, 0, 0);      // K-major x K-major, N = 128 queries
+            constexpr uint32_t idesc_ts = umma_idesc_bf16(kBT, D, 0, 1);       // A in TMEM, MN-major B, N = head_dim
+            constexpr uint32_t idesc_dq = umma_idesc_bf16(kBQ, D, 1, 1);       // MN-major A and B
+            // low descriptor words (16-byte units).  K-major use of a tile: K-step ks starts (ks % per_box) * 32 bytes into
+            // box ks / per_box.  MN-major use: rows are the contraction index, 16 rows per K-step; LBO = box stride.
+            constexpr uint32_t kPerBox = Cfg::kBoxElems / 16;
+            auto kmaj = [&](uint32_t lo, int ks) { return lo + uint32_t(ks / kPerBox) * (Cfg::kBoxBytes >> 4) + uint32_t(ks % kPerBox) * 2; };
+            constexpr uint32_t kMnStep = (16 * Cfg::kRowBytes) >> 4;
             const uint32_t ds_lo = umma_desc_lo(sbase + Cfg::kSmemDS, kBT * 128);   // two 64-query atoms 16 KB apart
-            // LSE / Delta of a sub-tile must be staged before its S^T is issued: the softmax warps then need no barrier
-            // of their own for them (S^T complete implies staged).  Folded: qdo_full completes only when the staging
-            // warp has arrived too, so there is nothing more to wait for here.
-            auto wait_stat = [&](uint32_t c) {
-                return Cfg::kStatFolded ? true : mbar_wait(&bars.stat_full[c % NS], (c / NS) & 1, &abort_flag);
-            };
-            constexpr uint32_t idesc_s = umma_idesc_bf16(kBT, kQS, 0, 0);      // K-major x K-major, N = 64 queries
-            constexpr uint32_t idesc_ts = umma_idesc_bf16(kBT, 64, 0, 1);      // A in TMEM, MN-major B, N = 64
-            constexpr uint32_t idesc_ts_t = umma_idesc_bf16(kBT, 16, 0, 1);    // same, 16-wide head-dim tail
-            constexpr uint32_t idesc_dq = umma_idesc_bf16(kBT, 64, 1, 1);      // MN-major A and B
-            constexpr uint32_t idesc_dq_t = umma_idesc_bf16(kBT, 16, 1, 1);
-            constexpr uint32_t kSubTailOff = Cfg::kSubMain >> 4;
-            // descriptor low words of the ring's Q / dO stages: base + stage * (stage bytes / 16); no carry out of the 14
-            // address bits as long as the stage lies in shared memory
             const uint32_t q_lo0 = umma_desc_lo(sbase + Cfg::kSmemQ, 0), do_lo0 = umma_desc_lo(sbase + Cfg::kSmemDO, 0);
-            auto q_lo_of = [&](uint32_t c) { return q_lo0 + (c % NR) * uint32_t(Cfg::kSub >> 4); };
-            auto do_lo_of = [&](uint32_t c) { return do_lo0 + (c % NR) * uint32_t(Cfg::kSub >> 4); };
-            // dst[128 keys x 64 q] = A[128 x D] * B[64 x D]^T, both K-major (main 64 columns + optional 16 tail)
-            auto issue_kk = [&](uint32_t dcol, uint32_t a, uint32_t at, uint32_t bq) {
+            const uint32_t q_mn0 = umma_desc_lo(sbase + Cfg::kSmemQ, Cfg::kBoxBytes), do_mn0 = umma_desc_lo(sbase + Cfg::kSmemDO, Cfg::kBoxBytes);
+            auto stage_off = [&](uint32_t c) { return (c % NR) * uint32_t(Cfg::kTile >> 4); };
+            constexpr uint32_t hi32 = umma_desc_hi(256, kSwizzle32);           // the extra K-step's operands
+            const uint32_t ones_lo = umma_desc_lo(sbase + Cfg::kSmemOnes, 0);
+            const uint32_t qx_lo0 = umma_desc_lo(sbase + Cfg::kSmemQX, 0), dox_lo0 = umma_desc_lo(sbase + Cfg::kSmemDOX, 0);
+            auto extra_off = [&](uint32_t c) { return (c % NR) * uint32_t(Cfg::kExtra >> 4); };
+            // dst[128 keys x 128 q] = A[128 x D] * B[128 x D]^T + 1 * x[q]: both K-major, then the row-term K-step
+            auto issue_kk = [&](uint32_t dcol, uint32_t a_lo, uint32_t b_lo, uint32_t x_lo) {
                 if (leader) {
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        umma_ss(tmem + dcol, umma_desc(a + ks * 2, hi128), umma_desc(bq + ks * 2, hi128), idesc_s, ks > 0);
-                    if (Cfg::kTail) umma_ss(tmem + dcol, umma_desc(at, hi32), umma_desc(bq + kSubTailOff, hi32), idesc_s, 1);
+                    for (int ks = 0; ks < Cfg::kKSteps; ++ks)
+                        umma_ss(tmem + dcol, umma_desc(kmaj(a_lo, ks), hi_t), umma_desc(kmaj(b_lo, ks), hi_t), idesc_s, ks > 0);
+                    umma_ss(tmem + dcol, umma_desc(ones_lo, hi32), umma_desc(x_lo, hi32), idesc_s, 1);
                 }
             };
-            // dst[128 keys x D] (+)= A^T-in-TMEM[128 keys x 64 q] * B[64 q x D] (B rows = q, MN-major)
-            auto issue_ts = [&](uint32_t dcol, uint32_t acol, uint32_t bq, bool acc) {
+            // dst[128 keys x D] (+)= A^T-in-TMEM[128 keys x 128 q] * B[128 q x D] (B rows = q, MN-major)
+            auto issue_ts = [&](uint32_t dcol, uint32_t acol, uint32_t b_mn, bool acc) {
                 if (leader) {
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        umma_ts(tmem + dcol, tmem + acol + ks * 8, umma_desc(bq + ks * 128, hi128), idesc_ts,
+                    for (int ks = 0; ks < kBQ / 16; ++ks)
+                        umma_ts(tmem + dcol, tmem + acol + (ks >> 2) * kQH + (ks & 3) * 8, umma_desc(b_mn + ks * kMnStep, hi_t), idesc_ts,
                                 (acc || ks > 0) ? 1u : 0u);
-                        if (Cfg::kTail)
-                            umma_ts(tmem + dcol + 64, tmem + acol + ks * 8, umma_desc(bq + kSubTailOff + ks * 32, hi32),
-                                    idesc_ts_t, (acc || ks > 0) ? 1u : 0u);
-                    }
                 }
             };
-            uint32_t unit_it = 0, sc = 0;   // sc: global sub-tile counter at the start of the unit (even)
+            uint32_t unit_it = 0, sc = 0;   // sc: global step counter at the start of the unit
             bool ok = true;
             mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
-                const mpipe_work_item_t it = it_next;
+                const mpipe_work_item_t it = checked(it_next, u);
                 it_next = item_at(unit_of(ur + 1));
-                const int n2 = subtiles_of(it);
+                const int nq = steps_of(it);
                 const int kb = unit_it % Cfg::kKVBufs;
                 const uint32_t kvb = sbase + kb * (2 * Cfg::kTile);
                 const uint32_t k_lo = umma_desc_lo(kvb + Cfg::kSmemK, 0), v_lo = umma_desc_lo(kvb + Cfg::kSmemV, 0);
-                const uint32_t kt_lo = umma_desc_lo(kvb + Cfg::kSmemK + Cfg::kTileMain, 0);
-                const uint32_t vt_lo = umma_desc_lo(kvb + Cfg::kSmemV + Cfg::kTileMain, 0);
-                // With two K/V buffers the stream of sub-tiles runs on across the unit boundary: the S^T / dP^T MMAs
-                // of the next unit's first two sub-tiles are issued inside this unit's last two iterations, from
-                // the other (prefetched) buffer, so the softmax warps never see the pipeline drain between units.
+                const uint32_t k_mn = umma_desc_lo(kvb + Cfg::kSmemK, Cfg::kBoxBytes);
+                // With two K/V buffers the stream of steps runs on across the unit boundary: S^T / dP^T of the next unit's
+                // first step are issued inside this unit's last step, from the other (prefetched) buffer, so the softmax
+                // warps never see the pipeline drain between units.
                 constexpr bool kStream = (Cfg::kKVBufs == 2);
                 const bool has_next = kStream && unit_of(ur + 1) < n_units;
                 const uint32_t kvb_n = sbase + (kb ^ 1) * (2 * Cfg::kTile);
                 const uint32_t k_lo_n = umma_desc_lo(kvb_n + Cfg::kSmemK, 0), v_lo_n = umma_desc_lo(kvb_n + Cfg::kSmemV, 0);
                 ok = mbar_wait(&bars.kv_full[kb], (unit_it / Cfg::kKVBufs) & 1, &abort_flag);
                 if (!ok) break;
-                if (!kStream || unit_it == 0) {
-                    for (int s = b0; s < 2; s += kStep) {   // prologue: S^T and dP^T of the first sub-tile of each stage served
-                        const uint32_t c = sc + s;
-                        ok = mbar_wait(&bars.qdo_full[c % NR], (c / NR) & 1, &abort_flag);
-                        if (!ok) break;
-                        ok = wait_stat(c);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_kk(Cfg::kColS + 64 * s, k_lo, kt_lo, q_lo_of(c));
-                        if (leader) umma_commit(&bars.s_full[s]);
-                        issue_kk(Cfg::kColDP + 64 * s, v_lo, vt_lo, do_lo_of(c));
-                        if (leader) umma_commit(&bars.dp_full[s]);
-                    }
+                if (!kStream || unit_it == 0) {   // prologue: S^T and dP^T of the unit's first step
+                    ok = mbar_wait(&bars.qdo_full[sc % NR], (sc / NR) & 1, &abort_flag);
                     if (!ok) break;
+                    tc_fence_after();
+                    issue_kk(Cfg::kColS, k_lo, q_lo0 + stage_off(sc), qx_lo0 + extra_off(sc));
+                    if (leader) umma_commit(&bars.s_full);
+                    issue_kk(Cfg::kColDP, v_lo, do_lo0 + stage_off(sc), dox_lo0 + extra_off(sc));
+                    if (leader) umma_commit(&bars.dp_full);
                 }
-                // One sub-tile of the issue order.  The TMEM stage b is a compile-time constant (the loop below is unrolled
-                // over the two stages), so stage offsets and barrier addresses fold into immediates.
-                auto sub_tile = [&](const int s, auto stage) -> bool {
-                    constexpr int b = decltype(stage)::value;
-                    const uint32_t c = sc + s;
-                    const uint32_t ph = (c >> 1) & 1;   // phase of the per-stage barriers
-                    const bool cross = (s + 2 >= n2) && has_next;   // sub-tile s+2 is the next unit's
-                    const bool more = (s + 2 < n2) || cross;
-                    const bool first = (s < 2);         // the stage's first sub-tile of the unit
-                    ok = mbar_wait(&bars.p_full[b], ph, &abort_flag);
-                    if (!ok) return false;
-                    if (first && b == 0) {          // the accumulators are free: the previous unit's epilogue has read them
+                for (int j = 0; j < nq && ok; ++j) {
+                    const uint32_t c = sc + j;
+                    const uint32_t ph = c & 1;
+                    const bool cross = (j + 1 == nq) && has_next;   // step j+1 is the next unit's first
+                    const bool more = (j + 1 < nq) || cross;
+                    ok = mbar_wait(&bars.p_full, ph, &abort_flag);
+                    if (!ok) break;
+                    if (j == 0) {   // the accumulators are free: the previous unit's epilogue has read them
                         ok = mbar_wait(&bars.dkv_empty, (unit_it & 1) ^ 1, &abort_flag);
-                        if (!ok) return false;
-                    } else if (first && kIssuers == 2) {   // ... and stage 0's overwriting dV MMA has been issued
-                        ok = mbar_wait(&bars.acc_v, unit_it & 1, &abort_flag);
-                        if (!ok) return false;
+                        if (!ok) break;
                     }
                     tc_fence_after();
-                    issue_ts(Cfg::kColDV, Cfg::kColS + 64 * b, do_lo_of(c), !(first && b == 0));         // dV += P^T dO
-                    if (first && b == 0 && kIssuers == 2) {
-                        tc_fence_before();
-                        if (leader) mbar_arrive(&bars.acc_v);
-                    }
+                    issue_ts(Cfg::kColDV, Cfg::kColS, do_mn0 + stage_off(c), j > 0);                              // dV += P^T dO
                     if (more) {
-                        if (cross && b == 0) {   // the next unit's K/V tiles (loaded while this unit ran)
+                        if (cross) {   // the next unit's K/V tiles (loaded while this unit ran)
                             ok = mbar_wait(&bars.kv_full[kb ^ 1], ((unit_it + 1) / Cfg::kKVBufs) & 1, &abort_flag);
-                            if (!ok) return false;
+                            if (!ok) break;
                         }
-                        ok = mbar_wait(&bars.qdo_full[(c + 2) % NR], ((c + 2) / NR) & 1, &abort_flag);
-                        if (!ok) return false;
-                        ok = wait_stat(c + 2);
-                        if (!ok) return false;
+                        ok = mbar_wait(&bars.qdo_full[(c + 1) % NR], ((c + 1) / NR) & 1, &abort_flag);
+                        if (!ok) break;
                         tc_fence_after();
-                        issue_kk(Cfg::kColS + 64 * b, cross ? k_lo_n : k_lo, kt_lo, q_lo_of(c + 2));       // S^T(s+2)
-                        if (leader) umma_commit(&bars.s_full[b]);
+                        issue_kk(Cfg::kColS, cross ? k_lo_n : k_lo, q_lo0 + stage_off(c + 1), qx_lo0 + extra_off(c + 1));                    // S^T(j+1)
+                        if (leader) umma_commit(&bars.s_full);
                     }
-                    ok = mbar_wait(&bars.ds_full[b], ph, &abort_flag);
-                    if (!ok) return false;
-                    if (first && b == 1 && kIssuers == 2) {
-                        ok = mbar_wait(&bars.acc_k, unit_it & 1, &abort_flag);
-                        if (!ok) return false;
-                    }
+                    ok = mbar_wait(&bars.ds_full, ph, &abort_flag);
+                    if (!ok) break;
                     tc_fence_after();
-                    issue_ts(Cfg::kColDK, Cfg::kColDP + 64 * b, q_lo_of(c), !(first && b == 0));          // dK += dS^T Q
-                    if (first && b == 0 && kIssuers == 2) {
-                        tc_fence_before();
-                        if (leader) mbar_arrive(&bars.acc_k);
-                    }
-                    if (leader) {
-                        umma_commit(&bars.qdo_empty[c % NR]);   // folded: also frees the LSE / Delta stage (dS^T(c) has arrived)
-                        if (!Cfg::kStatFolded) mbar_arrive(&bars.stat_empty[c % NS]);
-                    }
-                    if (more) {
-                        issue_kk(Cfg::kColDP + 64 * b, cross ? v_lo_n : v_lo, vt_lo, do_lo_of(c + 2));    // dP^T(s+2)
-                        if (leader) umma_commit(&bars.dp_full[b]);
-                    }
-                    if (b == 1) {                                                             // dQ of the 128-query pair
-                        if (kIssuers == 2) {   // the other half of dS^T (a single issuer has already waited for it)
-                            ok = mbar_wait(&bars.ds_full[0], ph, &abort_flag);
-                            if (!ok) return false;
-                            if (leader) mbar_arrive(&bars.ds0_seen);   // lets stage 0's warpgroup complete the next phase
-                        }
-                        ok = mbar_wait(&bars.dq_empty, ((c >> 1) & 1) ^ 1, &abort_flag);
-                        if (!ok) return false;
-                        tc_fence_after();
-                        if (leader) {
+                    issue_ts(Cfg::kColDK, Cfg::kColDP, q_mn0 + stage_off(c), j > 0);                              // dK += dS^T Q
+                    if (leader) umma_commit(&bars.qdo_empty[c % NR]);   // also frees the LSE / Delta stage (dS^T(j) has arrived)
+                    ok = mbar_wait(&bars.dq_empty, ph ^ 1, &abort_flag);   // the reducer has taken dQ(j-1) out of TMEM
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (leader) {                                                                                 // dQ(j) = dS K
 #pragma unroll
-                            for (int ks = 0; ks < 8; ++ks) {
-                                const uint64_t adesc = umma_desc(ds_lo + ph * (Cfg::kDSBytes >> 4) + ks * 128, hi128);
-                                umma_ss(tmem + Cfg::kColDQ, adesc, umma_desc(k_lo + ks * 128, hi128), idesc_dq, ks > 0);
-                                if (Cfg::kTail)
-                                    umma_ss(tmem + Cfg::kColDQ + 64, adesc, umma_desc(kt_lo + ks * 32, hi32), idesc_dq_t, ks > 0);
-                            }
-                            umma_commit(&bars.dq_full[ph]);
-                        }
+                        for (int ks = 0; ks < kBT / 16; ++ks)
+                            umma_ss(tmem + Cfg::kColDQ, umma_desc(ds_lo + ks * 128, hi128), umma_desc(k_mn + ks * kMnStep, hi_t), idesc_dq, ks > 0);
+                        umma_commit(&bars.dq_full);
                     }
-                    return true;
-                };
-                if (kStep == 1) {
-                    for (int s = 0; s < n2 && ok; s += 2) {
-                        ok = sub_tile(s, std::integral_constant<int, 0>{});
-                        if (ok) ok = sub_tile(s + 1, std::integral_constant<int, 1>{});
+                    if (more) {   // after dQ(j): its completion then implies that the dS^T tile in shared memory has been read
+                        issue_kk(Cfg::kColDP, cross ? v_lo_n : v_lo, do_lo0 + stage_off(c + 1), dox_lo0 + extra_off(c + 1));   // dP^T(j+1)
+                        if (leader) umma_commit(&bars.dp_full);
                     }
-                } else {
-                    for (int s = b0; s < n2 && ok; s += 2)
-                        ok = (b0 == 0) ? sub_tile(s, std::integral_constant<int, 0>{}) : sub_tile(s, std::integral_constant<int, 1>{});
                 }
                 if (!ok) break;
                 if (leader) umma_commit(&bars.dkv_full);
                 if (leader) umma_commit(&bars.kv_empty[kb]);
-                sc += n2;
+                sc += nq;
             }
         }
         __syncwarp();
     } else if (warp == 2) {
-        // ------------------------------------------------------------------ LSE / Delta staging
+        // ------------------------------------------------------------------ row-term staging
+        // Per step and query q: x_q = -LSE_q / softmax_scale and y_q = -Delta_q, each split into three bf16 parts
+        // (hi, then the remainder, then its remainder: together the fp32 value), written as the first three elements
+        // of row q of the step's two extra-K-step operands.  Query rows past the segment end get a hugely negative x
+        // (their probabilities become exp2(-large) = 0) and y = 0.
         setmaxnreg_dec<kRegsService>();
         uint32_t sc = 0;
         bool ok = true;
+        const float inv_scale = 1.0f / p.scale;
+        auto split3 = [](float a) {
+            const __nv_bfloat16 h = __float2bfloat16_rn(a);
+            const float r1 = a - __bfloat162float(h);
+            const __nv_bfloat16 m = __float2bfloat16_rn(r1);
+            const __nv_bfloat16 l = __float2bfloat16_rn(r1 - __bfloat162float(m));
+            return make_uint4(uint32_t(__bfloat16_as_ushort(h)) | (uint32_t(__bfloat16_as_ushort(m)) << 16),
+                              uint32_t(__bfloat16_as_ushort(l)), 0u, 0u);
+        };
         mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
         for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
-            const mpipe_work_item_t it = it_next;
+            const mpipe_work_item_t it = checked(it_next, u);
             it_next = item_at(unit_of(ur + 1));
             const int head = u % p.n_heads;
-            const int n2 = subtiles_of(it);
+            const int nq = steps_of(it);
             const int q_end = it.kv_start + it.kv_len;
-            for (int s = 0; s < n2; ++s, ++sc) {
-                const int rs = sc % NS;
-                float* dst = reinterpret_cast<float*>(smem + Cfg::kSmemStat + rs * (2 * kQS * 4));
-                const int q0 = it.kv_start + s * kQS;
-                float val[4];   // read from global memory before the stage is known to be free: the latency overlaps the wait
+            for (int j = 0; j < nq; ++j, ++sc) {
+                const int rs = sc % NR;
+                uint4* qx = reinterpret_cast<uint4*>(smem + Cfg::kSmemQX + rs * Cfg::kExtra);
+                uint4* dox = reinterpret_cast<uint4*>(smem + Cfg::kSmemDOX + rs * Cfg::kExtra);
+                const int q0 = it.kv_start + j * kBQ;
+                float xv[4], yv[4];   // read from global memory before the stage is known to be free: the latency overlaps the wait
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {   // e = 0, 1: -LSE*log2e of 64 query columns; e = 2, 3: -Delta
-                    const bool is_lse = (e < 2);
-                    const int q = q0 + lane + 32 * (e & 1);
-                    if (q < q_end) {   // stored negated: what the softmax warps add
-                        val[e] = -__ldg((is_lse ? p.lse : p.delta) + int64_t(head) * p.total_tokens + q);
-                        if (is_lse) val[e] *= 1.4426950408889634f;
-                    } else {
-                        val[e] = is_lse ? -CUDART_INF_F : 0.f;  // P = exp2(-inf) = 0 for query columns past the segment
-                    }
+                for (int e = 0; e < 4; ++e) {
+                    const int q = q0 + lane + 32 * e;
+                    const bool valid = q < q_end;
+                    xv[e] = valid ? -__ldg(p.lse + int64_t(head) * p.total_tokens + q) * inv_scale : -3.0e38f;
+                    yv[e] = valid ? -__ldg(p.delta + int64_t(head) * p.total_tokens + q) : 0.f;
                 }
-                // the stage is free when the MMAs that read the Q / dO sub-tile of four sub-tiles ago have completed
-                // (that commit follows the arrival of its dS^T, i.e. the softmax warps' last read of the stage)
-                ok = mbar_wait<kSleepAux>(Cfg::kStatFolded ? &bars.qdo_empty[rs] : &bars.stat_empty[rs],
-                                                   ((sc / NS) & 1) ^ 1, &abort_flag);
+                // the stage is free when the MMAs that read the Q / dO tile it travels with have completed
+                ok = mbar_wait<kSleepAux>(&bars.qdo_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
                 if (!ok) break;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) dst[((e < 2) ? 0 : kQS) + lane + 32 * (e & 1)] = val[e];
+                for (int e = 0; e < 4; ++e) {
+                    const int row = lane + 32 * e;
+                    qx[2 * row] = split3(xv[e]);
+                    qx[2 * row + 1] = make_uint4(0u, 0u, 0u, 0u);
+                    dox[2 * row] = split3(yv[e]);
+                    dox[2 * row + 1] = make_uint4(0u, 0u, 0u, 0u);
+                }
+                fence_async_smem();   // generic-proxy writes, read by the tensor core
                 __syncwarp();
-                if (lane == 0) mbar_arrive(Cfg::kStatFolded ? &bars.qdo_full[rs] : &bars.stat_full[rs]);
+                if (lane == 0) mbar_arrive(&bars.qdo_full[rs]);
             }
         }
     } else if (warp == 3) {
-        setmaxnreg_dec<kRegsService>();   // spare warp when one issuer is enough
+        setmaxnreg_dec<kRegsService>();   // spare warp
     } else if (warp < 12) {
         // ------------------------------------------------------------------ softmax / dS warps
-        // Warpgroup g owns TMEM stage g, i.e. every other 64-query sub-tile; thread = key row.
+        // Thread = key row; warpgroup g takes query columns [64 g, 64 g + 64) of every step.
         setmaxnreg_inc<kRegsSoftmax>();
         const int g = (warp - 4) >> 2;
         const int r = ((warp & 3) << 5) | lane;
         const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
-        const uint32_t t_s = tmem + lane_base + Cfg::kColS + g * 64;
-        const uint32_t t_dp = tmem + lane_base + Cfg::kColDP + g * 64;
+        const uint32_t t_s = tmem + lane_base + Cfg::kColS + g * kQH;
+        const uint32_t t_dp = tmem + lane_base + Cfg::kColDP + g * kQH;
         uint8_t* ds_row = smem + Cfg::kSmemDS + g * (kBT * 128) + r * 128;
-        uint32_t sc = 0;   // global sub-tile counter at the start of the unit (always even)
+        uint32_t sc = 0;   // global step counter at the start of the unit
         bool ok = true;
         mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
         for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
-            const mpipe_work_item_t it = it_next;
+            const mpipe_work_item_t it = checked(it_next, u);
             it_next = item_at(unit_of(ur + 1));
-            const int n2 = subtiles_of(it);
+            const int nq = steps_of(it);
             const bool key_valid = r < it.row_len;
             const bool ragged_keys = it.row_len < kBT;
-            for (int s = g; s < n2; s += 2) {
-                const uint32_t c = sc + s;
-                const int rs = c % NS;
-                const uint32_t ph = (c >> 1) & 1;   // phase of the per-stage barriers = dS^T buffer of the pair
-                const float* stat = reinterpret_cast<const float*>(smem + Cfg::kSmemStat + rs * (2 * kQS * 4));
-                const float4* lse4 = reinterpret_cast<const float4*>(stat);
-                const float4* dl4 = reinterpret_cast<const float4*>(stat + kQS);
-                // (the LSE / Delta stage was complete before this S^T was issued)
-                ok = mbar_wait(&bars.s_full[g], ph, &abort_flag);
+            for (int j = 0; j < nq; ++j) {
+                const uint32_t c = sc + j;
+                const uint32_t ph = c & 1;
+                ok = mbar_wait(&bars.s_full, ph, &abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                // P^T = exp2(S^T * scale*log2e - LSE*log2e): both 32-column halves are requested before the
-                // one wait; multiply-add on packed fp32 pairs
+                // P^T = exp2(scale*log2e * S'^T), S' already holding the row term: both 32-column halves are requested
+                // before the one wait; packed fp32 pairs for the multiply
                 float pr[64];
                 {
                     uint32_t sr[64];
@@ -489,12 +445,9 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                         uint32_t pk[16];
 #pragma unroll
                         for (int c4 = 0; c4 < 8; ++c4) {
-                            const float4 l4 = lse4[h * 8 + c4];
                             const int e = h * 32 + 4 * c4;
-                            const float2 x01 = fma2(make_float2(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), sc2,
-                                                    make_float2(l4.x, l4.y));
-                            const float2 x23 = fma2(make_float2(__uint_as_float(sr[e + 2]), __uint_as_float(sr[e + 3])), sc2,
-                                                    make_float2(l4.z, l4.w));
+                            const float2 x01 = mul2(make_float2(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1])), sc2);
+                            const float2 x23 = mul2(make_float2(__uint_as_float(sr[e + 2]), __uint_as_float(sr[e + 3])), sc2);
                             pr[e] = ex2_approx(x01.x);
                             pr[e + 1] = ex2_approx(x01.y);
                             pr[e + 2] = ex2_approx(x23.x);
@@ -502,24 +455,20 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                             pk[2 * c4] = pack_bf16(pr[e], pr[e + 1]);
                             pk[2 * c4 + 1] = pack_bf16(pr[e + 2], pr[e + 3]);
                         }
-                        tmem_st16(t_s + h * 16, pk);
+                        tmem_st16(t_s + h * 16, pk);   // over this thread's own scores, which are in registers
                     }
                 }
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bars.p_full[g]);
+                if (lane == 0) mbar_arrive(&bars.p_full);
 
-                ok = mbar_wait(&bars.dp_full[g], ph, &abort_flag);
+                // dP^T(j) complete also means dQ(j-1) has completed (issued before it, same thread): the dS^T tile in
+                // shared memory may be overwritten
+                ok = mbar_wait(&bars.dp_full, ph, &abort_flag);
                 if (!ok) break;
-                // dS^T buffer (pair & 1) is free once dQ of pair - 2 has completed. With one issuing warp that is implied
-                // by s_full above (S^T(c) was issued, in order, after that dQ); with two it is waited for.
-                if (kIssuers == 2 && (c >> 1) >= 2) {
-                    ok = mbar_wait(&bars.dq_full[ph], ((c >> 2) + 1) & 1, &abort_flag);
-                    if (!ok) break;
-                }
                 tc_fence_after();
-                // dS^T = P^T o (dP^T - Delta); key rows past the segment are zeroed on the packed words
+                // dS^T = P^T o dP'^T (dP' already holding -Delta); key rows past the segment are zeroed on the packed words
                 {
                     uint32_t dr[64];
                     tmem_ld32(t_dp, *reinterpret_cast<uint32_t(*)[32]>(&dr[0]));
@@ -528,14 +477,9 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     uint32_t pk[32];
 #pragma unroll
                     for (int c4 = 0; c4 < 16; ++c4) {
-                        const float4 d4 = dl4[c4];
                         const int e = 4 * c4;
-                        const float2 t01 = add2(make_float2(__uint_as_float(dr[e]), __uint_as_float(dr[e + 1])),
-                                                make_float2(d4.x, d4.y));
-                        const float2 t23 = add2(make_float2(__uint_as_float(dr[e + 2]), __uint_as_float(dr[e + 3])),
-                                                make_float2(d4.z, d4.w));
-                        const float2 s01 = mul2(make_float2(pr[e], pr[e + 1]), t01);
-                        const float2 s23 = mul2(make_float2(pr[e + 2], pr[e + 3]), t23);
+                        const float2 s01 = mul2(make_float2(pr[e], pr[e + 1]), make_float2(__uint_as_float(dr[e]), __uint_as_float(dr[e + 1])));
+                        const float2 s23 = mul2(make_float2(pr[e + 2], pr[e + 3]), make_float2(__uint_as_float(dr[e + 2]), __uint_as_float(dr[e + 3])));
                         pk[2 * c4] = pack_bf16(s01.x, s01.y);
                         pk[2 * c4 + 1] = pack_bf16(s23.x, s23.y);
                     }
@@ -545,10 +489,10 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     }
                     tmem_st16(t_dp, *reinterpret_cast<uint32_t(*)[16]>(&pk[0]));
                     tmem_st16(t_dp + 16, *reinterpret_cast<uint32_t(*)[16]>(&pk[16]));
-                    // the same 64 values as 8 x 16 bytes of row r of the [key][q] tile (128-byte swizzle)
+                    // the same 64 values as 8 x 16 bytes of row r of this warpgroup's [key][64 q] atom (128-byte swizzle)
 #pragma unroll
                     for (int chunk = 0; chunk < 8; ++chunk) {
-                        *reinterpret_cast<uint4*>(ds_row + ph * Cfg::kDSBytes + ((chunk ^ (r & 7)) << 4)) =
+                        *reinterpret_cast<uint4*>(ds_row + ((chunk ^ (r & 7)) << 4)) =
                             make_uint4(pk[4 * chunk], pk[4 * chunk + 1], pk[4 * chunk + 2], pk[4 * chunk + 3]);
                     }
                 }
@@ -556,93 +500,60 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 fence_async_smem();
                 tc_fence_before();
                 __syncwarp();
-                // With two issuing warps ds_full[0] has two consumers; the second (stage 1's issuer, before dQ) can lag, and
-                // a parity wait cannot tell phase n from n + 2: do not complete a phase before it has seen the last one.
-                if (kIssuers == 2 && g == 0 && (c >> 1) >= 1) {
-                    ok = mbar_wait(&bars.ds0_seen, ((c >> 1) - 1) & 1, &abort_flag);
-                    if (!ok) break;
-                }
-                if (lane == 0) mbar_arrive(&bars.ds_full[g]);
+                if (lane == 0) mbar_arrive(&bars.ds_full);
             }
-            sc += n2;
+            sc += nq;
         }
     } else {
         // ------------------------------------------------------------------ dQ reducer + dK/dV epilogue
-        // dQ of a 128-query pair: TMEM -> registers -> swizzled staging in shared memory -> one TMA
-        // reduce-add per 32 fp32 columns into the global accumulator (the copy engine does the atomics).
+        // dQ of a step: TMEM -> registers -> swizzled staging in shared memory -> one TMA reduce-add per 16 fp32
+        // columns into the global accumulator (the copy engine does the atomics).
         setmaxnreg_dec<kRegsReducer>();
         const int r = ((warp & 3) << 5) | lane;
         const int rt = tid - 12 * 32;   // 0..127 inside the warpgroup
         const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
-        uint32_t pc = 0, unit_it = 0;   // pair counter
+        uint32_t pc = 0, gc = 0, unit_it = 0;   // step counter, staging-chunk counter
         bool ok = true;
         mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
         for (int ur = 0, u = unit_of(0); u < n_units; ++ur, u = unit_of(ur), ++unit_it) {
-            const mpipe_work_item_t it = it_next;
+            const mpipe_work_item_t it = checked(it_next, u);
             it_next = item_at(unit_of(ur + 1));
             const int head = u % p.n_heads;
-            const int npairs = (it.kv_len + kBT - 1) / kBT;
+            const int nq = steps_of(it);
             // No early exit inside this loop: the four warps meet at named barriers, so after a time-out
             // they keep walking the (now empty) iterations together instead of leaving one another behind.
-            for (int i = 0; i < npairs; ++i, ++pc) {
-                if (ok) ok = mbar_wait<kSleepAux>(&bars.dq_full[pc & 1], (pc >> 1) & 1, &abort_flag);
+            for (int i = 0; i < nq; ++i, ++pc) {
+                if (ok) ok = mbar_wait<kSleepAux>(&bars.dq_full, pc & 1, &abort_flag);
                 tc_fence_after();
-                uint8_t* stage = smem + Cfg::kSmemStage;
-                const int q0 = it.kv_start + i * kBT;
-                // Two steps through one [128 rows][128 B] staging box (128-byte swizzle): columns 0..31, then 32..63; the
-                // D = 80 tail (columns 64..79, [128 rows][64 B], 64-byte swizzle) rides with the first step. The second
-                // half leaves TMEM before the first is handed to the copy engine, so the next pair's dQ MMA can start.
-                if (rt == 0) bulk_wait_group_read<0>();   // the box must have been read before it is overwritten
-                named_barrier_sync(1, 128);
-                uint32_t v1[2][16];
-                if (ok) {
-                    uint32_t v0[2][16];
-                    tmem_ld16(tmem + lane_base + Cfg::kColDQ, v0[0]);
-                    tmem_ld16(tmem + lane_base + Cfg::kColDQ + 16, v0[1]);
-                    tmem_wait_ld();
+                const int q0 = it.kv_start + i * kBQ;
+                // One round per 16 columns: read them from TMEM, write this thread's 64-byte row of box gc % 3, and
+                // after the warpgroup's barrier hand the box to the copy engine.  Box gc % 3 was last used three rounds
+                // ago; before each barrier the issuing thread waits until at most ONE reduction is still reading its
+                // box, so the box of the next round is free when the barrier opens -- one barrier per round.
 #pragma unroll
-                    for (int chunk = 0; chunk < 8; ++chunk)
-                        *reinterpret_cast<uint4*>(stage + r * 128 + ((chunk ^ (r & 7)) << 4)) =
-                            make_uint4(v0[chunk / 4][4 * (chunk & 3)], v0[chunk / 4][4 * (chunk & 3) + 1],
-                                       v0[chunk / 4][4 * (chunk & 3) + 2], v0[chunk / 4][4 * (chunk & 3) + 3]);
-                    tmem_ld16(tmem + lane_base + Cfg::kColDQ + 32, v1[0]);
-                    tmem_ld16(tmem + lane_base + Cfg::kColDQ + 48, v1[1]);
-                    if (Cfg::kTail) {
-                        uint32_t vt[16];
-                        tmem_ld16(tmem + lane_base + Cfg::kColDQ + 64, vt);
+                for (int ch = 0; ch < D / 16; ++ch, ++gc) {
+                    uint8_t* box = smem + Cfg::kSmemStage + (gc % Cfg::kStageBoxes) * Cfg::kStageBox;
+                    if (ok) {
+                        uint32_t v[16];
+                        tmem_ld16(tmem + lane_base + Cfg::kColDQ + 16 * ch, v);
                         tmem_wait_ld();
+                        if (ch == D / 16 - 1) {   // the whole row has left TMEM: the next step's dQ may be issued
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&bars.dq_empty);
+                        }
 #pragma unroll
-                        for (int chunk = 0; chunk < 4; ++chunk)
-                            *reinterpret_cast<uint4*>(stage + Cfg::kStageMain + r * 64 + ((chunk ^ ((r >> 1) & 3)) << 4)) =
-                                make_uint4(vt[4 * chunk], vt[4 * chunk + 1], vt[4 * chunk + 2], vt[4 * chunk + 3]);
-                    } else {
-                        tmem_wait_ld();
+                        for (int c4 = 0; c4 < 4; ++c4)
+                            *reinterpret_cast<uint4*>(box + r * 64 + ((c4 ^ ((r >> 1) & 3)) << 4)) =
+                                make_uint4(v[4 * c4], v[4 * c4 + 1], v[4 * c4 + 2], v[4 * c4 + 3]);
                     }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars.dq_empty);   // the whole row has left TMEM
-                }
-                fence_async_smem();
-                named_barrier_sync(1, 128);
-                if (ok && rt == 0 && it.seg >= 0) {
-                    tma_reduce_add_3d(&maps.dq_acc, stage, 0, head, q0);
-                    if (Cfg::kTail) tma_reduce_add_3d(&maps.dq_acc_tail, stage + Cfg::kStageMain, 64, head, q0);
-                    bulk_commit_group();
-                }
-                if (rt == 0) bulk_wait_group_read<0>();
-                named_barrier_sync(1, 128);
-                if (ok) {
-#pragma unroll
-                    for (int chunk = 0; chunk < 8; ++chunk)
-                        *reinterpret_cast<uint4*>(stage + r * 128 + ((chunk ^ (r & 7)) << 4)) =
-                            make_uint4(v1[chunk / 4][4 * (chunk & 3)], v1[chunk / 4][4 * (chunk & 3) + 1],
-                                       v1[chunk / 4][4 * (chunk & 3) + 2], v1[chunk / 4][4 * (chunk & 3) + 3]);
-                }
-                fence_async_smem();
-                named_barrier_sync(1, 128);
-                if (ok && rt == 0 && it.seg >= 0) {
-                    tma_reduce_add_3d(&maps.dq_acc, stage, 32, head, q0);
-                    bulk_commit_group();
+                    fence_async_smem();
+                    if (rt == 0) bulk_wait_group_read<1>();
+                    named_barrier_sync(1, 128);
+                    if (rt == 0) {
+                        if (ok && it.seg >= 0) tma_reduce_add_3d(&maps.dq_acc, box, 16 * ch, head, q0);
+                        bulk_commit_group();   // (an empty group when nothing was issued keeps the round count in step)
+                    }
                 }
             }
             if (ok) ok = mbar_wait<kSleepAux>(&bars.dkv_full, unit_it & 1, &abort_flag);
@@ -759,21 +670,14 @@ static int32_t launch_bwd(const void* dout, const void* q, const void* k, const 
                           int32_t n_heads, BwdParams prm, float* delta, float* dq_acc, cudaStream_t stream) {
     using Cfg = BwdCfg<D>;
     BwdMaps m;
-    if (!make_tensor_map_thd(&m.q, q, total_tokens, n_heads, D, ts_qkv, hs_qkv, 64, kQS, 128) ||
-        !make_tensor_map_thd(&m.k, k, total_tokens, n_heads, D, ts_qkv, hs_qkv, 64, kBT, 128) ||
-        !make_tensor_map_thd(&m.v, v, total_tokens, n_heads, D, ts_qkv, hs_qkv, 64, kBT, 128) ||
-        !make_tensor_map_thd(&m.dout, dout, total_tokens, n_heads, D, ts_o, hs_o, 64, kQS, 128) ||
-        !make_tensor_map_thd(&m.dq_acc, dq_acc, total_tokens, n_heads, D, int64_t(n_heads) * D, D, 32, kBT, 128, 4))
+    constexpr uint32_t box = Cfg::kBoxElems;
+    constexpr int swz = Cfg::kRowBytes;
+    if (!make_tensor_map_thd(&m.q, q, total_tokens, n_heads, D, ts_qkv, hs_qkv, box, kBQ, swz) ||
+        !make_tensor_map_thd(&m.k, k, total_tokens, n_heads, D, ts_qkv, hs_qkv, box, kBT, swz) ||
+        !make_tensor_map_thd(&m.v, v, total_tokens, n_heads, D, ts_qkv, hs_qkv, box, kBT, swz) ||
+        !make_tensor_map_thd(&m.dout, dout, total_tokens, n_heads, D, ts_o, hs_o, box, kBQ, swz) ||
+        !make_tensor_map_thd(&m.dq_acc, dq_acc, total_tokens, n_heads, D, int64_t(n_heads) * D, D, 16, kBQ, 64, 4))
         return MPIPE_ERR_CUDA;
-    m.q_tail = m.q, m.k_tail = m.k, m.v_tail = m.v, m.dout_tail = m.dout, m.dq_acc_tail = m.dq_acc;
-    if (Cfg::kTail) {
-        if (!make_tensor_map_thd(&m.q_tail, q, total_tokens, n_heads, D, ts_qkv, hs_qkv, 16, kQS, 32) ||
-            !make_tensor_map_thd(&m.k_tail, k, total_tokens, n_heads, D, ts_qkv, hs_qkv, 16, kBT, 32) ||
-            !make_tensor_map_thd(&m.v_tail, v, total_tokens, n_heads, D, ts_qkv, hs_qkv, 16, kBT, 32) ||
-            !make_tensor_map_thd(&m.dout_tail, dout, total_tokens, n_heads, D, ts_o, hs_o, 16, kQS, 32) ||
-            !make_tensor_map_thd(&m.dq_acc_tail, dq_acc, total_tokens, n_heads, D, int64_t(n_heads) * D, D, 16, kBT, 64, 4))
-            return MPIPE_ERR_CUDA;
-    }
     if (!ensure_dynamic_smem<attn_bwd_kernel<D>>(Cfg::kSmemAlloc)) return MPIPE_ERR_CUDA;
     const int64_t rows = int64_t(total_tokens) * n_heads;
     const int64_t prepass_blocks = (rows + (D == 64 ? 32 : 16) - 1) / (D == 64 ? 32 : 16);

@@ -122,10 +122,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         return round * g + ((round & 1) ? g - 1 - i : i);
     };
     // Items are clamped to the tensors before use (see sanitize_item): a corrupt plan cannot make a store leave them.
-    auto item_at = [&](int u) {
+    auto item_at = [&](int u) {   // the raw item, loaded one unit ahead of its use
         mpipe_work_item_t z = {0, 0, 0, 0, 0, 0};
-        if (u >= n_units) return z;
-        z = p.items[u / p.n_heads];
+        return (u < n_units) ? p.items[u / p.n_heads] : z;
+    };
+    auto checked = [&](mpipe_work_item_t z, int u) {   // clamped at the point of use, so that the load stays off the critical path
         if (sanitize_item(z, 2 * kTileM, p.total_tokens) && tid == 4 * 32) report_status(p.status_buf, MPIPE_ERR_INDEX, u);
         return z;
     };
@@ -138,7 +139,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             bool ok = true;
             mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
-                const mpipe_work_item_t it = it_next;
+                const mpipe_work_item_t it = checked(it_next, u);
                 it_next = item_at(unit_of(ur + 1));
                 const int head = u % p.n_heads;
                 const bool two = it.row_len > kTileM;
@@ -218,7 +219,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             };
             mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
-                const mpipe_work_item_t it = it_next;
+                const mpipe_work_item_t it = checked(it_next, u);
                 it_next = item_at(unit_of(ur + 1));
                 const bool two = it.row_len > kTileM;
                 const int nkv = (it.kv_len + kTileN - 1) / kTileN;
@@ -300,7 +301,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         bool ok = true;
         mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
         for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
-            const mpipe_work_item_t it = it_next;
+            const mpipe_work_item_t it = checked(it_next, u);
             it_next = item_at(unit_of(ur + 1));
             const int head = u % p.n_heads;
             const int rows_here = it.row_len - w * kTileM;  // valid rows of this tile

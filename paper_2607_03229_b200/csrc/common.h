@@ -26,6 +26,11 @@ inline bool ensure_dynamic_smem(int bytes) {
     return true;
 }
 
+// Defined in gemm.cu, used by the layer forward: one projection that stores both GELU(u) and u.
+int32_t linear_fwd_gelu_keep_preact(const void* a, const void* w, const void* bias, void* act, void* pre, int32_t M, int32_t N,
+                                    int32_t K, int64_t lda, int64_t ldw, int64_t ldact, int64_t ldpre, int32_t* status_buf,
+                                    void* stream);
+
 // Optional measurement aid (mpipe_set_profile_events): events recorded around one kernel launch.  The slots
 // are thread-local: they affect only launches made by the thread that set them, so concurrent callers of the
 // library share no mutable state.

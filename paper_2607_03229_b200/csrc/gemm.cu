@@ -47,6 +47,7 @@ struct GemmParams {
     __nv_bfloat16* C;                // [M, ldc]
     int64_t ldr, ldc;
     int32_t gelu;
+    int32_t store_pre;               // with gelu: also store the pre-activation (bf16) through map_u
     int32_t splits;                  // weight gradient: parts the contraction (token) range is cut into
     int32_t* status_buf;
 };
@@ -62,7 +63,7 @@ struct GemmBarriers {
 template <int kBMode>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
-                  const __grid_constant__ CUtensorMap map_c, const GemmParams p) {
+                  const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_u, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ GemmBarriers bars;
@@ -209,6 +210,7 @@ linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             for (int c0 = 0; c0 < kGemmBN / 2; c0 += 32, ++box_it) {
                 uint32_t v[32];
                 uint32_t out[16];
+                uint32_t pre[16];   // pre-activation of the same 32 columns (only with store_pre)
                 uint4 rcur[4];
                 uint4 xcur[4];
                 if (p.residual != nullptr) {
@@ -246,8 +248,12 @@ linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                             }
                         }
                         if (p.gelu) {
+                            if (p.store_pre) {
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);
+                                for (int i = 0; i < 4; ++i) pre[4 * g8 + i] = pack_bf16(f[2 * i], f[2 * i + 1]);
+                            }
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) f[i] = gelu_erf(f[i]);   // of the fp32 value, in both modes
                         }
                         if (p.aux != nullptr) {
                             const uint32_t xw[4] = {xcur[g8].x, xcur[g8].y, xcur[g8].z, xcur[g8].w};
@@ -286,21 +292,29 @@ linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                     }
                     continue;
                 }
-                uint8_t* box = boxes + (box_it & 1) * kGemmOutBox;
-                if (wt == 0) bulk_wait_group_read<1>();   // the store issued two boxes ago has read this box
-                named_barrier_sync(1 + wg, 128);
-                if (ok) {
+                // one [128 rows][32 bf16] box per output: the result, and before it the pre-activation if asked for
+                auto emit = [&](const CUtensorMap* map, const uint32_t (&w)[16]) {
+                    uint8_t* box = boxes + (box_it & 1) * kGemmOutBox;
+                    if (wt == 0) bulk_wait_group_read<1>();   // the store issued two boxes ago has read this box
+                    named_barrier_sync(1 + wg, 128);
+                    if (ok) {
 #pragma unroll
-                    for (int g8 = 0; g8 < 4; ++g8)
-                        *reinterpret_cast<uint4*>(box + r * 64 + ((g8 ^ ((r >> 1) & 3)) << 4)) =
-                            make_uint4(out[4 * g8], out[4 * g8 + 1], out[4 * g8 + 2], out[4 * g8 + 3]);
+                        for (int g8 = 0; g8 < 4; ++g8)
+                            *reinterpret_cast<uint4*>(box + r * 64 + ((g8 ^ ((r >> 1) & 3)) << 4)) =
+                                make_uint4(w[4 * g8], w[4 * g8 + 1], w[4 * g8 + 2], w[4 * g8 + 3]);
+                    }
+                    fence_async_smem();
+                    named_barrier_sync(1 + wg, 128);
+                    if (ok && wt == 0) {
+                        tma_store_3d(map, box, n_base + c0, 0, m0);
+                        bulk_commit_group();
+                    }
+                };
+                if (p.gelu && p.store_pre) {
+                    emit(&map_u, pre);
+                    ++box_it;
                 }
-                fence_async_smem();
-                named_barrier_sync(1 + wg, 128);
-                if (ok && wt == 0) {
-                    tma_store_3d(&map_c, box, n_base + c0, 0, m0);
-                    bulk_commit_group();
-                }
+                emit(&map_c, out);
             }
         }
         if (wt == 0) bulk_wait_group<0>();   // shared memory must outlive the copy engine's reads
@@ -317,9 +331,11 @@ linear_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
 namespace mpipe {
 
 // Shared host side of the two entry points.  n_out / n_contract are the output columns and the contraction length.
+// `pre` (optional, forward with GELU only): bf16 [M, ldp] that receives the pre-activation a W^T + bias as well.
 static int32_t launch_linear(int b_mode, const void* a, const void* w, const void* bias, const void* residual, const void* aux,
                              void* c, int32_t M, int32_t n_out, int32_t n_contract, int64_t lda, int64_t ldw, int64_t ldr,
-                             int64_t ldx, int64_t ldc, int32_t gelu, int32_t* status_buf, void* stream) {
+                             int64_t ldx, int64_t ldc, int32_t gelu, int32_t* status_buf, void* stream,
+                             void* pre = nullptr, int64_t ldp = 0) {
     if (M < 0 || n_out <= 0 || n_contract <= 0) return MPIPE_ERR_INVALID_ARG;
     if (M == 0) return MPIPE_OK;
     if (a == nullptr || w == nullptr || c == nullptr) return MPIPE_ERR_INVALID_ARG;
@@ -331,10 +347,13 @@ static int32_t launch_linear(int b_mode, const void* a, const void* w, const voi
         return MPIPE_ERR_UNSUPPORTED;
     if (!aligned16(a) || !aligned16(w) || !aligned16(c) || !aligned16(bias) || !aligned16(residual) || !aligned16(aux))
         return MPIPE_ERR_UNSUPPORTED;
+    if (pre != nullptr && (b_mode != 0 || !gelu || ldp < n_out || (ldp % 8) != 0 || !aligned16(pre))) return MPIPE_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    CUtensorMap map_a, map_w, map_c;
+    CUtensorMap map_a, map_w, map_c, map_u;
     bool ok = make_tensor_map_thd(&map_a, a, M, 1, n_contract, lda, lda, kGemmBK, kGemmBM, 128) &&
               make_tensor_map_thd(&map_c, c, M, 1, n_out, ldc, ldc, 32, kGemmBM, 64);
+    map_u = map_c;
+    if (pre != nullptr) ok = ok && make_tensor_map_thd(&map_u, pre, M, 1, n_out, ldp, ldp, 32, kGemmBM, 64);
     if (b_mode == 0)   // W[n_out rows, n_contract columns]: boxes of 256 rows x 64 k
         ok = ok && make_tensor_map_thd(&map_w, w, n_out, 1, n_contract, ldw, ldw, kGemmBK, kGemmBN, 128);
     else               // W[n_contract rows, n_out columns]: boxes of 64 contraction rows x 64 output columns
@@ -350,6 +369,7 @@ static int32_t launch_linear(int b_mode, const void* a, const void* w, const voi
     p.C = static_cast<__nv_bfloat16*>(c);
     p.ldr = ldr; p.ldx = ldx; p.ldc = ldc;
     p.gelu = gelu;
+    p.store_pre = pre != nullptr ? 1 : 0;
     p.splits = 1;
     p.status_buf = status_buf;
     const long long tiles = (long long)p.tiles_m * p.tiles_n;
@@ -357,10 +377,10 @@ static int32_t launch_linear(int b_mode, const void* a, const void* w, const voi
     profile_start(kProfileLinear, st);
     if (b_mode == 0) {
         if (!ensure_dynamic_smem<linear_kernel<0>>(kGemmSmem)) return MPIPE_ERR_CUDA;
-        linear_kernel<0><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, p);
+        linear_kernel<0><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, map_u, p);
     } else {
         if (!ensure_dynamic_smem<linear_kernel<1>>(kGemmSmem)) return MPIPE_ERR_CUDA;
-        linear_kernel<1><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, p);
+        linear_kernel<1><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, map_u, p);
     }
     profile_stop(kProfileLinear, st);
     return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
@@ -387,6 +407,7 @@ static int32_t launch_wgrad(const void* dy, const void* x, float* dw, int32_t to
     p.bias = nullptr; p.residual = nullptr; p.aux = nullptr; p.C = nullptr;
     p.ldr = p.ldx = p.ldc = 0;
     p.gelu = 0;
+    p.store_pre = 0;
     p.status_buf = status_buf;
     // split the token range so that (tiles x splits) fills whole waves of the SMs; more splits mean more reduction traffic
     const int sms = sm_count(), tiles = p.tiles_m * p.tiles_n, nk = cdiv(tokens, kGemmBK);
@@ -403,9 +424,17 @@ static int32_t launch_wgrad(const void* dy, const void* x, float* dw, int32_t to
     const int grid = int(items < sms ? items : sms);
     if (!ensure_dynamic_smem<linear_kernel<2>>(kGemmSmem)) return MPIPE_ERR_CUDA;
     profile_start(kProfileLinear, st);
-    linear_kernel<2><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, p);
+    linear_kernel<2><<<grid, kGemmThreads, kGemmSmem, st>>>(map_a, map_w, map_c, map_c, p);
     profile_stop(kProfileLinear, st);
     return cudaGetLastError() == cudaSuccess ? MPIPE_OK : MPIPE_ERR_CUDA;
+}
+
+// fc1 of a TRAINED layer forward: act = GELU(a W^T + bias) and pre = a W^T + bias from ONE accumulator, so that the
+// activation is computed from the same fp32 value as in the FROZEN forward (freezing changes no forward bit).
+int32_t linear_fwd_gelu_keep_preact(const void* a, const void* w, const void* bias, void* act, void* pre, int32_t M, int32_t N,
+                                    int32_t K, int64_t lda, int64_t ldw, int64_t ldact, int64_t ldpre, int32_t* status_buf,
+                                    void* stream) {
+    return launch_linear(0, a, w, bias, nullptr, nullptr, act, M, N, K, lda, ldw, 0, 0, ldact, 1, status_buf, stream, pre, ldpre);
 }
 
 }  // namespace mpipe

@@ -290,22 +290,6 @@ __global__ void __launch_bounds__(256) colsum_kernel(const __nv_bfloat16* __rest
     }
 }
 
-// f = GELU(u), element-wise over a contiguous bf16 array (16 bytes per thread).  Used by a trained forward, which keeps
-// the pre-activation u for the backward and therefore cannot fuse the activation into the projection's epilogue.
-__global__ void __launch_bounds__(256) gelu_kernel(const uint4* __restrict__ u, uint4* __restrict__ f, int64_t n_chunks) {
-    const int64_t i = int64_t(blockIdx.x) * 256 + threadIdx.x;
-    if (i >= n_chunks) return;
-    const uint4 q = u[i];
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-    uint32_t o[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const __nv_bfloat162 pk = __floats2bfloat162_rn(gelu_erf(__uint_as_float(w[j] << 16)), gelu_erf(__uint_as_float(w[j] & 0xffff0000u)));
-        o[j] = *reinterpret_cast<const uint32_t*>(&pk);
-    }
-    f[i] = make_uint4(o[0], o[1], o[2], o[3]);
-}
-
 static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 
 }  // namespace mpipe
@@ -466,13 +450,9 @@ int32_t mpipe_encoder_layer_fwd(const void* x, void* y, const mpipe_layer_weight
     if ((rc = mpipe_linear_fwd(attn, w->w_o, w->b_o, x, x1, n_tokens, hidden, hidden, hidden, hidden, hidden, hidden, 0,
                                status_buf, stream)) != MPIPE_OK) return rc;
     if ((rc = mpipe_layernorm_fwd(x1, w->ln2_gamma, w->ln2_beta, norm, n_tokens, hidden, hidden, hidden, ln_eps, stream)) != MPIPE_OK) return rc;
-    if (mode == MPIPE_ENC_TRAINED) {   // the backward needs the pre-activation: keep it, apply the activation separately
-        if ((rc = mpipe_linear_fwd(norm, w->w_fc1, w->b_fc1, nullptr, ubuf, n_tokens, ffn, hidden, hidden, hidden, 0, ffn, 0,
-                                   status_buf, stream)) != MPIPE_OK) return rc;
-        const int64_t n_chunks = int64_t(t) * ffn / 8;
-        gelu_kernel<<<int((n_chunks + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
-            reinterpret_cast<const uint4*>(ubuf), reinterpret_cast<uint4*>(fc1), n_chunks);
-        if (cudaGetLastError() != cudaSuccess) return MPIPE_ERR_CUDA;
+    if (mode == MPIPE_ENC_TRAINED) {   // the backward needs the pre-activation: the same launch stores it beside GELU(u)
+        if ((rc = linear_fwd_gelu_keep_preact(norm, w->w_fc1, w->b_fc1, fc1, ubuf, n_tokens, ffn, hidden, hidden, hidden, ffn, ffn,
+                                              status_buf, stream)) != MPIPE_OK) return rc;
     } else if ((rc = mpipe_linear_fwd(norm, w->w_fc1, w->b_fc1, nullptr, fc1, n_tokens, ffn, hidden, hidden, hidden, 0, ffn,
                                       MPIPE_LINEAR_GELU, status_buf, stream)) != MPIPE_OK) {
         return rc;

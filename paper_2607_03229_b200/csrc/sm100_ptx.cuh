@@ -174,6 +174,13 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
         : "memory");
 }
 
+// Copy 128 rows x 32 bytes from shared memory (matrix descriptor as for a K-major MMA operand: one K-step of 16 bf16)
+// into 8 consecutive TMEM columns of the 128 lanes, lane = row.  Issued by one thread; executes in order with the
+// tcgen05.mma instructions that thread issues before and after it.
+__device__ __forceinline__ void tmem_cp_128x256b(uint32_t taddr, uint64_t s_desc) {
+    asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(taddr), "l"(s_desc) : "memory");
+}
+
 // Instruction descriptor of tcgen05.mma.kind::f16 with bf16 operands and fp32 accumulation.
 // a_mn / b_mn = 1 selects an MN-major (transposed) operand in shared memory.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, int a_mn, int b_mn) {
@@ -199,6 +206,7 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr, uint32_t 
     return d;
 }
 constexpr uint32_t kSwizzle128 = 2;
+constexpr uint32_t kSwizzle64 = 4;
 constexpr uint32_t kSwizzle32 = 6;
 
 // The same descriptor as two 32-bit halves, so that the issuing loop only adds a constant to the low
