@@ -113,10 +113,12 @@ size_t mpipe_attn_workspace_bytes(int32_t total_tokens, int32_t n_heads, int32_t
  *                    items, which carry the same boundaries, and do not read it)
  *   fwd_items_dev    device mpipe_work_item_t[n_fwd_items] from mpipe_seg_plan with
  *                    fwd_tile_rows = mpipe_fwd_tile_rows().  The host cannot inspect device memory at
- *                    launch time, so the kernel clamps every item to [0, total_tokens) rows before use:
- *                    an item that does not fit (a plan made for another total_tokens, a corrupted
- *                    buffer) sets status_buf[0] = MPIPE_ERR_INDEX, status_buf[1] = the unit index, and
- *                    whatever part of it lies outside the tensors is neither read nor written.
+ *                    launch time, so the kernel checks the whole list before it does anything else:
+ *                    every item's row range and key range must be non-empty and lie inside
+ *                    [0, total_tokens), the row range at most one tile.  If one does not (a plan made
+ *                    for another total_tokens, a corrupted buffer) the plan is rejected as a whole:
+ *                    status_buf[0] = MPIPE_ERR_INDEX, status_buf[1] = the index of a bad item, and the
+ *                    kernel returns without reading or writing any tensor.
  *   total_tokens == 0 or n_fwd_items == 0: returns MPIPE_OK without launching.
  * Rows past a segment's end inside a tile are computed but never stored.  fp32 accumulation,
  * bf16 probabilities; results are deterministic run to run.
@@ -140,7 +142,8 @@ int32_t mpipe_varlen_attn_fwd(const void* q, const void* k, const void* v, void*
  *   workspace      device, >= mpipe_attn_workspace_bytes(...), 256-byte aligned; contents are scratch
  *                  (fp32 dQ accumulator + Delta).  The alignment is a requirement of the TMA tensor map
  *                  through which the accumulator is updated.
- *   Items are clamped to [0, total_tokens) on the device exactly as in the forward (MPIPE_ERR_INDEX).
+ *   The item list is checked on the device exactly as in the forward (MPIPE_ERR_INDEX); a rejected plan leaves dk
+ *   and dv untouched and dq all zeros (its accumulator is cleared and converted independently of the plan).
  * dQ is summed over key tiles in fp32 by the copy engine (TMA reduce-add from shared memory); the order
  * of those additions is not fixed, so the low bits of dQ may differ from run to run.  dK and dV are
  * reproducible at head_dim 64.

@@ -92,6 +92,12 @@ struct BwdCfg {
     static constexpr int kSmemAlloc = kSmemTotal + 1024;
     // TMEM columns; P^T / dS^T (bf16) overlay the first 32 columns of each warpgroup's 64-column half of S^T / dP^T
     static constexpr int kColS = 0, kColDP = 128, kColDV = 256, kColDK = 256 + D, kColDQ = 256 + 2 * D;
+    // head_dim 64 leaves 64 columns: P^T (128 queries as bf16) gets them instead of overlaying S^T.  The next step's
+    // S^T can then be issued as soon as the softmax warps have READ the current one, not only after dV has consumed
+    // P^T, which takes the issuing thread and the tensor pipe out of the softmax warps' step-to-step loop.
+    static constexpr bool kPSeparate = (kColDQ + D + kBQ / 2 <= 512);
+    static constexpr int kColP = kPSeparate ? kColDQ + D : kColS;
+    static constexpr int kPStride = kPSeparate ? kQH / 2 : kQH;   // columns between the two warpgroups' halves of P^T
     static_assert(kSmemAlloc <= 227 * 1024, "shared memory budget");
     static_assert(kColDQ + D <= 512, "TMEM budget");
 };
@@ -110,7 +116,7 @@ struct BwdParams {
 struct BwdBarriers {
     uint64_t kv_full[2], kv_empty[2], dkv_full, dkv_empty;
     uint64_t qdo_full[4], qdo_empty[4];
-    uint64_t s_full, p_full, dp_full, ds_full, dq_full, dq_empty;
+    uint64_t s_full, s_read, p_full, pv_done, dp_full, ds_full, dq_full, dq_empty;
 };
 
 struct BwdMaps {
@@ -145,6 +151,8 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             mbar_init(&bars.qdo_empty[s], 1);
         }
         mbar_init(&bars.s_full, 1);
+        mbar_init(&bars.s_read, 8);             // (separate P^T only) S^T is in the softmax warps' registers
+        mbar_init(&bars.pv_done, 1);            // (separate P^T only) dV has consumed P^T
         mbar_init(&bars.p_full, 8);             // one arrival per softmax warp
         mbar_init(&bars.dp_full, 1);
         mbar_init(&bars.ds_full, 8);
@@ -168,22 +176,19 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
-    const int n_units = p.n_items * p.n_heads;
+    // The plan comes from device memory: it is checked as a whole before any role starts (see plan_ok_cta); a
+    // rejected plan leaves every role with nothing to do.
+    __shared__ int plan_flag;
+    const int n_units = plan_ok_cta(p.items, p.n_items, kBT, p.total_tokens, p.status_buf, &plan_flag) ? p.n_items * p.n_heads : 0;
     // Units are sorted by decreasing cost; CTAs walk them in boustrophedon order (0..G-1, then G-1..0, ...) so
     // that the CTA that got the most expensive unit of one round gets the cheapest of the next.
     auto unit_of = [&](int round) {
         const int g = int(gridDim.x), i = int(blockIdx.x);
         return round * g + ((round & 1) ? g - 1 - i : i);
     };
-    // Items are clamped to the tensors before use (see sanitize_item): a corrupt plan cannot make a store, a
-    // reduction or an LSE / Delta read leave them.
-    auto item_at = [&](int u) {   // the raw item, loaded one unit ahead of its use
+    auto item_at = [&](int u) {
         mpipe_work_item_t z = {0, 0, 0, 0, 0, 0};
         return (u < n_units) ? p.items[u / p.n_heads] : z;
-    };
-    auto checked = [&](mpipe_work_item_t z, int u) {   // clamped at the point of use, so that the load stays off the critical path
-        if (sanitize_item(z, kBT, p.total_tokens) && tid == 12 * 32) report_status(p.status_buf, MPIPE_ERR_INDEX, u);
-        return z;
     };
     // Steps of a unit: the 128-query tiles of the segment; rows of the last one past the segment end contribute
     // nothing because their probabilities are forced to zero.
@@ -202,7 +207,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             };
             mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
-                const mpipe_work_item_t it = checked(it_next, u);
+                const mpipe_work_item_t it = it_next;
                 it_next = item_at(unit_of(ur + 1));
                 const int head = u % p.n_heads;
                 const int nq = steps_of(it);
@@ -263,11 +268,11 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 }
             };
             // dst[128 keys x D] (+)= A^T-in-TMEM[128 keys x 128 q] * B[128 q x D] (B rows = q, MN-major)
-            auto issue_ts = [&](uint32_t dcol, uint32_t acol, uint32_t b_mn, bool acc) {
+            auto issue_ts = [&](uint32_t dcol, uint32_t acol, uint32_t astride, uint32_t b_mn, bool acc) {
                 if (leader) {
 #pragma unroll
                     for (int ks = 0; ks < kBQ / 16; ++ks)
-                        umma_ts(tmem + dcol, tmem + acol + (ks >> 2) * kQH + (ks & 3) * 8, umma_desc(b_mn + ks * kMnStep, hi_t), idesc_ts,
+                        umma_ts(tmem + dcol, tmem + acol + (ks >> 2) * astride + (ks & 3) * 8, umma_desc(b_mn + ks * kMnStep, hi_t), idesc_ts,
                                 (acc || ks > 0) ? 1u : 0u);
                 }
             };
@@ -275,7 +280,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             bool ok = true;
             mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
-                const mpipe_work_item_t it = checked(it_next, u);
+                const mpipe_work_item_t it = it_next;
                 it_next = item_at(unit_of(ur + 1));
                 const int nq = steps_of(it);
                 const int kb = unit_it % Cfg::kKVBufs;
@@ -305,6 +310,21 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     const uint32_t ph = c & 1;
                     const bool cross = (j + 1 == nq) && has_next;   // step j+1 is the next unit's first
                     const bool more = (j + 1 < nq) || cross;
+                    auto issue_next_s = [&]() -> bool {   // S^T(j+1), from the next unit's K tile at a unit's last step
+                        if (cross) {   // the next unit's K/V tiles (loaded while this unit ran)
+                            if (!mbar_wait(&bars.kv_full[kb ^ 1], ((unit_it + 1) / Cfg::kKVBufs) & 1, &abort_flag)) return false;
+                        }
+                        if (!mbar_wait(&bars.qdo_full[(c + 1) % NR], ((c + 1) / NR) & 1, &abort_flag)) return false;
+                        tc_fence_after();
+                        issue_kk(Cfg::kColS, cross ? k_lo_n : k_lo, q_lo0 + stage_off(c + 1), qx_lo0 + extra_off(c + 1));
+                        if (leader) umma_commit(&bars.s_full);
+                        return true;
+                    };
+                    if (Cfg::kPSeparate && more) {   // S^T(j) has been read: S^T(j+1) may replace it at once
+                        ok = mbar_wait(&bars.s_read, ph, &abort_flag);
+                        if (ok) ok = issue_next_s();
+                        if (!ok) break;
+                    }
                     ok = mbar_wait(&bars.p_full, ph, &abort_flag);
                     if (!ok) break;
                     if (j == 0) {   // the accumulators are free: the previous unit's epilogue has read them
@@ -312,22 +332,17 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                         if (!ok) break;
                     }
                     tc_fence_after();
-                    issue_ts(Cfg::kColDV, Cfg::kColS, do_mn0 + stage_off(c), j > 0);                              // dV += P^T dO
-                    if (more) {
-                        if (cross) {   // the next unit's K/V tiles (loaded while this unit ran)
-                            ok = mbar_wait(&bars.kv_full[kb ^ 1], ((unit_it + 1) / Cfg::kKVBufs) & 1, &abort_flag);
-                            if (!ok) break;
-                        }
-                        ok = mbar_wait(&bars.qdo_full[(c + 1) % NR], ((c + 1) / NR) & 1, &abort_flag);
+                    issue_ts(Cfg::kColDV, Cfg::kColP, Cfg::kPStride, do_mn0 + stage_off(c), j > 0);               // dV += P^T dO
+                    if (Cfg::kPSeparate) {
+                        if (leader) umma_commit(&bars.pv_done);
+                    } else if (more) {   // P^T overlays S^T: only now may S^T(j+1) be written
+                        ok = issue_next_s();
                         if (!ok) break;
-                        tc_fence_after();
-                        issue_kk(Cfg::kColS, cross ? k_lo_n : k_lo, q_lo0 + stage_off(c + 1), qx_lo0 + extra_off(c + 1));                    // S^T(j+1)
-                        if (leader) umma_commit(&bars.s_full);
                     }
                     ok = mbar_wait(&bars.ds_full, ph, &abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_ts(Cfg::kColDK, Cfg::kColDP, q_mn0 + stage_off(c), j > 0);                              // dK += dS^T Q
+                    issue_ts(Cfg::kColDK, Cfg::kColDP, kQH, q_mn0 + stage_off(c), j > 0);                              // dK += dS^T Q
                     if (leader) umma_commit(&bars.qdo_empty[c % NR]);   // also frees the LSE / Delta stage (dS^T(j) has arrived)
                     ok = mbar_wait(&bars.dq_empty, ph ^ 1, &abort_flag);   // the reducer has taken dQ(j-1) out of TMEM
                     if (!ok) break;
@@ -370,7 +385,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         };
         mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
         for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
-            const mpipe_work_item_t it = checked(it_next, u);
+            const mpipe_work_item_t it = it_next;
             it_next = item_at(unit_of(ur + 1));
             const int head = u % p.n_heads;
             const int nq = steps_of(it);
@@ -414,13 +429,14 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         const int r = ((warp & 3) << 5) | lane;
         const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
         const uint32_t t_s = tmem + lane_base + Cfg::kColS + g * kQH;
+        const uint32_t t_p = tmem + lane_base + Cfg::kColP + g * Cfg::kPStride;
         const uint32_t t_dp = tmem + lane_base + Cfg::kColDP + g * kQH;
         uint8_t* ds_row = smem + Cfg::kSmemDS + g * (kBT * 128) + r * 128;
         uint32_t sc = 0;   // global step counter at the start of the unit
         bool ok = true;
         mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
         for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
-            const mpipe_work_item_t it = checked(it_next, u);
+            const mpipe_work_item_t it = it_next;
             it_next = item_at(unit_of(ur + 1));
             const int nq = steps_of(it);
             const bool key_valid = r < it.row_len;
@@ -439,6 +455,11 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     tmem_ld32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&sr[0]));
                     tmem_ld32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[32]));
                     tmem_wait_ld();
+                    if (Cfg::kPSeparate) {   // the scores are in registers: the next step's S^T may be written
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars.s_read);
+                    }
                     const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
@@ -455,8 +476,13 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                             pk[2 * c4] = pack_bf16(pr[e], pr[e + 1]);
                             pk[2 * c4 + 1] = pack_bf16(pr[e + 2], pr[e + 3]);
                         }
-                        tmem_st16(t_s + h * 16, pk);   // over this thread's own scores, which are in registers
+                        if (Cfg::kPSeparate && h == 0 && c > 0) {   // dV(j-1) has read the previous P^T (long since, as a rule)
+                            ok = mbar_wait(&bars.pv_done, (c - 1) & 1, &abort_flag);
+                            tc_fence_after();
+                        }
+                        tmem_st16(t_p + h * 16, pk);   // (overlay: over this thread's own scores, which are in registers)
                     }
+                    if (!ok) break;
                 }
                 tmem_wait_st();
                 tc_fence_before();
@@ -516,7 +542,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         bool ok = true;
         mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
         for (int ur = 0, u = unit_of(0); u < n_units; ++ur, u = unit_of(ur), ++unit_it) {
-            const mpipe_work_item_t it = checked(it_next, u);
+            const mpipe_work_item_t it = it_next;
             it_next = item_at(unit_of(ur + 1));
             const int head = u % p.n_heads;
             const int nq = steps_of(it);
@@ -551,15 +577,15 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                     if (rt == 0) bulk_wait_group_read<1>();
                     named_barrier_sync(1, 128);
                     if (rt == 0) {
-                        if (ok && it.seg >= 0) tma_reduce_add_3d(&maps.dq_acc, box, 16 * ch, head, q0);
-                        bulk_commit_group();   // (an empty group when nothing was issued keeps the round count in step)
+                        if (ok) tma_reduce_add_3d(&maps.dq_acc, box, 16 * ch, head, q0);
+                        bulk_commit_group();   // (an empty group after a time-out keeps the round count in step)
                     }
                 }
             }
             if (ok) ok = mbar_wait<kSleepAux>(&bars.dkv_full, unit_it & 1, &abort_flag);
             if (!ok) continue;   // keep walking the units so that the named barriers above stay matched
             tc_fence_after();
-            const bool store = r < it.row_len && it.seg >= 0;
+            const bool store = r < it.row_len;
             const int64_t tok = int64_t(it.row_start) + r;
             __nv_bfloat16* dv_row = p.dv + tok * p.tok_stride_g + int64_t(head) * p.head_stride_g;
             __nv_bfloat16* dk_row = p.dk + tok * p.tok_stride_g + int64_t(head) * p.head_stride_g;

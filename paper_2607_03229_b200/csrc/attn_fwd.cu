@@ -114,21 +114,19 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
     // TMEM columns: S_0 [0,128), S_1 [128,256), O_0 [256,256+D), O_1 [384,384+D); P_w overlays S_w.
-    const int n_units = p.n_items * p.n_heads;
+    // The plan comes from device memory: it is checked as a whole before any role starts (see plan_ok_cta); a
+    // rejected plan leaves every role with nothing to do.
+    __shared__ int plan_flag;
+    const int n_units = plan_ok_cta(p.items, p.n_items, 2 * kTileM, p.total_tokens, p.status_buf, &plan_flag) ? p.n_items * p.n_heads : 0;
     // Units are sorted by decreasing cost; CTAs walk them in boustrophedon order (0..G-1, then G-1..0, ...) so
     // that the CTA that got the most expensive unit of one round gets the cheapest of the next.
     auto unit_of = [&](int round) {
         const int g = int(gridDim.x), i = int(blockIdx.x);
         return round * g + ((round & 1) ? g - 1 - i : i);
     };
-    // Items are clamped to the tensors before use (see sanitize_item): a corrupt plan cannot make a store leave them.
-    auto item_at = [&](int u) {   // the raw item, loaded one unit ahead of its use
+    auto item_at = [&](int u) {
         mpipe_work_item_t z = {0, 0, 0, 0, 0, 0};
         return (u < n_units) ? p.items[u / p.n_heads] : z;
-    };
-    auto checked = [&](mpipe_work_item_t z, int u) {   // clamped at the point of use, so that the load stays off the critical path
-        if (sanitize_item(z, 2 * kTileM, p.total_tokens) && tid == 4 * 32) report_status(p.status_buf, MPIPE_ERR_INDEX, u);
-        return z;
     };
 
     if (warp == 0) {
@@ -139,7 +137,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             bool ok = true;
             mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
-                const mpipe_work_item_t it = checked(it_next, u);
+                const mpipe_work_item_t it = it_next;
                 it_next = item_at(unit_of(ur + 1));
                 const int head = u % p.n_heads;
                 const bool two = it.row_len > kTileM;
@@ -219,7 +217,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             };
             mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
-                const mpipe_work_item_t it = checked(it_next, u);
+                const mpipe_work_item_t it = it_next;
                 it_next = item_at(unit_of(ur + 1));
                 const bool two = it.row_len > kTileM;
                 const int nkv = (it.kv_len + kTileN - 1) / kTileN;
@@ -301,7 +299,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         bool ok = true;
         mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
         for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
-            const mpipe_work_item_t it = checked(it_next, u);
+            const mpipe_work_item_t it = it_next;
             it_next = item_at(unit_of(ur + 1));
             const int head = u % p.n_heads;
             const int rows_here = it.row_len - w * kTileM;  // valid rows of this tile
@@ -390,7 +388,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             ++ocnt;
             tc_fence_after();
             const float inv_l = 1.0f / l;
-            const bool store = r < rows_here && it.seg >= 0;
+            const bool store = r < rows_here;
             const int64_t tok = int64_t(it.row_start) + w * kTileM + r;
             __nv_bfloat16* orow = p.o + tok * p.tok_stride_o + int64_t(head) * p.head_stride_o;
 #pragma unroll

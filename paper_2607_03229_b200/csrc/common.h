@@ -51,30 +51,27 @@ __device__ __forceinline__ void report_status(int32_t* status_buf, int32_t code,
     if (status_buf != nullptr && atomicCAS(status_buf, 0, code) == 0) status_buf[1] = detail;
 }
 
-// Work items are read from device memory that the host cannot inspect when it launches.  Every range of an
-// item is therefore clamped to the tensors (token rows [0, T), at most tile_rows rows per item), so that no
-// load, store or reduction derived from it can leave them.  An item that is empty after clamping is replaced
-// by a one-token stand-in whose results are not stored (seg = -1): the pipeline then runs a regular unit and
-// every role keeps the same trip counts.  Returns true if the item had to be altered; the caller reports
-// MPIPE_ERR_INDEX.  A plan made by mpipe_seg_plan for the same total_tokens is never altered.
-__device__ __forceinline__ bool sanitize_item(mpipe_work_item_t& it, int32_t tile_rows, int32_t T) {
-    const mpipe_work_item_t in = it;
-    // intersection of [start, start + len) with [0, T), in 64-bit so that no sum wraps
-    const int64_t r0 = max(int64_t(in.row_start), int64_t(0)), r1 = min(int64_t(in.row_start) + in.row_len, int64_t(T));
-    const int64_t k0 = max(int64_t(in.kv_start), int64_t(0)), k1 = min(int64_t(in.kv_start) + in.kv_len, int64_t(T));
-    it.row_start = int32_t(min(r0, int64_t(T)));
-    it.row_len = int32_t(min(max(r1 - r0, int64_t(0)), int64_t(tile_rows)));
-    it.kv_start = int32_t(min(k0, int64_t(T)));
-    it.kv_len = int32_t(max(k1 - k0, int64_t(0)));
-    bool altered = in.seg < 0 || it.row_start != in.row_start || it.row_len != in.row_len ||
-                   it.kv_start != in.kv_start || it.kv_len != in.kv_len;
-    if (it.row_len == 0 || it.kv_len == 0 || in.seg < 0) {
-        it.seg = -1;
-        it.row_start = it.kv_start = 0;
-        it.row_len = it.kv_len = 1;
-        altered = true;
-    }
-    return altered;
+// Work items are read from device memory that the host cannot inspect when it launches, so every CTA checks
+// the whole list before it does anything else: an item is acceptable if its row range and its key range are
+// non-empty, lie inside [0, T) and the row range is at most one tile.  One bad item rejects the plan as a whole --
+// the kernel reports MPIPE_ERR_INDEX with the item's index and returns without reading or writing a tensor --
+// which keeps every check out of the pipeline's loops.  A plan made by mpipe_seg_plan for the same total_tokens
+// always passes.
+__device__ __forceinline__ bool plan_item_ok(const mpipe_work_item_t& it, int32_t tile_rows, int32_t T) {
+    return it.row_start >= 0 && it.row_len >= 1 && it.row_len <= tile_rows && it.row_start <= T - it.row_len &&
+           it.kv_start >= 0 && it.kv_len >= 1 && it.kv_start <= T - it.kv_len;
+}
+// Returns true if every item passes.  All threads of the CTA must call it; `flag` is a shared-memory word.
+__device__ __noinline__ bool plan_ok_cta(const mpipe_work_item_t* items, int32_t n_items, int32_t tile_rows, int32_t T,
+                                            int32_t* status_buf, int* flag) {
+    if (threadIdx.x == 0) *flag = -1;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_items; i += blockDim.x)
+        if (!plan_item_ok(items[i], tile_rows, T)) atomicMax(flag, i);
+    __syncthreads();
+    const int bad = *flag;
+    if (bad >= 0 && blockIdx.x == 0 && threadIdx.x == 0) report_status(status_buf, MPIPE_ERR_INDEX, bad);
+    return bad < 0;
 }
 
 }  // namespace mpipe

@@ -1,6 +1,7 @@
-"""The work items reach the kernels through device memory the host cannot inspect at launch, so the kernels clamp
-them to the tensors.  These tests hand the attention calls plans that do not fit the tensors and check that nothing
-outside the tensors is written, that MPIPE_ERR_INDEX is reported, and that everything that does fit is still right.
+"""The work items reach the kernels through device memory the host cannot inspect at launch, so each kernel checks
+the whole list before doing anything else and rejects a plan that does not fit the tensors.  These tests hand the
+attention calls such plans and check that nothing at all is written, inside or outside the tensors, and that
+MPIPE_ERR_INDEX is reported with the index of an offending item.
 
 Every out-of-range row used here lies inside canary padding allocated around the outputs (and the inputs are read
 through TMA, which fills out-of-range rows with zeros), so not even a missing guard could touch unowned memory."""
@@ -42,49 +43,66 @@ def _run(plan, q, k, v, do, scale):
     return o, lse, [g[1] for g in gbufs], st_f.cpu().tolist(), st_b.cpu().tolist()
 
 
+def _untouched(o, lse, grads):
+    """O, LSE, dK, dV keep their fill values; dQ is all zeros (the accumulator is cleared and converted by the two
+    helper kernels, which do not depend on the plan, and no item has added to it)."""
+    dq, dk, dv = grads
+    return bool(torch.all(o == 777.0) and torch.all(lse == -555.0) and torch.all(dk == 333.0) and torch.all(dv == 333.0)
+                and torch.all(dq == 0.0))
+
+
 @pytest.mark.parametrize("D", [64, 80])
-def test_plan_made_for_more_tokens_is_clamped_and_flagged(D):
-    """The plan's last segment is 40 tokens longer than the tensors: its items overrun them by 40 rows.  Clamped to
-    the tensors the items describe segments of 300 and 200 tokens, so the results must be those."""
+def test_plan_made_for_more_tokens_is_rejected(D):
+    """The plan's last segment is 40 tokens longer than the tensors: its last items overrun them by 40 rows."""
     H, T, scale = 2, 500, float(np.float32(1.0 / np.sqrt(D)))
     q, k, v, do = (W.normal_bf16(91, s, (T, H, D)) for s in (1, 2, 3, 4))
     plan = B.seg_plan([300, 240], B.TRAINED)
     assert plan.total_tokens == 540
     plan.total_tokens = T          # what the caller claims; the items still name rows up to 540
     plan.to_device()
-    o, lse, (dq, dk, dv), st_f, st_b = _run(plan, q, k, v, do, scale)
+    o, lse, grads, st_f, st_b = _run(plan, q, k, v, do, scale)
     assert st_f[0] == B.ERR_INDEX and st_b[0] == B.ERR_INDEX
-    cu = np.array([0, 300, 500], dtype=np.int32)
-    O_ref, L_ref = oracle.attn_fwd(q, k, v, cu, scale)
-    assert max_abs(to_f64(o), O_ref) <= O_MAX_ABS and rel_l2(to_f64(o), O_ref) <= O_REL_L2
-    assert max_abs(to_f64(lse), L_ref) <= LSE_MAX_ABS
-    for g, r in zip((dq, dk, dv), oracle.attn_bwd(do, q, k, v, cu, scale)):
-        assert rel_l2(to_f64(g), r) <= GRAD_REL_L2
+    assert plan.fwd_items[st_f[1]]["seg"] == 1 and plan.bwd_items[st_b[1]]["seg"] == 1     # an item of the long segment
+    assert _untouched(o, lse, grads)
 
 
-def test_items_outside_the_tensors_store_nothing():
-    """Items that lie wholly behind the tensors' end or before their start (inside the padding) are replaced by a
-    stand-in unit that stores nothing; the other items are unaffected."""
+def test_items_outside_the_tensors_reject_the_plan():
+    """One item moved wholly behind the tensors' end (forward list) or before their start (backward list), inside
+    the padding: the plan is rejected, nothing is written, the status names the item."""
     H, D, scale = 2, 64, 0.125
     counts = [200, 150, 90]
     T = sum(counts)
     q, k, v, do = (W.normal_bf16(92, s, (T, H, D)) for s in (1, 2, 3, 4))
     plan = B.seg_plan(counts, B.TRAINED)
-    # the 90-token segment's item: forward, moved 8 rows behind the tensors' end; backward, moved to end 10 rows
-    # before their start
-    for items, victim_seg, start in ((plan.fwd_items, 2, T + 8), (plan.bwd_items, 2, -100)):
-        idx = [i for i in range(items.size) if items[i]["seg"] == victim_seg][-1]
+    moved = []
+    for items, start in ((plan.fwd_items, T + 8), (plan.bwd_items, -100)):
+        idx = [i for i in range(items.size) if items[i]["seg"] == 2][-1]
         items[idx]["row_start"] = start
         items[idx]["kv_start"] = start
+        moved.append(idx)
     plan.to_device()
-    o, lse, (dq, dk, dv), st_f, st_b = _run(plan, q, k, v, do, scale)
+    o, lse, grads, st_f, st_b = _run(plan, q, k, v, do, scale)
+    assert st_f[:2] == [B.ERR_INDEX, moved[0]] and st_b[:2] == [B.ERR_INDEX, moved[1]]
+    assert _untouched(o, lse, grads)
+
+
+def test_a_good_plan_after_a_rejected_one_runs_normally():
+    """Rejection leaves no state behind: the same tensors with the right plan give the right answer."""
+    H, D, scale = 2, 64, 0.125
+    counts = [200, 150, 90]
+    T = sum(counts)
+    q, k, v, do = (W.normal_bf16(93, s, (T, H, D)) for s in (1, 2, 3, 4))
+    bad = B.seg_plan(counts, B.TRAINED)
+    bad.fwd_items[0]["kv_len"] = T + 1
+    bad.bwd_items[0]["row_len"] = 0
+    bad.to_device()
+    _, _, _, st_f, st_b = _run(bad, q, k, v, do, scale)
     assert st_f[0] == B.ERR_INDEX and st_b[0] == B.ERR_INDEX
-    a = 350                       # rows of the 90-token segment
-    assert torch.all(o[a:] == 777.0) and torch.all(lse[:, a:] == -555.0)          # never stored
-    assert torch.all(dk[a:] == 333.0) and torch.all(dv[a:] == 333.0)
+    o, lse, (dq, dk, dv), st_f, st_b = _run(B.seg_plan(counts, B.TRAINED).to_device(), q, k, v, do, scale)
+    assert st_f[0] == 0 and st_b[0] == 0
     cu = np.array([0, 200, 350, 440], dtype=np.int32)
-    O_ref, _ = oracle.attn_fwd(q, k, v, cu, scale)
-    assert rel_l2(to_f64(o[:a]), O_ref[:a]) <= O_REL_L2
-    ref = oracle.attn_bwd(do, q, k, v, cu, scale)
-    for g, r in zip((dq, dk, dv), ref):
-        assert rel_l2(to_f64(g[:a]), r[:a]) <= GRAD_REL_L2
+    O_ref, L_ref = oracle.attn_fwd(q, k, v, cu, scale)
+    assert max_abs(to_f64(o), O_ref) <= O_MAX_ABS and rel_l2(to_f64(o), O_ref) <= O_REL_L2
+    assert max_abs(to_f64(lse), L_ref) <= LSE_MAX_ABS
+    for g, r in zip((dq, dk, dv), oracle.attn_bwd(do, q, k, v, cu, scale)):
+        assert rel_l2(to_f64(g), r) <= GRAD_REL_L2
