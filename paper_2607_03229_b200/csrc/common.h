@@ -62,7 +62,7 @@ __device__ __forceinline__ bool plan_item_ok(const mpipe_work_item_t& it, int32_
            it.kv_start >= 0 && it.kv_len >= 1 && it.kv_start <= T - it.kv_len;
 }
 // Returns true if every item passes.  All threads of the CTA must call it; `flag` is a shared-memory word.
-__device__ __noinline__ bool plan_ok_cta(const mpipe_work_item_t* items, int32_t n_items, int32_t tile_rows, int32_t T,
+static __device__ __noinline__ bool plan_ok_cta(const mpipe_work_item_t* items, int32_t n_items, int32_t tile_rows, int32_t T,
                                             int32_t* status_buf, int* flag) {
     if (threadIdx.x == 0) *flag = -1;
     __syncthreads();
