@@ -47,6 +47,11 @@ struct FwdCfg {
     static constexpr int kSmemV = kSmemK + kStages * kQBytes;
     static constexpr int kSmemTotal = kSmemV + kStages * kVBytes;
     static constexpr int kSmemAlloc = kSmemTotal + 1024;              // slack for manual 1024-byte alignment
+    // TMEM: S_w at 128 w, O_w at 256 + 128 w.  head_dim 64 leaves 64 columns behind each O_w: P_w (128 keys as bf16) goes
+    // there instead of overlaying S_w, so that S_w(j+1) can be issued as soon as the softmax warps have READ S_w(j)
+    // and runs under their exponentials, instead of waiting behind P_w(j) V(j).
+    static constexpr bool kPSep = (D + kTileN / 2 <= 128);
+    static constexpr int kColP0 = kPSep ? 256 + 64 : 0, kColPStride = 128;
 };
 
 struct FwdParams {
@@ -63,7 +68,7 @@ struct FwdParams {
 struct FwdBarriers {
     uint64_t q_full, q_empty;
     uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
-    uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t s_full[2], p_full[2], o_full[2], s_read[2], pv_done[2];
 };
 
 template <int D>
@@ -97,6 +102,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             mbar_init(&bars.s_full[w], 1);
             mbar_init(&bars.p_full[w], 4);  // one arrival per softmax warp
             mbar_init(&bars.o_full[w], 1);
+            mbar_init(&bars.s_read[w], 4);   // (separate P only) S_w is in the softmax warps' registers
+            mbar_init(&bars.pv_done[w], 1);  // (separate P only) P_w V has consumed P_w and updated O_w
         }
         fence_mbar_init();
     }
@@ -203,7 +210,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const uint32_t vlo = umma_desc_lo(sbase + Cfg::kSmemV + s * Cfg::kVBytes, kTileN * 128);
                 constexpr uint32_t idesc = umma_idesc_bf16(kTileM, D, 0, 1);
                 const uint32_t d = tmem + 256 + w * 128;
-                const uint32_t pa = tmem + w * 128;
+                const uint32_t pa = tmem + Cfg::kColP0 + w * Cfg::kColPStride;
                 if (leader) {
                     if (n_keys == kTileN) {
 #pragma unroll
@@ -241,6 +248,63 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                     if (leader) umma_commit(&bars.k_empty[s]);
                     if (nkv == 1) if (leader) umma_commit(&bars.q_empty);
                 }
+                if (Cfg::kPSep) {
+                    // Order per KV tile j:  S_0(j+1) | PV_1(j-1) | S_1(j+1) | PV_0(j): each S goes out as soon as its
+                    // predecessor has been read, each PV as soon as its P is complete, and the two query tiles stay half
+                    // a pass apart.
+                    for (int j = 0; j < nkv; ++j) {
+                        const uint32_t itv = kv_it + j;
+                        const int sv = itv % NS;
+                        const bool more = (j + 1 < nkv);
+                        const int sk = (itv + 1) % NS;
+                        if (more) {
+                            ok = mbar_wait(&bars.k_full[sk], ((itv + 1) / NS) & 1, &abort_flag);
+                            if (ok) ok = mbar_wait(&bars.s_read[0], (cnt[0] + j) & 1, &abort_flag);
+                            if (!ok) break;
+                            tc_fence_after();
+                            issue_s(0, sk, cols_of(j + 1));
+                            if (leader) umma_commit(&bars.s_full[0]);
+                        }
+                        if (two && j > 0) {
+                            ok = mbar_wait(&bars.p_full[1], (cnt[1] + j - 1) & 1, &abort_flag);
+                            if (!ok) break;
+                            tc_fence_after();
+                            issue_pv(1, (itv - 1) % NS, cols_of(j - 1), j - 1 > 0);
+                            if (leader) umma_commit(&bars.pv_done[1]);
+                            if (leader) umma_commit(&bars.v_empty[(itv - 1) % NS]);
+                        }
+                        if (more) {
+                            if (two) {
+                                ok = mbar_wait(&bars.s_read[1], (cnt[1] + j) & 1, &abort_flag);
+                                if (!ok) break;
+                                tc_fence_after();
+                                issue_s(1, sk, cols_of(j + 1));
+                                if (leader) umma_commit(&bars.s_full[1]);
+                            }
+                            if (leader) umma_commit(&bars.k_empty[sk]);
+                            if (j + 2 == nkv) if (leader) umma_commit(&bars.q_empty);
+                        }
+                        ok = mbar_wait(&bars.v_full[sv], (itv / NS) & 1, &abort_flag);
+                        if (ok) ok = mbar_wait(&bars.p_full[0], (cnt[0] + j) & 1, &abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(0, sv, cols_of(j), j > 0);
+                        if (leader) umma_commit(&bars.pv_done[0]);
+                        if (!more) if (leader) umma_commit(&bars.o_full[0]);
+                        if (!two) if (leader) umma_commit(&bars.v_empty[sv]);
+                    }
+                    if (ok && two) {   // PV_1 of the unit's last KV tile
+                        const uint32_t itv = kv_it + nkv - 1;
+                        ok = mbar_wait(&bars.p_full[1], (cnt[1] + nkv - 1) & 1, &abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(1, itv % NS, cols_of(nkv - 1), nkv - 1 > 0);
+                        if (leader) umma_commit(&bars.pv_done[1]);
+                        if (leader) umma_commit(&bars.o_full[1]);
+                        if (leader) umma_commit(&bars.v_empty[itv % NS]);
+                    }
+                    if (!ok) break;
+                } else
                 for (int j = 0; j < nkv; ++j) {
                     const uint32_t itv = kv_it + j;
                     const int sv = itv % NS;
@@ -295,6 +359,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
         const uint32_t t_s = tmem + lane_base + w * 128;
         const uint32_t t_o = tmem + lane_base + 256 + w * 128;
+        const uint32_t t_p = tmem + lane_base + Cfg::kColP0 + w * Cfg::kColPStride;   // = t_s when P overlays S
         uint32_t cnt = 0, ocnt = 0;
         bool ok = true;
         mpipe_work_item_t it_next = item_at(unit_of(0));   // one unit ahead: the global load is off the unit's critical path
@@ -317,6 +382,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 tmem_ld32(t_s + 64, *reinterpret_cast<uint32_t(*)[32]>(&sr[64]));
                 tmem_ld32(t_s + 96, *reinterpret_cast<uint32_t(*)[32]>(&sr[96]));
                 tmem_wait_ld();
+                if (Cfg::kPSep) {   // the scores are in registers: S_w of the next KV tile may be written
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars.s_read[w]);
+                }
                 const int n_valid = it.kv_len - j * kTileN;
                 if (n_valid < kTileN) {
 #pragma unroll
@@ -340,9 +410,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const float m_new = grow ? m_tile : m_ref;
                 const float alpha = ex2_approx(m_ref - m_new);         // 0 on the first tile, 1 if unchanged
                 m_ref = m_new;
+                if (Cfg::kPSep && j > 0) {   // P_w V of the previous KV tile has read P_w and updated O_w (long since, as a rule)
+                    ok = mbar_wait(&bars.pv_done[w], (cnt + j - 1) & 1, &abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
                 if (j > 0 && __any_sync(0xffffffffu, grow)) {
-                    // rescale this warp's rows of the accumulator; PV(j-1) has completed (it was issued
-                    // before S(j), whose completion we just observed)
+                    // rescale this warp's rows of the accumulator; PV(j-1) has completed (overlaid P: it was issued
+                    // before S(j), whose completion we just observed; separate P: waited for above)
 #pragma unroll
                     for (int c0 = 0; c0 < D; c0 += 16) {
                         uint32_t orr[16];
@@ -371,7 +446,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         acc[(c >> 1) & 3] = add2(acc[(c >> 1) & 3], e);
                         pk[c >> 1] = pack_bf16(e.x, e.y);
                     }
-                    tmem_st16(t_s + (c0 >> 1), pk);
+                    tmem_st16(t_p + (c0 >> 1), pk);
                 }
                 const float2 s01 = add2(add2(acc[0], acc[1]), add2(acc[2], acc[3]));
                 l = l * alpha + (s01.x + s01.y);
