@@ -186,13 +186,39 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         const int g = int(gridDim.x), i = int(blockIdx.x);
         return round * g + ((round & 1) ? g - 1 - i : i);
     };
+    // Unit u -> (work item, head).  The items of one segment are consecutive in the list (tile 0, 1, ...), and their
+    // units occupy the same stretch of the unit sequence whichever way it is ordered inside.  Short segments: tile by
+    // tile, heads innermost.  Segments of more than kHeadMajorTiles key tiles: head by head, so that the CTAs running
+    // at the same time share the Q / dO tiles and the dQ accumulator of one or two heads through L2 instead of all
+    // heads' at once (16 heads x 16 384 tokens of Q, dO and fp32 dQ do not fit in L2 beside K and V; DRAM traffic of
+    // the Qwen2-VL-like backward was 6.4 x the algorithmic bytes).  The head is returned in the item's `seg` field,
+    // which the kernel does not otherwise use.
+    constexpr int kHeadMajorTiles = 32;
     auto item_at = [&](int u) {
         mpipe_work_item_t z = {0, 0, 0, 0, 0, 0};
-        return (u < n_units) ? p.items[u / p.n_heads] : z;
+        if (u >= n_units) return z;
+        const int i0 = u / p.n_heads;
+        const mpipe_work_item_t a = p.items[i0];
+        const int nt = (a.kv_len + kBT - 1) / kBT;                   // key tiles of this item's segment
+        if (nt <= kHeadMajorTiles) {
+            z = a;
+            z.seg = u % p.n_heads;
+            return z;
+        }
+        const int first = i0 - a.tile;                               // the segment's first item
+        const int l = u - first * p.n_heads;
+        const int head = l / nt;
+        z = p.items[min(max(first + (l - head * nt), 0), p.n_items - 1)];
+        z.seg = min(max(head, 0), p.n_heads - 1);
+        return z;
     };
     // Steps of a unit: the 128-query tiles of the segment; rows of the last one past the segment end contribute
     // nothing because their probabilities are forced to zero.
     auto steps_of = [](const mpipe_work_item_t& it) { return (it.kv_len + kBQ - 1) / kBQ; };
+    // The j-th step of a unit works on query tile (j + key tile index) mod steps: the CTAs that hold the key tiles of
+    // one (segment, head) run at the same time, and started on the same query tile they would all add to the same rows
+    // of the dQ accumulator at once (fp32 adds to one address serialise in L2) and ask for the same Q / dO tile.
+    auto q_tile_of = [](const mpipe_work_item_t& it, int j, int nq) { return (j + (it.tile >= 0 ? it.tile : 0)) % nq; };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -209,7 +235,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
             for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur), ++unit_it) {
                 const mpipe_work_item_t it = it_next;
                 it_next = item_at(unit_of(ur + 1));
-                const int head = u % p.n_heads;
+                const int head = it.seg;
                 const int nq = steps_of(it);
                 const int kb = unit_it % Cfg::kKVBufs;            // K/V buffer of this unit
                 uint8_t* kv = smem + kb * (2 * Cfg::kTile);
@@ -220,7 +246,7 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
                 load_tile(kv + Cfg::kSmemV, &maps.v, &bars.kv_full[kb], head, it.row_start);
                 for (int j = 0; j < nq; ++j, ++sc) {
                     const int rs = sc % NR;
-                    const int row = it.kv_start + j * kBQ;
+                    const int row = it.kv_start + q_tile_of(it, j, nq) * kBQ;
                     ok = mbar_wait<kSleepAux>(&bars.qdo_empty[rs], ((sc / NR) & 1) ^ 1, &abort_flag);
                     if (!ok) break;
                     mbar_expect_tx(&bars.qdo_full[rs], 2 * Cfg::kTile);
@@ -387,14 +413,14 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         for (int ur = 0, u = unit_of(0); u < n_units && ok; ++ur, u = unit_of(ur)) {
             const mpipe_work_item_t it = it_next;
             it_next = item_at(unit_of(ur + 1));
-            const int head = u % p.n_heads;
+            const int head = it.seg;
             const int nq = steps_of(it);
             const int q_end = it.kv_start + it.kv_len;
             for (int j = 0; j < nq; ++j, ++sc) {
                 const int rs = sc % NR;
                 uint4* qx = reinterpret_cast<uint4*>(smem + Cfg::kSmemQX + rs * Cfg::kExtra);
                 uint4* dox = reinterpret_cast<uint4*>(smem + Cfg::kSmemDOX + rs * Cfg::kExtra);
-                const int q0 = it.kv_start + j * kBQ;
+                const int q0 = it.kv_start + q_tile_of(it, j, nq) * kBQ;
                 float xv[4], yv[4];   // read from global memory before the stage is known to be free: the latency overlaps the wait
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -544,14 +570,14 @@ attn_bwd_kernel(const __grid_constant__ BwdMaps maps, const BwdParams p) {
         for (int ur = 0, u = unit_of(0); u < n_units; ++ur, u = unit_of(ur), ++unit_it) {
             const mpipe_work_item_t it = it_next;
             it_next = item_at(unit_of(ur + 1));
-            const int head = u % p.n_heads;
+            const int head = it.seg;
             const int nq = steps_of(it);
             // No early exit inside this loop: the four warps meet at named barriers, so after a time-out
             // they keep walking the (now empty) iterations together instead of leaving one another behind.
             for (int i = 0; i < nq; ++i, ++pc) {
                 if (ok) ok = mbar_wait<kSleepAux>(&bars.dq_full, pc & 1, &abort_flag);
                 tc_fence_after();
-                const int q0 = it.kv_start + i * kBQ;
+                const int q0 = it.kv_start + q_tile_of(it, i, nq) * kBQ;
                 // One round per 16 columns: read them from TMEM, write this thread's 64-byte row of box gc % 3, and
                 // after the warpgroup's barrier hand the box to the copy engine.  Box gc % 3 was last used three rounds
                 // ago; before each barrier the issuing thread waits until at most ONE reduction is still reading its
