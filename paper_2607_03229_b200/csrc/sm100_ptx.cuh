@@ -283,11 +283,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
 }
 
 // Packed pairs of fp32 (sm_100): one instruction for two lanes of a row's arithmetic.
-#ifdef MPIPE_NO_F32X2
-__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return make_float2(fmaf(a.x, b.x, c.x), fmaf(a.y, b.y, c.y)); }
-__device__ __forceinline__ float2 add2(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
-__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return make_float2(a.x * b.x, a.y * b.y); }
-#else
 __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
     float2 d;
     asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
@@ -319,7 +314,6 @@ __device__ __forceinline__ float2 mul2(float2 a, float2 b) {
     return d;
 }
 
-#endif
 
 // 2^x for a pair of values on the FMA/ALU pipes instead of the special-function unit (which delivers
 // only 16 results per clock per SM and is the forward softmax's bottleneck at head_dim 64):
