@@ -28,7 +28,6 @@ constexpr int kFwdThreads = 384;
 constexpr int kTileM = 128;        // query rows per tile (= TMEM lanes)
 constexpr int kTileN = 128;        // keys per K/V tile
 constexpr float kRescaleThreshold = 8.0f;  // in log2 units
-constexpr unsigned kPolyMask = 0x52;   // bit i: column pair i (mod 8) uses the polynomial exp2 (3 of 8)
 // setmaxnreg: the 4 light warps release what the 8 softmax warps take (an increase blocks until the CTA's
 // own pool has the registers).
 constexpr int kFwdRegsLaunch = 168, kFwdRegsLight = 56, kFwdRegsSoftmax = 224;
@@ -51,6 +50,11 @@ struct FwdCfg {
     // there instead of overlaying S_w, so that S_w(j+1) can be issued as soon as the softmax warps have READ S_w(j)
     // and runs under their exponentials, instead of waiting behind P_w(j) V(j).
     static constexpr bool kPSep = (D + kTileN / 2 <= 128);
+    // bit i: column pair i (mod 8) of a row forms its exponential with the polynomial on the FMA pipes instead of the
+    // special-function unit.  3 of 8 balances the two when the query tiles' softmax passes alternate (head_dim 80);
+    // with separate P columns the two passes run side by side and 2 of 8 measured best (all-MUFU 752, 1 of 8 781,
+    // 2 of 8 800, 3 of 8 770 TFLOP/s on the ViT-L workload).
+    static constexpr unsigned kPolyMask = kPSep ? 0x12u : 0x52u;
     static constexpr int kColP0 = kPSep ? 256 + 64 : 0, kColPStride = 128;
 };
 
@@ -441,7 +445,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                         const float2 x = fma2(make_float2(__uint_as_float(sr[c0 + c]), __uint_as_float(sr[c0 + c + 1])), sc2, nm2);
                         // kPolyMask picks, out of every 8 column pairs, those whose exponential runs on the FMA
                         // pipes; the rest use the special-function unit.  The split balances the two.
-                        const float2 e = ((kPolyMask >> ((c >> 1) & 7)) & 1) ? exp2_poly2(x)
+                        const float2 e = ((Cfg::kPolyMask >> ((c >> 1) & 7)) & 1) ? exp2_poly2(x)
                                                                            : make_float2(ex2_approx(x.x), ex2_approx(x.y));
                         acc[(c >> 1) & 3] = add2(acc[(c >> 1) & 3], e);
                         pk[c >> 1] = pack_bf16(e.x, e.y);
