@@ -21,6 +21,8 @@
  *   - "host" / "device" is stated for every pointer.  The caller owns all memory, the workspace and
  *     the CUDA stream; the library allocates no device memory.  Device calls enqueue work on `stream`
  *     (a cudaStream_t passed as void*, NULL = default stream) and return without synchronising.
+ *     They may therefore be captured in a CUDA graph and replayed (per-kernel attributes are set on a
+ *     kernel's first launch: make one plain call of each entry point before the capture).
  *   - Argument errors are detected on the host before anything is launched; outputs are untouched.
  *   - bf16 = bfloat16.  Token tensors are [tokens, heads, head_dim] with explicit token and head
  *     strides in ELEMENTS; head_dim is contiguous.  Base pointers must be 16-byte aligned and the
