@@ -312,6 +312,11 @@ def rates(w, ms_step, kern_ms, clocks, peaks):
     return out
 
 
+def repeat_count(ms_per_step: float, K: int, min_seconds: float, cap: int = 40) -> int:
+    """How many K-step regions to time so that they cover `min_seconds` of GPU time, between 1 and `cap`."""
+    return int(min(cap, max(1, np.ceil(min_seconds * 1e3 / max(ms_per_step * K, 1e-3)))))
+
+
 def pick_peak(clocks, peaks):
     """The measured peak whose clock regime matches the run.  The burst GEMM figure was taken at the maximum SM
     clock, the sustained one power-capped at about two thirds of it: a run whose median sampled clock is within
@@ -392,7 +397,10 @@ def ours_arm(args):
     # that the measurement covers at least ~2 s of GPU time (clocks settle, the sampler sees them); ms_per_step
     # is the median over the repeats and every repeat's clocks are reported.
     ms0, _, _ = timed_region(torch, B, H, w, buf, K, uuid, D.barrier)
-    R = 1 if args.profile_mode else int(min(40, max(1, np.ceil(args.min_seconds * 1e3 / max(ms0 * K, 1e-3)))))
+    # every rank must run the same number of regions (each one ends in a barrier): the count comes from the
+    # slowest rank's first region, not from this rank's
+    (ms0_all,), _ = D.reduce_max_sum([ms0], [0.0], device=dev)
+    R = 1 if args.profile_mode else repeat_count(ms0_all, K, args.min_seconds)
     repeats = [timed_region(torch, B, H, w, buf, K, uuid, D.barrier) for _ in range(R)]
     order = np.argsort([r[0] for r in repeats])
     ms_step, kern_ms, clocks = repeats[int(order[len(order) // 2])]

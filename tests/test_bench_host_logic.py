@@ -68,3 +68,11 @@ def test_rates_fractions_are_consistent():
     assert np.isclose(out["step_frac"]["of_cycle_peak_at_sampled_clock"], tf / cyc)
     assert np.isclose(out["fwd_tflops"], w.flops(True, False) / 0.6e-3 / 1e12)
     assert np.isclose(out["bwd_main_tflops"], w.flops(False, True) / 1.3e-3 / 1e12)
+
+
+def test_repeat_count_covers_the_minimum_time_within_its_bounds():
+    assert bench.repeat_count(2.0, 200, 2.0) == 5           # 0.4 s per region -> five regions
+    assert bench.repeat_count(2.0, 200, 2.1) == 6
+    assert bench.repeat_count(50.0, 200, 2.0) == 1          # one region is already longer
+    assert bench.repeat_count(0.01, 3, 2.0) == 40           # capped
+    assert bench.repeat_count(0.0, 3, 2.0) == 40            # a zero time does not divide by zero

@@ -22,7 +22,15 @@ def _worker(rank, world, port, out):
     wl = bench.workload_for(rank)
     D.barrier()
     (t_max, e_max), (flops, launches) = D.reduce_max_sum([1.0 + rank, 5.0 - rank], [wl.flops(), 5.0])
-    out.put((rank, wl.seed, wl.total_tokens, wl.flops(), t_max, e_max, flops, launches))
+    # the number of timed regions (each ends in a barrier) must be the same on every rank although their own first
+    # regions differ: it is derived from the slowest rank's time
+    ms0 = 1.9 if rank == 0 else 2.3
+    (ms0_all,), _ = D.reduce_max_sum([ms0], [0.0])
+    regions = bench.repeat_count(ms0_all, 200, 2.0)
+    assert bench.repeat_count(1.9, 200, 2.0) != bench.repeat_count(2.3, 200, 2.0)   # the local values would disagree
+    for _ in range(regions):
+        D.barrier()
+    out.put((rank, wl.seed, wl.total_tokens, wl.flops(), t_max, e_max, flops, launches, regions))
     D.shutdown()
 
 
@@ -37,7 +45,8 @@ def test_two_ranks_shard_by_microbatch_and_reduce():
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
-    (r0, s0, t0, f0, mx0, ex0, fl0, l0), (r1, s1, t1, f1, mx1, ex1, fl1, l1) = res
+    (r0, s0, t0, f0, mx0, ex0, fl0, l0, n0), (r1, s1, t1, f1, mx1, ex1, fl1, l1, n1) = res
+    assert n0 == n1 == 5
     assert s0 != s1 and (t0, f0) != (t1, f1)          # different microbatches per rank
     assert mx0 == mx1 == 2.0 and ex0 == ex1 == 5.0    # max over ranks
     assert abs(fl0 - (f0 + f1)) < 1e-3 * fl0 and fl0 == fl1 and l0 == l1 == 10.0   # work sums
